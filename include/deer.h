@@ -1,0 +1,227 @@
+/*
+ * deer.h -- C ABI of the DEER draft-verify hot path for NVIDIA B200 (sm_100a).
+ *
+ * One draft-verify cycle of the paper's inference routine (Section 3.2,
+ * Algorithm 1) is: a block of k <= 32 draft tokens proposed for the prefix
+ * x_{1:j}; the verifier's distributions p_AR(. | x_{1:j+i-1}), i = 1..k, from
+ * one parallel pass; the acceptance rule (Eq. 5, Eq. 6); the accepted tokens
+ * appended to the prefix.  This library holds the data-parallel parts of that
+ * cycle as four calls -- deer_block_attn, deer_lmhead_select, deer_accept,
+ * deer_kv_commit (with deer_kv_reserve as its counterpart) -- over a paged
+ * bf16 KV cache that represents the prefix.
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless its comment says "host".  The
+ *     caller owns all memory; the library allocates no device memory.
+ *   - Every call returns an int status (DEER_OK = 0), validates its arguments
+ *     on the host before launching, and is asynchronous on the CUDA stream
+ *     passed last as `void*` (a cudaStream_t; NULL = the default stream).
+ *   - Data-dependent failures (page pool exhausted, a page id out of range)
+ *     are written by the kernels to the cache's device status word and read
+ *     with deer_kv_status(); kernels never trap and never spin unboundedly.
+ *   - Tensors are dense, row-major, last index fastest, 16-byte aligned.
+ *     bf16 tensors are passed as `void*`.
+ *   - Shapes: B sequences in the call, k block rows (1..32), Hq query heads,
+ *     Hkv KV heads (Hq % Hkv == 0; query head h reads KV head h / (Hq/Hkv)),
+ *     D head dim (64 or 128), page size 16 tokens, M = B*k rows, V vocabulary,
+ *     hid hidden size (multiple of 64).
+ */
+#ifndef DEER_H_
+#define DEER_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DEER_OK               0
+#define DEER_ERR_INVALID_ARG  1   /* null pointer, misaligned pointer, bad size              */
+#define DEER_ERR_UNSUPPORTED  2   /* k > 32, head dim not 64/128, page size not 16, ...       */
+#define DEER_ERR_NO_PAGES     3   /* device status: reserve found too few free pages          */
+#define DEER_ERR_CUDA         4   /* a CUDA runtime call failed; see deer_last_error()        */
+#define DEER_ERR_WORKSPACE    5   /* workspace smaller than the *_workspace_bytes() figure    */
+#define DEER_ERR_BAD_PAGE     6   /* device status: a kernel met an unmapped/out-of-range page */
+
+#define DEER_MASK_CAUSAL 0   /* verifier: block row i sees block rows j <= i           */
+#define DEER_MASK_BIDIR  1   /* drafter single-step fill: every block row sees all k   */
+
+#define DEER_SEL_ARGMAX          0   /* ids only (temperature 0)                         */
+#define DEER_SEL_ARGMAX_LOGPROB  1   /* ids + fp32 log-probability of the argmax (T = 1) */
+#define DEER_SEL_SOFTMAX         2   /* ids + logsumexp(z/T) + draft-token logit (+ logits) */
+
+#define DEER_ACC_GREEDY 0
+#define DEER_ACC_SAMPLE 1
+
+#define DEER_MAX_BLOCK 32
+#define DEER_PAGE_SIZE 16
+
+/* Text of the last host-side error of the calling thread (host pointer, never NULL). */
+const char* deer_last_error(void);
+
+/* ------------------------------------------------------------------------
+ * Paged KV cache = the committed prefix x_{1:j} of each sequence
+ * (Section 3.2: "the chosen token is appended to the prefix and becomes part
+ * of the context"; Algorithm 1: j <- length(x)).
+ *
+ * State, all caller-allocated device arrays described by deer_kv_desc:
+ *   k_pool, v_pool  bf16 [num_pages][Hkv][16][D]
+ *   page_table      i32  [max_seqs][max_pages]   physical page of logical page p, -1 if unmapped
+ *   seq_len         i32  [max_seqs]              committed tokens n_s
+ *   n_pages         i32  [max_seqs]              mapped logical pages (>= ceil(n_s/16))
+ *   free_stack      i32  [num_pages]             free page ids in [0, *free_top); a pop takes the top
+ *   free_top        i32  [1]
+ *   status          i32  [1]                     0, or the first DEER_ERR_* a kernel recorded
+ * Token t of sequence s lives at pool[page_table[s][t/16]][h][t%16][:].
+ * The handle is a small host struct; destroying it frees nothing on the device.
+ * ---------------------------------------------------------------------- */
+typedef struct deer_kv deer_kv;
+
+typedef struct deer_kv_desc {
+    void*    k_pool;
+    void*    v_pool;
+    int32_t* page_table;
+    int32_t* seq_len;
+    int32_t* n_pages;
+    int32_t* free_stack;
+    int32_t* free_top;
+    int32_t* status;
+    int32_t  num_pages;
+    int32_t  n_kv_heads;
+    int32_t  head_dim;
+    int32_t  page_size;
+    int32_t  max_seqs;
+    int32_t  max_pages;
+} deer_kv_desc;
+
+/* `desc` is a host pointer; its contents are copied. */
+int deer_kv_create(deer_kv** kv, const deer_kv_desc* desc);
+int deer_kv_destroy(deer_kv* kv);
+
+/* Map pages so that each listed sequence can hold seq_len + k tokens:
+ * sequences in the order of seq_ids, logical pages ascending, each page popped
+ * from the top of the free stack.  If the free stack or max_pages is too small
+ * nothing changes and the status word becomes DEER_ERR_NO_PAGES.
+ * seq_ids: i32 [B], distinct.  B <= 1024. */
+int deer_kv_reserve(deer_kv* kv, const int32_t* seq_ids, int B, int k, void* stream);
+
+/* (4) Commit / roll back (Algorithm 1, "Update j <- length(x)"): seq_len[s] += keep[b]
+ * with keep clamped to [0, k]; block rows written at positions >= the new length
+ * are thereby dropped, and pages wholly beyond it return to the free stack --
+ * sequences in order, logical pages descending.  `keep` is a device array
+ * (e.g. deer_accept's accept_len), so no host round-trip is needed. */
+int deer_kv_commit(deer_kv* kv, const int32_t* seq_ids, const int32_t* keep, int B, int k, void* stream);
+
+/* Copy the status word to *code (host pointer) after synchronising `stream`,
+ * and reset it to 0 on the device. */
+int deer_kv_status(deer_kv* kv, int32_t* code, void* stream);
+
+/* ------------------------------------------------------------------------
+ * (1) Block attention (Section 3.2: the verifier scores all k block
+ * positions in one pass, p_AR(. | x_{1:j+i-1}); the drafter fills the k masked
+ * positions jointly from x_{1:j}).  For sequence b, head h, block row i:
+ *     out = softmax(scale * q . K^T) V
+ * over the keys {cache tokens 0..n_b-1} U {block rows j allowed by `mask`},
+ * fp32 accumulation, bf16 output.
+ *   q            bf16 [B][k][Hq][D]
+ *   k_blk,v_blk  bf16 [B][k][Hkv][D]    keys/values of the block rows themselves
+ *   out          bf16 [B][k][Hq][D]
+ *   append       1: also write k_blk/v_blk into the cache at token positions
+ *                n_b .. n_b+k-1 (pages must have been reserved); seq_len is
+ *                NOT changed -- deer_kv_commit decides how many rows survive.
+ *   max_seq_len  host-known upper bound on n_b over the batch; it only steers
+ *                how the context is split over thread blocks and sizes the
+ *                workspace.  A sequence longer than it sets DEER_ERR_INVALID_ARG
+ *                in the status word and is skipped.
+ *   workspace    >= deer_block_attn_workspace_bytes(...) bytes, 16-byte aligned;
+ *                holds the split-context partial results.
+ * ---------------------------------------------------------------------- */
+size_t deer_block_attn_workspace_bytes(int B, int k, int Hq, int Hkv, int D, int max_seq_len);
+
+int deer_block_attn(deer_kv* kv, const int32_t* seq_ids,
+                    const void* q, const void* k_blk, const void* v_blk, void* out,
+                    int B, int k, int Hq, int mask, int append, float scale, int max_seq_len,
+                    void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------
+ * (2) LM head + selection: z = h w^T (bf16 x bf16 -> fp32), the verifier's
+ * p_AR = softmax(z / T) of Eq. 5, reduced on the fly.
+ *   h  bf16 [M][hid]      w  bf16 [V][hid]
+ *   out_ids          i32 [M]  argmax_v z (lowest index among equal maxima)
+ *   out_max_logprob  f32 [M]  max z - logsumexp(z)         (DEER_SEL_ARGMAX_LOGPROB)
+ *   out_lse          f32 [M]  logsumexp(z / temperature)   (DEER_SEL_SOFTMAX)
+ *   out_draft_logit  f32 [M]  z[draft_ids[m]]              (DEER_SEL_SOFTMAX, draft_ids != NULL)
+ *   out_logits       f32 [M][V], optional in any mode (NULL = not stored)
+ * Outputs not used by `mode` may be NULL.  temperature > 0 (ignored for ARGMAX).
+ * ---------------------------------------------------------------------- */
+size_t deer_lmhead_workspace_bytes(int M, int hid, int V);
+
+int deer_lmhead_select(const void* h, const void* w, int M, int hid, int V,
+                       int mode, float temperature, const int32_t* draft_ids,
+                       int32_t* out_ids, float* out_max_logprob, float* out_lse,
+                       float* out_draft_logit, float* out_logits,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------
+ * (3) Acceptance rule (Eq. 5, Eq. 6, Algorithm 1 inner loop; the first
+ * rejection ends the block because later rows were conditioned on the
+ * rejected draft).
+ * GREEDY (temperature 0): accept_len = longest prefix with draft == target;
+ *   the emitted tokens are the accepted drafts followed, if accept_len < k, by
+ *   target_ids at the first mismatch.
+ * SAMPLE: alpha_i = min(1, p(y_i)/q(y_i)), p = softmax(target_logits/T),
+ *   q = softmax(draft_logits); accept iff u[b][i] <= alpha_i; at the first
+ *   rejection one token is drawn from max(0, p - q) normalised, by inverse CDF
+ *   in vocabulary order with r[b] (fp64 sums); if that mass is zero, from p.
+ * No extra token is emitted when all k are accepted.  If eos_id >= 0 nothing is
+ * emitted after the first emitted eos_id.
+ *   draft_ids           i32 [B][k]
+ *   target_ids          i32 [B][k]        GREEDY
+ *   target_logits       f32 [B][k][V]     SAMPLE (deer_lmhead_select's out_logits)
+ *   target_lse          f32 [B][k]        SAMPLE logsumexp(target_logits / T)
+ *   target_draft_logit  f32 [B][k]        SAMPLE target_logits[b][i][draft_ids[b][i]]
+ *   draft_logits        f32 [B][k][V]     SAMPLE
+ *   u f32 [B][k] in (0,1);  r f32 [B] in (0,1)
+ *   accept_len i32 [B];  out_ids i32 [B][k] (-1 padded);  n_out i32 [B]
+ * ---------------------------------------------------------------------- */
+size_t deer_accept_workspace_bytes(int mode, int B, int k, int V);
+
+int deer_accept(int mode, int B, int k, int V,
+                const int32_t* draft_ids, const int32_t* target_ids,
+                const float* target_logits, const float* target_lse, const float* target_draft_logit,
+                float temperature, const float* draft_logits, const float* u, const float* r,
+                int32_t eos_id, int32_t* accept_len, int32_t* out_ids, int32_t* n_out,
+                void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------
+ * One whole greedy verify step with HOST inputs and outputs (Algorithm 1, one
+ * iteration of the while loop on the verifier side): copies the block's
+ * q/k_blk/v_blk, hidden states and draft ids from host memory to the device
+ * staging buffers in `dev`, runs reserve -> block_attn(causal, append) ->
+ * lmhead_select(argmax) -> accept(greedy) -> commit(keep = accept_len), and
+ * copies accept_len / out_ids / n_out back.  Model state (w, the KV cache)
+ * stays on the device.  Returns after the stream has been synchronised.
+ * ---------------------------------------------------------------------- */
+typedef struct deer_step_dev {
+    void* q; void* k_blk; void* v_blk; void* attn_out;     /* bf16 staging, shapes as in deer_block_attn */
+    void* h;                                               /* bf16 [M][hid] */
+    int32_t* seq_ids;                                      /* i32 [B], already filled */
+    int32_t* draft_ids; int32_t* target_ids;               /* i32 [B][k] */
+    int32_t* accept_len; int32_t* out_ids; int32_t* n_out;
+    void* attn_ws; size_t attn_ws_bytes;
+    void* lm_ws;   size_t lm_ws_bytes;
+} deer_step_dev;
+
+int deer_verify_step_host(deer_kv* kv, const deer_step_dev* dev /*host struct*/,
+                          const void* w /*device bf16 [V][hid]*/,
+                          const void* q_host, const void* k_blk_host, const void* v_blk_host,
+                          const void* h_host, const int32_t* draft_ids_host,
+                          int B, int k, int Hq, int hid, int V, float scale, int max_seq_len,
+                          int32_t* accept_len_host, int32_t* out_ids_host, int32_t* n_out_host,
+                          void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DEER_H_ */

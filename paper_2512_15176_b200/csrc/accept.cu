@@ -1,0 +1,397 @@
+// (3) Acceptance rule of the draft-verify cycle (Eq. 5, Eq. 6, Algorithm 1's
+// inner loop, stopped at the first rejection).
+//
+// GREEDY: integer prefix match.
+// SAMPLE: (a) one streaming pass over the drafter logits for log-sum-exp and
+// the draft token's logit of every block row; (b) a per-sequence scan for the
+// first rejection, log alpha_i = min(0, log p(y_i) - log q(y_i)) against log u;
+// (c) for each rejected sequence the residual max(0, p - q) of that one row in
+// fp64, split over NS thread blocks, then an inverse-CDF search in vocabulary
+// order.  Only (a) touches more than a few rows.
+
+#include "common.cuh"
+
+namespace {
+
+constexpr int NS = 8;              // vocabulary slices per rejected row
+constexpr int RES_THREADS = 512;
+constexpr int LOC_THREADS = 1024;
+
+// ---------------------------------------------------------------- greedy
+__global__ void accept_greedy_kernel(int B, int k, const int32_t* __restrict__ draft, const int32_t* __restrict__ target,
+                                     int32_t eos_id, int32_t* __restrict__ accept_len, int32_t* __restrict__ out_ids,
+                                     int32_t* __restrict__ n_out) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    const int32_t* d = draft + (size_t)b * k;
+    const int32_t* t = target + (size_t)b * k;
+    int32_t* o = out_ids + (size_t)b * k;
+    int a = 0;
+    while (a < k && d[a] == t[a]) ++a;
+    int n = a < k ? a + 1 : a;
+    for (int i = 0; i < k; ++i) o[i] = i < a ? d[i] : (i == a ? t[i] : -1);
+    if (eos_id >= 0) {
+        for (int i = 0; i < n; ++i)
+            if (o[i] == eos_id) {
+                for (int j = i + 1; j < n; ++j) o[j] = -1;
+                n = i + 1;
+                a = min(a, n);
+                break;
+            }
+    }
+    accept_len[b] = a;
+    n_out[b] = n;
+}
+
+// ---------------------------------------------------------------- sample (a)
+// One block per block row: log-sum-exp of the drafter logits and the draft
+// token's logit.
+__global__ void __launch_bounds__(256) draft_row_stats_kernel(int V, const float* __restrict__ q_logits,
+                                                              const int32_t* __restrict__ draft, float* __restrict__ lse_q,
+                                                              float* __restrict__ zq_draft) {
+    const int row = blockIdx.x;
+    const float* z = q_logits + (size_t)row * V;
+    float m = -INFINITY, s = 0.f;
+    auto push = [&](float x) {
+        if (x > m) {
+            s = s * __expf(m - x) + 1.f;
+            m = x;
+        } else {
+            s += __expf(x - m);
+        }
+    };
+    if ((V & 3) == 0) {
+        const float4* z4 = reinterpret_cast<const float4*>(z);
+        for (int i = threadIdx.x; i < V / 4; i += blockDim.x) {
+            const float4 x = __ldg(z4 + i);
+            const float mx = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
+            if (mx > m) {
+                s *= __expf(m - mx);
+                m = mx;
+            }
+            s += __expf(x.x - m) + __expf(x.y - m) + __expf(x.z - m) + __expf(x.w - m);
+        }
+    } else {
+        for (int i = threadIdx.x; i < V; i += blockDim.x) push(z[i]);
+    }
+    __shared__ float sm[8], ss[8];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, m, o);
+        const float os = __shfl_xor_sync(0xffffffffu, s, o);
+        const float nm = fmaxf(m, om);
+        s = (m > -INFINITY ? s * __expf(m - nm) : 0.f) + (om > -INFINITY ? os * __expf(om - nm) : 0.f);
+        m = nm;
+    }
+    if (lane == 0) {
+        sm[warp] = m;
+        ss[warp] = s;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float M = -INFINITY;
+        for (int w = 0; w < 8; ++w) M = fmaxf(M, sm[w]);
+        float S = 0.f;
+        for (int w = 0; w < 8; ++w) S += (sm[w] > -INFINITY) ? ss[w] * __expf(sm[w] - M) : 0.f;
+        lse_q[row] = M + logf(S);
+        const int y = draft[row];
+        zq_draft[row] = (y >= 0 && y < V) ? z[y] : -INFINITY;
+    }
+}
+
+// ---------------------------------------------------------------- sample (b)
+// One warp per sequence, lane i = block row i.
+__global__ void __launch_bounds__(128) accept_scan_kernel(int B, int k, const int32_t* __restrict__ draft,
+                                                          const float* __restrict__ lse_p, const float* __restrict__ zp_draft,
+                                                          float inv_t, const float* __restrict__ lse_q,
+                                                          const float* __restrict__ zq_draft, const float* __restrict__ u,
+                                                          int32_t* __restrict__ accept_len, int32_t* __restrict__ out_ids,
+                                                          int32_t* __restrict__ n_out, int32_t* __restrict__ rej_pos) {
+    const int b = blockIdx.x * 4 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (b >= B) return;
+    bool acc = true;
+    int y = -1;
+    if (lane < k) {
+        const size_t r = (size_t)b * k + lane;
+        y = draft[r];
+        const float log_alpha = fminf(0.f, (zp_draft[r] * inv_t - lse_p[r]) - (zq_draft[r] - lse_q[r]));
+        acc = logf(u[r]) <= log_alpha;
+    }
+    const unsigned rejected = ~__ballot_sync(0xffffffffu, acc);
+    const int a = rejected ? __ffs(rejected) - 1 : k;     // lanes >= k always vote "accepted"
+    if (lane < k) out_ids[(size_t)b * k + lane] = lane < a ? y : -1;
+    if (lane == 0) {
+        accept_len[b] = a;
+        n_out[b] = a < k ? a + 1 : k;
+        rej_pos[b] = a < k ? a : -1;
+    }
+}
+
+// ---------------------------------------------------------------- sample (c)
+struct ResidualArgs {
+    int B, k, V, slice;
+    const int32_t* rej_pos;
+    const float* target_logits;   // [B][k][V]
+    const float* draft_logits;    // [B][k][V]
+    const float* lse_p;
+    const float* lse_q;
+    double temperature;
+    const float* r;
+    double* e_p;                  // [B][V]  exp(z_p/T - lse_p)
+    double* e_q;                  // [B][V]
+    double* sums;                 // [B][NS][4]: sum e_p, sum e_q, sum residual, unused
+    int32_t* out_ids;
+    int32_t eos_id;
+    int32_t* accept_len;
+    int32_t* n_out;
+};
+
+__device__ __forceinline__ double block_sum(double v, double* sh) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();
+    if (lane == 0) sh[warp] = v;
+    __syncthreads();
+    double t = 0.0;
+    for (int w = 0; w < nw; ++w) t += sh[w];
+    return t;
+}
+
+// Pass 1: unnormalised probabilities of the rejected row in fp64, and their slice sums.
+__global__ void __launch_bounds__(RES_THREADS) residual_exp_kernel(ResidualArgs a) {
+    __shared__ double sh[32];
+    const int b = blockIdx.y, sl = blockIdx.x;
+    const int i = a.rej_pos[b];
+    if (i < 0) return;
+    const size_t row = (size_t)b * a.k + i;
+    const float* zp = a.target_logits + row * a.V;
+    const float* zq = a.draft_logits + row * a.V;
+    const double lp = (double)a.lse_p[row], lq = (double)a.lse_q[row], T = a.temperature;
+    const int v0 = sl * a.slice, v1 = min(a.V, v0 + a.slice);
+    double sp = 0.0, sq = 0.0;
+    for (int v = v0 + threadIdx.x; v < v1; v += RES_THREADS) {
+        const double ep = exp((double)zp[v] / T - lp);
+        const double eq = exp((double)zq[v] - lq);
+        a.e_p[(size_t)b * a.V + v] = ep;
+        a.e_q[(size_t)b * a.V + v] = eq;
+        sp += ep;
+        sq += eq;
+    }
+    sp = block_sum(sp, sh);
+    sq = block_sum(sq, sh);
+    if (threadIdx.x == 0) {
+        a.sums[((size_t)b * NS + sl) * 4 + 0] = sp;
+        a.sums[((size_t)b * NS + sl) * 4 + 1] = sq;
+    }
+}
+
+// Pass 2: residual mass of each slice.
+__global__ void __launch_bounds__(RES_THREADS) residual_mass_kernel(ResidualArgs a) {
+    __shared__ double sh[32];
+    const int b = blockIdx.y, sl = blockIdx.x;
+    if (a.rej_pos[b] < 0) return;
+    double Sp = 0.0, Sq = 0.0;
+    for (int j = 0; j < NS; ++j) {
+        Sp += a.sums[((size_t)b * NS + j) * 4 + 0];
+        Sq += a.sums[((size_t)b * NS + j) * 4 + 1];
+    }
+    const double ip = 1.0 / Sp, iq = 1.0 / Sq;
+    const int v0 = sl * a.slice, v1 = min(a.V, v0 + a.slice);
+    double acc = 0.0;
+    for (int v = v0 + threadIdx.x; v < v1; v += RES_THREADS) {
+        const double res = a.e_p[(size_t)b * a.V + v] * ip - a.e_q[(size_t)b * a.V + v] * iq;
+        acc += res > 0.0 ? res : 0.0;
+    }
+    acc = block_sum(acc, sh);
+    if (threadIdx.x == 0) a.sums[((size_t)b * NS + sl) * 4 + 2] = acc;
+}
+
+// Pass 3: inverse CDF in vocabulary order: the smallest v whose cumulative
+// residual reaches r * (total residual mass); from p itself if that mass is 0.
+__global__ void __launch_bounds__(LOC_THREADS) residual_locate_kernel(ResidualArgs a) {
+    __shared__ double seg[LOC_THREADS];
+    __shared__ int found_v;
+    const int b = blockIdx.x;
+    const int i = a.rej_pos[b];
+    const int tid = threadIdx.x;
+    if (i >= 0) {
+        double Sp = 0.0, Sq = 0.0, S = 0.0;
+        for (int j = 0; j < NS; ++j) {
+            Sp += a.sums[((size_t)b * NS + j) * 4 + 0];
+            Sq += a.sums[((size_t)b * NS + j) * 4 + 1];
+            S += a.sums[((size_t)b * NS + j) * 4 + 2];
+        }
+        const bool use_p = !(S > 0.0);
+        const double ip = 1.0 / Sp, iq = 1.0 / Sq;
+        const double total = use_p ? 1.0 : S;
+        const double target = (double)a.r[b] * total;
+        // slice that contains the target
+        double base = 0.0;
+        int sl = 0;
+        for (; sl < NS - 1; ++sl) {
+            const double m = use_p ? a.sums[((size_t)b * NS + sl) * 4 + 0] * ip : a.sums[((size_t)b * NS + sl) * 4 + 2];
+            if (base + m >= target) break;
+            base += m;
+        }
+        const int v0 = sl * a.slice, v1 = min(a.V, v0 + a.slice);
+        const int per = (v1 - v0 + LOC_THREADS - 1) / LOC_THREADS;
+        const int s0 = min(v1, v0 + tid * per), s1 = min(v1, s0 + per);
+        const double* ep = a.e_p + (size_t)b * a.V;
+        const double* eq = a.e_q + (size_t)b * a.V;
+        auto weight = [&](int v) -> double {
+            if (use_p) return ep[v] * ip;
+            const double res = ep[v] * ip - eq[v] * iq;
+            return res > 0.0 ? res : 0.0;
+        };
+        double mine = 0.0;
+        for (int v = s0; v < s1; ++v) mine += weight(v);
+        seg[tid] = mine;
+        if (tid == 0) found_v = -1;
+        __syncthreads();
+        if (tid == 0) {
+            // sequential walk over the 1024 segment sums, then inside the one segment
+            double cum = base;
+            int t = 0;
+            for (; t < LOC_THREADS - 1; ++t) {
+                if (cum + seg[t] >= target) break;
+                cum += seg[t];
+            }
+            const int q0 = min(v1, v0 + t * per), q1 = min(v1, q0 + per);
+            int hit = -1;
+            for (int v = q0; v < q1; ++v) {
+                cum += weight(v);
+                if (cum >= target) {
+                    hit = v;
+                    break;
+                }
+            }
+            if (hit < 0) {
+                // rounding left the running sum just short: take the last token with positive weight
+                for (int v = a.V - 1; v >= 0; --v)
+                    if (weight(v) > 0.0) {
+                        hit = v;
+                        break;
+                    }
+            }
+            found_v = hit;
+        }
+        __syncthreads();
+        if (tid == 0) a.out_ids[(size_t)b * a.k + i] = found_v;
+    }
+    // Algorithm 1's EOS break: nothing is emitted after the first EOS
+    if (a.eos_id >= 0) {
+        __syncthreads();
+        if (tid == 0) {
+            int32_t* o = a.out_ids + (size_t)b * a.k;
+            const int n = a.n_out[b];
+            for (int j = 0; j < n; ++j)
+                if (o[j] == a.eos_id) {
+                    for (int t = j + 1; t < n; ++t) o[t] = -1;
+                    a.n_out[b] = j + 1;
+                    a.accept_len[b] = min(a.accept_len[b], j + 1);
+                    break;
+                }
+        }
+    }
+}
+
+struct SampleWs {
+    float* lse_q;
+    float* zq_draft;
+    int32_t* rej_pos;
+    double* e_p;
+    double* e_q;
+    double* sums;
+    size_t bytes;
+};
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+SampleWs carve(void* base, int B, int k, int V) {
+    SampleWs w;
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        void* p = base ? static_cast<char*>(base) + off : nullptr;
+        off = align_up(off + bytes, 256);
+        return p;
+    };
+    w.lse_q = static_cast<float*>(take((size_t)B * k * sizeof(float)));
+    w.zq_draft = static_cast<float*>(take((size_t)B * k * sizeof(float)));
+    w.rej_pos = static_cast<int32_t*>(take((size_t)B * sizeof(int32_t)));
+    w.e_p = static_cast<double*>(take((size_t)B * V * sizeof(double)));
+    w.e_q = static_cast<double*>(take((size_t)B * V * sizeof(double)));
+    w.sums = static_cast<double*>(take((size_t)B * NS * 4 * sizeof(double)));
+    w.bytes = off;
+    return w;
+}
+
+}  // namespace
+
+extern "C" size_t deer_accept_workspace_bytes(int mode, int B, int k, int V) {
+    if (mode != DEER_ACC_SAMPLE || B <= 0 || k <= 0 || V <= 0) return 0;
+    return carve(nullptr, B, k, V).bytes;
+}
+
+extern "C" int deer_accept(int mode, int B, int k, int V, const int32_t* draft_ids, const int32_t* target_ids,
+                           const float* target_logits, const float* target_lse, const float* target_draft_logit,
+                           float temperature, const float* draft_logits, const float* u, const float* r, int32_t eos_id,
+                           int32_t* accept_len, int32_t* out_ids, int32_t* n_out, void* workspace, size_t workspace_bytes,
+                           void* stream) {
+    DEER_CHECK_ARG(mode == DEER_ACC_GREEDY || mode == DEER_ACC_SAMPLE, DEER_ERR_INVALID_ARG, "deer_accept: bad mode");
+    DEER_CHECK_ARG(draft_ids && accept_len && out_ids && n_out, DEER_ERR_INVALID_ARG, "deer_accept: null argument");
+    DEER_CHECK_ARG(k >= 1 && k <= DEER_MAX_BLOCK, DEER_ERR_UNSUPPORTED, "deer_accept: k must be in [1, 32]");
+    DEER_CHECK_ARG(B >= 0 && B <= 65535, DEER_ERR_UNSUPPORTED, "deer_accept: B must be in [0, 65535]");
+    if (B == 0) return DEER_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (mode == DEER_ACC_GREEDY) {
+        DEER_CHECK_ARG(target_ids, DEER_ERR_INVALID_ARG, "deer_accept: target_ids is required in GREEDY mode");
+        accept_greedy_kernel<<<(B + 127) / 128, 128, 0, st>>>(B, k, draft_ids, target_ids, eos_id, accept_len, out_ids, n_out);
+        DEER_CUDA(cudaGetLastError());
+        return DEER_OK;
+    }
+    DEER_CHECK_ARG(target_logits && target_lse && target_draft_logit && draft_logits && u && r, DEER_ERR_INVALID_ARG,
+                   "deer_accept: SAMPLE mode needs target_logits, target_lse, target_draft_logit, draft_logits, u and r");
+    DEER_CHECK_ARG(V > 0 && temperature > 0.f, DEER_ERR_INVALID_ARG, "deer_accept: V and temperature must be positive");
+    DEER_CHECK_ARG(deer_aligned16(draft_logits) && deer_aligned16(target_logits) && deer_aligned16(workspace),
+                   DEER_ERR_INVALID_ARG, "deer_accept: logits and workspace must be 16-byte aligned");
+    const size_t need = deer_accept_workspace_bytes(mode, B, k, V);
+    DEER_CHECK_ARG(workspace && workspace_bytes >= need, DEER_ERR_WORKSPACE,
+                   "deer_accept: workspace of %zu bytes needed, %zu given", need, workspace_bytes);
+    const SampleWs w = carve(workspace, B, k, V);
+
+    draft_row_stats_kernel<<<B * k, 256, 0, st>>>(V, draft_logits, draft_ids, w.lse_q, w.zq_draft);
+    DEER_CUDA(cudaGetLastError());
+    accept_scan_kernel<<<(B + 3) / 4, 128, 0, st>>>(B, k, draft_ids, target_lse, target_draft_logit, 1.f / temperature,
+                                                     w.lse_q, w.zq_draft, u, accept_len, out_ids, n_out, w.rej_pos);
+    DEER_CUDA(cudaGetLastError());
+
+    ResidualArgs a;
+    a.B = B;
+    a.k = k;
+    a.V = V;
+    a.slice = ((V + NS - 1) / NS + 3) / 4 * 4;
+    a.rej_pos = w.rej_pos;
+    a.target_logits = target_logits;
+    a.draft_logits = draft_logits;
+    a.lse_p = target_lse;
+    a.lse_q = w.lse_q;
+    a.temperature = (double)temperature;
+    a.r = r;
+    a.e_p = w.e_p;
+    a.e_q = w.e_q;
+    a.sums = w.sums;
+    a.out_ids = out_ids;
+    a.eos_id = eos_id;
+    a.accept_len = accept_len;
+    a.n_out = n_out;
+    residual_exp_kernel<<<dim3(NS, B), RES_THREADS, 0, st>>>(a);
+    DEER_CUDA(cudaGetLastError());
+    residual_mass_kernel<<<dim3(NS, B), RES_THREADS, 0, st>>>(a);
+    DEER_CUDA(cudaGetLastError());
+    residual_locate_kernel<<<B, LOC_THREADS, 0, st>>>(a);
+    DEER_CUDA(cudaGetLastError());
+    return DEER_OK;
+}

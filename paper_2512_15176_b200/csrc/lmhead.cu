@@ -1,0 +1,127 @@
+// (2) LM head + selection: z = h w^T, p_AR = softmax(z / T) of Eq. 5 reduced
+// on the fly to argmax / log-sum-exp / the draft token's logit.
+//
+// Host entry point, the cross-part finalisation, and kernel dispatch.
+
+#include "lmhead_mma.cuh"
+
+namespace lmhead {
+
+struct FinalizeArgs {
+    const Partial* part;
+    int nparts, M;
+    float inv_t_log2, inv_t;
+    int32_t* out_ids;
+    float* out_max_logprob;
+    float* out_lse;
+};
+
+__global__ void __launch_bounds__(128) lmhead_finalize_kernel(FinalizeArgs a) {
+    const int m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m >= a.M) return;
+    float rm = -INFINITY, rs = 0.f;
+    int32_t ri = 0x7fffffff;
+    for (int pt = 0; pt < a.nparts; ++pt) {
+        const Partial pr = a.part[(size_t)pt * a.M + m];
+        merge_sel(rm, ri, rs, pr.m, pr.idx, pr.s, a.inv_t_log2);
+    }
+    if (a.out_ids) a.out_ids[m] = ri;
+    const float ls = logf(rs);
+    if (a.out_max_logprob) a.out_max_logprob[m] = -ls;          // max z - logsumexp(z), T = 1
+    if (a.out_lse) a.out_lse[m] = rm * a.inv_t + ls;            // logsumexp(z / T)
+}
+
+struct Plan {
+    int bm, m_tiles, nparts;
+};
+
+static Plan plan(int M, int V) {
+    Plan pl;
+    pl.bm = (M <= 32) ? 32 : (M <= 64 ? 64 : 128);
+    pl.m_tiles = (M + pl.bm - 1) / pl.bm;
+    const int resident = 148 * (pl.bm <= 64 ? 2 : 1);
+    int np = resident / pl.m_tiles;
+    if (np < 1) np = 1;
+    const int vt = (V + VT - 1) / VT;
+    if (np > vt) np = vt;
+    pl.nparts = np;
+    return pl;
+}
+
+template <int BM>
+static int launch(const Params& p, const Plan& pl, cudaStream_t st) {
+    constexpr int SM = STAGES * (VT * KT * 2 + BM * KT * 2) + 8 * BM * (int)sizeof(Partial);
+    DEER_CUDA(cudaFuncSetAttribute(lmhead_mma_kernel<BM>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM));
+    dim3 grid(pl.m_tiles, pl.nparts);
+    lmhead_mma_kernel<BM><<<grid, THREADS, SM, st>>>(p);
+    DEER_CUDA(cudaGetLastError());
+    return DEER_OK;
+}
+
+}  // namespace lmhead
+
+extern "C" size_t deer_lmhead_workspace_bytes(int M, int hid, int V) {
+    (void)hid;
+    if (M <= 0 || V <= 0) return 0;
+    // room for the largest split any kernel variant uses
+    return (size_t)2 * 148 * M * sizeof(lmhead::Partial);
+}
+
+extern "C" int deer_lmhead_select(const void* h, const void* w, int M, int hid, int V, int mode, float temperature,
+                                  const int32_t* draft_ids, int32_t* out_ids, float* out_max_logprob, float* out_lse,
+                                  float* out_draft_logit, float* out_logits, void* workspace, size_t workspace_bytes,
+                                  void* stream) {
+    using namespace lmhead;
+    DEER_CHECK_ARG(h && w && out_ids, DEER_ERR_INVALID_ARG, "deer_lmhead_select: null argument");
+    DEER_CHECK_ARG(deer_aligned16(h) && deer_aligned16(w) && deer_aligned16(workspace) && deer_aligned16(out_logits),
+                   DEER_ERR_INVALID_ARG, "deer_lmhead_select: pointers must be 16-byte aligned");
+    DEER_CHECK_ARG(M >= 0 && V > 0 && hid > 0, DEER_ERR_INVALID_ARG, "deer_lmhead_select: bad sizes");
+    DEER_CHECK_ARG(hid % KT == 0, DEER_ERR_UNSUPPORTED, "deer_lmhead_select: hid must be a multiple of 64");
+    DEER_CHECK_ARG(mode == DEER_SEL_ARGMAX || mode == DEER_SEL_ARGMAX_LOGPROB || mode == DEER_SEL_SOFTMAX,
+                   DEER_ERR_INVALID_ARG, "deer_lmhead_select: bad mode");
+    float t = 1.f;
+    if (mode == DEER_SEL_SOFTMAX) {
+        DEER_CHECK_ARG(temperature > 0.f, DEER_ERR_INVALID_ARG, "deer_lmhead_select: temperature must be > 0");
+        DEER_CHECK_ARG(out_lse, DEER_ERR_INVALID_ARG, "deer_lmhead_select: out_lse is required in SOFTMAX mode");
+        t = temperature;
+    }
+    if (mode == DEER_SEL_ARGMAX_LOGPROB)
+        DEER_CHECK_ARG(out_max_logprob, DEER_ERR_INVALID_ARG, "deer_lmhead_select: out_max_logprob is required");
+    if (M == 0) return DEER_OK;
+    const size_t need = deer_lmhead_workspace_bytes(M, hid, V);
+    DEER_CHECK_ARG(workspace && workspace_bytes >= need, DEER_ERR_WORKSPACE,
+                   "deer_lmhead_select: workspace of %zu bytes needed, %zu given", need, workspace_bytes);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    const Plan pl = plan(M, V);
+    Params p;
+    p.h = static_cast<const __nv_bfloat16*>(h);
+    p.w = static_cast<const __nv_bfloat16*>(w);
+    p.M = M;
+    p.hid = hid;
+    p.V = V;
+    p.inv_t_log2 = LOG2E / t;
+    p.draft_ids = (mode == DEER_SEL_SOFTMAX) ? draft_ids : nullptr;
+    p.out_draft_logit = (mode == DEER_SEL_SOFTMAX) ? out_draft_logit : nullptr;
+    p.out_logits = out_logits;
+    p.part = static_cast<Partial*>(workspace);
+    p.nparts = pl.nparts;
+    int rc;
+    if (pl.bm == 32) rc = launch<32>(p, pl, st);
+    else if (pl.bm == 64) rc = launch<64>(p, pl, st);
+    else rc = launch<128>(p, pl, st);
+    if (rc != DEER_OK) return rc;
+
+    FinalizeArgs fa;
+    fa.part = p.part;
+    fa.nparts = pl.nparts;
+    fa.M = M;
+    fa.inv_t_log2 = p.inv_t_log2;
+    fa.inv_t = 1.f / t;
+    fa.out_ids = out_ids;
+    fa.out_max_logprob = (mode == DEER_SEL_ARGMAX_LOGPROB) ? out_max_logprob : nullptr;
+    fa.out_lse = (mode == DEER_SEL_SOFTMAX) ? out_lse : nullptr;
+    lmhead_finalize_kernel<<<(M + 127) / 128, 128, 0, st>>>(fa);
+    DEER_CUDA(cudaGetLastError());
+    return DEER_OK;
+}

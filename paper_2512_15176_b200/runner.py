@@ -1,0 +1,120 @@
+"""Device buffers and call sequencing for one draft-verify step.
+
+Plumbing only: torch allocates the tensors, the library's kernels do all of
+the work.  ``VerifyStep.run()`` issues reserve -> block_attn -> lmhead_select
+-> accept -> commit on the current stream without any host synchronisation.
+"""
+from __future__ import annotations
+
+import math
+from typing import Optional
+
+import torch
+
+from . import binding as L
+from .workload import MASK_BIDIR, MASK_CAUSAL, StepConfig
+
+
+def _ws(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(16, (nbytes + 15) // 16 * 16), dtype=torch.uint8, device=device)
+
+
+class VerifyStep:
+    """Buffers of one step for ``cfg``; ``kv`` is a ``binding.KVCache`` and ``w``
+    the device-resident LM-head weight [V, hid] bf16."""
+
+    def __init__(self, cfg: StepConfig, kv: L.KVCache, w: torch.Tensor, max_seq_len: int, device="cuda",
+                 store_logits: Optional[bool] = None):
+        self.cfg, self.kv, self.w, self.max_seq_len = cfg, kv, w, int(max_seq_len)
+        B, k, Hq, Hkv, D, M, V = cfg.B, cfg.k, cfg.Hq, cfg.Hkv, cfg.D, cfg.M, cfg.V
+        bf, i32, f32 = torch.bfloat16, torch.int32, torch.float32
+        dev = device
+        self.seq_ids = torch.arange(B, dtype=i32, device=dev)
+        self.q = torch.empty(B, k, Hq, D, dtype=bf, device=dev)
+        self.k_blk = torch.empty(B, k, Hkv, D, dtype=bf, device=dev)
+        self.v_blk = torch.empty(B, k, Hkv, D, dtype=bf, device=dev)
+        self.attn_out = torch.empty(B, k, Hq, D, dtype=bf, device=dev)
+        self.h = torch.empty(M, cfg.hid, dtype=bf, device=dev)
+        self.draft_ids = torch.zeros(B, k, dtype=i32, device=dev)
+        self.target_ids = torch.empty(B, k, dtype=i32, device=dev)
+        self.accept_len = torch.empty(B, dtype=i32, device=dev)
+        self.out_ids = torch.empty(B, k, dtype=i32, device=dev)
+        self.n_out = torch.empty(B, dtype=i32, device=dev)
+        self.max_logprob = torch.empty(M, dtype=f32, device=dev) if cfg.mode == "argmax_logprob" else None
+        sample = cfg.mode == "sample"
+        self.store_logits = sample if store_logits is None else store_logits
+        self.lse = torch.empty(M, dtype=f32, device=dev) if sample else None
+        self.draft_logit = torch.empty(M, dtype=f32, device=dev) if sample else None
+        self.logits = torch.empty(M, V, dtype=f32, device=dev) if self.store_logits else None
+        self.q_logits = torch.empty(B, k, V, dtype=f32, device=dev) if sample else None
+        self.u = torch.empty(B, k, dtype=f32, device=dev) if sample else None
+        self.r = torch.empty(B, dtype=f32, device=dev) if sample else None
+        self.attn_ws = _ws(L.deer_block_attn_workspace_bytes(B, k, Hq, Hkv, D, self.max_seq_len), dev)
+        self.lm_ws = _ws(L.deer_lmhead_workspace_bytes(M, cfg.hid, V), dev)
+        self.acc_ws = _ws(L.deer_accept_workspace_bytes(L.DEER_ACC_SAMPLE if sample else L.DEER_ACC_GREEDY, B, k, V), dev)
+        self.scale = 1.0 / math.sqrt(D)
+
+    # ---- inputs -------------------------------------------------------------
+    def load(self, q=None, k_blk=None, v_blk=None, h=None, draft_ids=None, q_logits=None, u=None, r=None):
+        for dst, src in ((self.q, q), (self.k_blk, k_blk), (self.v_blk, v_blk), (self.h, h), (self.draft_ids, draft_ids),
+                         (self.q_logits, q_logits), (self.u, u), (self.r, r)):
+            if src is not None:
+                if not torch.is_tensor(src):
+                    src = torch.as_tensor(src)
+                dst.copy_(src.to(dst.dtype).reshape(dst.shape), non_blocking=True)
+
+    # ---- the four calls -------------------------------------------------------
+    def reserve(self):
+        L.deer_kv_reserve(self.kv, self.seq_ids, self.cfg.k)
+
+    def attn(self, append: Optional[bool] = None):
+        causal = self.cfg.mask == MASK_CAUSAL
+        if append is None:
+            append = causal
+        L.deer_block_attn(self.kv, self.seq_ids, self.q, self.k_blk, self.v_blk, self.attn_out,
+                          L.DEER_MASK_CAUSAL if causal else L.DEER_MASK_BIDIR, append, self.scale, self.max_seq_len,
+                          self.attn_ws)
+
+    def lmhead(self):
+        c = self.cfg
+        if c.mode == "greedy":
+            L.deer_lmhead_select(self.h, self.w, L.DEER_SEL_ARGMAX, 1.0, None, self.target_ids, None, None, None,
+                                 self.logits, self.lm_ws)
+        elif c.mode == "argmax_logprob":
+            L.deer_lmhead_select(self.h, self.w, L.DEER_SEL_ARGMAX_LOGPROB, 1.0, None, self.target_ids, self.max_logprob,
+                                 None, None, self.logits, self.lm_ws)
+        else:
+            L.deer_lmhead_select(self.h, self.w, L.DEER_SEL_SOFTMAX, c.temperature, self.draft_ids, self.target_ids, None,
+                                 self.lse, self.draft_logit, self.logits, self.lm_ws)
+
+    def accept(self):
+        c = self.cfg
+        if c.mode == "sample":
+            L.deer_accept(L.DEER_ACC_SAMPLE, c.B, c.k, c.V, self.draft_ids, None, self.logits, self.lse, self.draft_logit,
+                          c.temperature, self.q_logits, self.u, self.r, -1, self.accept_len, self.out_ids, self.n_out,
+                          self.acc_ws)
+        else:
+            L.deer_accept(L.DEER_ACC_GREEDY, c.B, c.k, c.V, self.draft_ids, self.target_ids, None, None, None, 1.0, None,
+                          None, None, -1, self.accept_len, self.out_ids, self.n_out, None)
+
+    def commit(self):
+        L.deer_kv_commit(self.kv, self.seq_ids, self.accept_len, self.cfg.k)
+
+    def run(self):
+        """One whole step.  The drafter block fill (bidirectional mask) has no
+        acceptance and commits nothing."""
+        if self.cfg.mask == MASK_BIDIR:
+            self.attn(append=False)
+            self.lmhead()
+            return
+        self.reserve()
+        self.attn(append=True)
+        self.lmhead()
+        self.accept()
+        self.commit()
+
+    #: kernels launched by one run(), by mode (attn + merge, lmhead + finalize, accept, reserve/commit)
+    def launches_per_step(self) -> int:
+        if self.cfg.mask == MASK_BIDIR:
+            return 4
+        return 2 + 2 + 2 + (5 if self.cfg.mode == "sample" else 1)

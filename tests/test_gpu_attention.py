@@ -1,0 +1,83 @@
+"""GPU parity of deer_block_attn against the oracle, element by element."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2512_15176_b200 import workload as W
+from tests import harness as Hn
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(cfg, lengths=None, stress=False, append=False, max_seq_len=None):
+    from paper_2512_15176_b200 import binding as L
+    st = Hn.draw_state(cfg, lengths, stress)
+    q, kb, vb = Hn.draw_block(cfg, 0, stress)
+    okv = Hn.oracle_kv(st)
+    want = Hn.oracle_attention(cfg, okv, q, kb, vb)
+    kv = Hn.gpu_kv(st)
+    seq_ids = torch.arange(cfg.B, dtype=torch.int32, device="cuda")
+    msl = int(st.lengths.max()) if max_seq_len is None else max_seq_len
+    ws = torch.empty(max(16, L.deer_block_attn_workspace_bytes(cfg.B, cfg.k, cfg.Hq, cfg.Hkv, cfg.D, msl)), dtype=torch.uint8, device="cuda")
+    out = torch.full((cfg.B, cfg.k, cfg.Hq, cfg.D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    if append:
+        L.deer_kv_reserve(kv, seq_ids, cfg.k)
+        assert okv.reserve(np.arange(cfg.B), cfg.k)
+        okv.append(np.arange(cfg.B), Hn.f64(kb).astype(np.float32), Hn.f64(vb).astype(np.float32))
+    L.deer_block_attn(kv, seq_ids, q.cuda(), kb.cuda(), vb.cuda(), out, cfg.mask, append, 1.0 / math.sqrt(cfg.D), msl, ws)
+    torch.cuda.synchronize()
+    assert L.deer_kv_status(kv) == 0
+    Hn.check_attention(out.cpu(), want, cfg.name)
+    if append:
+        # rows written at n .. n+k-1: make them visible by committing all k on both sides
+        keep = torch.full((cfg.B,), cfg.k, dtype=torch.int32, device="cuda")
+        L.deer_kv_commit(kv, seq_ids, keep, cfg.k)
+        okv.commit(np.arange(cfg.B), [cfg.k] * cfg.B)
+        torch.cuda.synchronize()
+        Hn.kv_state_equal(kv, okv, cfg.name)
+        Hn.kv_contents_equal(kv, okv, label=cfg.name)
+    return out
+
+
+@pytest.mark.parametrize("stress", [False, True])
+def test_tiny_config(stress):
+    _run(W.config(0), stress=stress, append=True)
+
+
+@pytest.mark.parametrize("mask", [W.MASK_CAUSAL, W.MASK_BIDIR])
+@pytest.mark.parametrize("B,k,Hq,Hkv,D,lens", [
+    (3, 8, 8, 2, 64, [0, 1, 255]),            # empty prefix, single token, ragged tail
+    (2, 1, 4, 4, 128, [16, 700]),             # k = 1, G = 1
+    (2, 32, 32, 8, 128, [1500, 777]),         # several chunks, 128 rows per KV head
+    (2, 32, 32, 4, 128, [300, 1031]),         # 256 rows per KV head -> two row tiles
+    (1, 5, 6, 2, 64, [97]),                   # odd k, G = 3
+    (4, 16, 16, 8, 128, [64, 65, 63, 4096]),  # page/tile boundaries
+])
+def test_shapes_and_edges(mask, B, k, Hq, Hkv, D, lens):
+    cfg = W.StepConfig("edge", B, Hq, Hkv, D, k, 64, 64, (min(lens), max(lens)), mask=mask, seed=77)
+    _run(cfg, lengths=lens, stress=True, append=(mask == W.MASK_CAUSAL))
+
+
+def test_split_is_invisible():
+    """The same inputs with different context splits (steered by max_seq_len)
+    give the same result within rounding."""
+    cfg = W.StepConfig("split", 1, 8, 2, 128, 8, 64, 64, (3000, 3000), seed=78)
+    a = _run(cfg, stress=True, max_seq_len=3000)
+    b = _run(cfg, stress=True, max_seq_len=60000)
+    assert (a.float() - b.float()).abs().max() < 1e-2
+
+
+def test_sequence_longer_than_bound_is_reported():
+    from paper_2512_15176_b200 import binding as L
+    cfg = W.StepConfig("bound", 1, 4, 2, 64, 4, 64, 64, (100, 100), seed=79)
+    st = Hn.draw_state(cfg)
+    q, kb, vb = Hn.draw_block(cfg)
+    kv = Hn.gpu_kv(st)
+    seq_ids = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = torch.empty(L.deer_block_attn_workspace_bytes(1, 4, 4, 2, 64, 50), dtype=torch.uint8, device="cuda")
+    out = torch.zeros(1, 4, 4, 64, dtype=torch.bfloat16, device="cuda")
+    L.deer_block_attn(kv, seq_ids, q.cuda(), kb.cuda(), vb.cuda(), out, 0, 0, 0.125, 50, ws)
+    assert L.deer_kv_status(kv) == L.DEER_ERR_INVALID_ARG
+    assert L.deer_kv_status(kv) == 0          # reading clears it
