@@ -17,6 +17,7 @@ pytestmark = pytest.mark.gpu
 def _greedy_step(cfg, stress=False, steps=1, lengths=None):
     from paper_2512_15176_b200 import binding as L
     from paper_2512_15176_b200.runner import VerifyStep
+    cfg = cfg.with_(growth=max(cfg.growth, steps * cfg.k))
     st = Hn.draw_state(cfg, lengths, stress)
     okv = Hn.oracle_kv(st)
     kv = Hn.gpu_kv(st)
@@ -103,7 +104,6 @@ def test_c4_qwen3_30b_a3b_sampling_step():
     w64 = Hn.f64(w)
     q, kb, vb = Hn.draw_block(cfg)
     h, z, _ = Hn.draw_hidden_with_margin(cfg, w64)
-    # drafter logits centred on the target's so that accept lengths spread out
     zt = z.reshape(cfg.B, cfg.k, cfg.V)
     T = float(np.float32(cfg.temperature))
     ql, drafts, u, r, _ = Hn.sampling_inputs(cfg, zt.astype(np.float32), r_margin=1e-12)
