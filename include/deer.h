@@ -164,6 +164,38 @@ int deer_lmhead_select(const void* h, const void* w, int M, int hid, int V,
                        void* workspace, size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------
+ * LM head + selection WITHOUT any caller-provided scratch.  (The paper has no
+ * counterpart to this call; it exists for the library's users.)
+ *
+ * For callers that cannot allocate device memory where they call the library --
+ * a serving loop whose memory pool is sealed after start-up, a plug-in that
+ * receives only its input and output buffers, code that must stay out of the
+ * CUDA allocator -- the split-vocabulary partial results live in a fixed
+ * array inside the library image instead of a workspace.  Same arguments,
+ * outputs and results as deer_lmhead_select, minus the workspace.
+ *   - M must not exceed DEER_STATIC_MAX_ROWS (deer_lmhead_static_max_rows());
+ *     larger M returns DEER_ERR_UNSUPPORTED and launches nothing.
+ *   - The array (2*148*DEER_STATIC_MAX_ROWS*16 bytes, about 1.2 MB) is held by
+ *     every GPU that loads the library until the process exits.
+ *   - The call allocates and frees nothing, on the device or through any
+ *     library routine.  The first call on each device looks up the array's
+ *     device address (with that device current); make that first call outside
+ *     any stream capture.
+ *   - All calls on one GPU share the array, which keeps the previous call's
+ *     contents; each call overwrites every slot it later reads, so no clearing
+ *     is needed, but two calls that overlap on the GPU (different streams) race
+ *     on it -- serialise them.
+ * ---------------------------------------------------------------------- */
+#define DEER_STATIC_MAX_ROWS 256
+
+size_t deer_lmhead_static_max_rows(void);
+
+int deer_lmhead_select_static(const void* h, const void* w, int M, int hid, int V,
+                              int mode, float temperature, const int32_t* draft_ids,
+                              int32_t* out_ids, float* out_max_logprob, float* out_lse,
+                              float* out_draft_logit, float* out_logits, void* stream);
+
+/* ------------------------------------------------------------------------
  * (3) Acceptance rule (Eq. 5, Eq. 6, Algorithm 1 inner loop; the first
  * rejection ends the block because later rows were conditioned on the
  * rejected draft).

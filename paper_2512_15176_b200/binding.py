@@ -25,6 +25,7 @@ EXPORTS = [
     "deer_last_error", "deer_kv_create", "deer_kv_destroy", "deer_kv_reserve", "deer_kv_commit", "deer_kv_status",
     "deer_block_attn_workspace_bytes", "deer_block_attn", "deer_lmhead_workspace_bytes", "deer_lmhead_select",
     "deer_accept_workspace_bytes", "deer_accept", "deer_verify_step_host",
+    "deer_lmhead_static_max_rows", "deer_lmhead_select_static",
 ]
 
 
@@ -75,6 +76,10 @@ def lib() -> ctypes.CDLL:
     L.deer_lmhead_workspace_bytes.argtypes = [c_int] * 3
     L.deer_lmhead_select.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_float, c_void_p, c_void_p, c_void_p,
                                      c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    L.deer_lmhead_static_max_rows.restype = c_size_t
+    L.deer_lmhead_static_max_rows.argtypes = []
+    L.deer_lmhead_select_static.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_float, c_void_p, c_void_p,
+                                            c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     L.deer_accept_workspace_bytes.restype = c_size_t
     L.deer_accept_workspace_bytes.argtypes = [c_int] * 4
     L.deer_accept.argtypes = [c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_float,
@@ -190,6 +195,22 @@ def deer_lmhead_select(h, w, mode, temperature, draft_ids, out_ids, out_max_logp
                                     _ptr(out_logits), _ptr(workspace),
                                     workspace.numel() * workspace.element_size() if workspace is not None else 0,
                                     _stream(stream)))
+
+
+def deer_lmhead_static_max_rows() -> int:
+    return lib().deer_lmhead_static_max_rows()
+
+
+def deer_lmhead_select_static(h, w, mode, temperature, draft_ids, out_ids, out_max_logprob, out_lse, out_draft_logit,
+                              out_logits, stream=None):
+    """deer_lmhead_select for callers that cannot supply (or allocate) a workspace:
+    the scratch is a fixed array inside the library, so M is limited to
+    deer_lmhead_static_max_rows() and calls on one GPU must not overlap."""
+    M, hid = h.shape
+    V = w.shape[0]
+    _check(lib().deer_lmhead_select_static(_ptr(h), _ptr(w), M, hid, V, int(mode), float(temperature), _ptr(draft_ids),
+                                           _ptr(out_ids), _ptr(out_max_logprob), _ptr(out_lse), _ptr(out_draft_logit),
+                                           _ptr(out_logits), _stream(stream)))
 
 
 def deer_accept_workspace_bytes(mode, B, k, V) -> int:
