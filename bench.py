@@ -199,10 +199,17 @@ def run_ours(args, cfg):
     drafts = W.plant_drafts(cfg, target, W.planted_prefix_lengths(cfg))
     vs.load(draft_ids=drafts)
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    flush_rd = torch.zeros(64 << 20, dtype=torch.int32, device=dev)      # 256 MiB
+
+    def flush_l2():
+        """Evict L2 between steps: a 512 MiB write, then a 256 MiB read so that the
+        write's dirty lines are back in HBM before the timed step starts."""
+        flush.zero_()
+        flush_rd.max()
 
     def one_step(events=None):
         restore()
-        flush.zero_()                                   # evict L2 between steps (512 MiB write)
+        flush_l2()
         if events is not None:
             events[0].record()
         vs.reserve()
@@ -258,7 +265,7 @@ def run_ours(args, cfg):
     e2e_s = 0.0
     for s in range(3 + args.steps):
         restore()
-        flush.zero_()
+        flush_l2()
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         L.deer_verify_step_host(kv, sd, w, hq, hkb, hvb, hh, hd, cfg.B, cfg.k, cfg.Hq, cfg.hid, cfg.V, vs.scale,
@@ -289,7 +296,7 @@ def run_ours(args, cfg):
         "config": {"workload": cfg.name, "B": cfg.B, "k": cfg.k, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D,
                    "ctx": [int(lengths.min()), int(lengths.max())], "hid": cfg.hid, "V": cfg.V, "mask": "causal",
                    "accept": "greedy, planted Geometric(0.1) prefix capped at k", "parallelism": f"replicas x{world}",
-                   "l2": "flushed by a 512 MiB write between steps; the 1.2 GB weight stream exceeds L2 by itself"},
+                   "l2": "flushed between steps by a 512 MiB write followed by a 256 MiB read; the 1.2 GB weight stream exceeds L2 by itself"},
         "roofline": {"bound": "hbm", "kernel": "deer_lmhead_select", "achieved": achieved, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
                      "bytes_per_launch": ab["lmhead"], "avg_launch_ms": lm_avg_s * 1e3,

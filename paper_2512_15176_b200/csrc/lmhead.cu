@@ -3,9 +3,15 @@
 //
 // Host entry point, the cross-part finalisation, and kernel dispatch.
 
+#include <stdlib.h>
+#include <string.h>
+
 #include "lmhead_mma.cuh"
 
 namespace lmhead {
+
+bool umma_supported(int M, int hid, int V);
+int launch_umma(const Params& p, int need_sum, int* nparts_out, cudaStream_t st);
 
 struct FinalizeArgs {
     const Partial* part;
@@ -16,16 +22,29 @@ struct FinalizeArgs {
     float* out_lse;
 };
 
-__global__ void __launch_bounds__(128) lmhead_finalize_kernel(FinalizeArgs a) {
-    const int m = blockIdx.x * blockDim.x + threadIdx.x;
+// One warp per row: the lanes stride over the vocabulary parts, then merge by shuffles.
+__global__ void __launch_bounds__(256) lmhead_finalize_kernel(FinalizeArgs a) {
+    const int m = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
     if (m >= a.M) return;
     float rm = -INFINITY, rs = 0.f;
     int32_t ri = 0x7fffffff;
-    for (int pt = 0; pt < a.nparts; ++pt) {
+    bool aborted = false;
+    for (int pt = lane; pt < a.nparts; pt += 32) {
         const Partial pr = a.part[(size_t)pt * a.M + m];
+        aborted |= (pr.idx == PARTIAL_ABORTED);
         merge_sel(rm, ri, rs, pr.m, pr.idx, pr.s, a.inv_t_log2);
     }
-    if (a.out_ids) a.out_ids[m] = ri;
+    aborted = __any_sync(0xffffffffu, aborted);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, rm, o);
+        const int32_t oi = __shfl_xor_sync(0xffffffffu, ri, o);
+        const float os = __shfl_xor_sync(0xffffffffu, rs, o);
+        merge_sel(rm, ri, rs, om, oi, os, a.inv_t_log2);
+    }
+    if (lane != 0) return;
+    if (a.out_ids) a.out_ids[m] = aborted ? PARTIAL_ABORTED : ri;
     const float ls = logf(rs);
     if (a.out_max_logprob) a.out_max_logprob[m] = -ls;          // max z - logsumexp(z), T = 1
     if (a.out_lse) a.out_lse[m] = rm * a.inv_t + ls;            // logsumexp(z / T)
@@ -106,22 +125,27 @@ extern "C" int deer_lmhead_select(const void* h, const void* w, int M, int hid, 
     p.out_logits = out_logits;
     p.part = static_cast<Partial*>(workspace);
     p.nparts = pl.nparts;
+    // DEER_LMHEAD_IMPL=mma forces the warp-level kernel (used to cross-check the tcgen05 one)
+    const char* force = getenv("DEER_LMHEAD_IMPL");
+    const bool use_umma = umma_supported(M, hid, V) && !(force && strcmp(force, "mma") == 0);
+    int nparts = pl.nparts;
     int rc;
-    if (pl.bm == 32) rc = launch<32>(p, pl, st);
+    if (use_umma) rc = launch_umma(p, mode != DEER_SEL_ARGMAX, &nparts, st);
+    else if (pl.bm == 32) rc = launch<32>(p, pl, st);
     else if (pl.bm == 64) rc = launch<64>(p, pl, st);
     else rc = launch<128>(p, pl, st);
     if (rc != DEER_OK) return rc;
 
     FinalizeArgs fa;
     fa.part = p.part;
-    fa.nparts = pl.nparts;
+    fa.nparts = nparts;
     fa.M = M;
     fa.inv_t_log2 = p.inv_t_log2;
     fa.inv_t = 1.f / t;
     fa.out_ids = out_ids;
     fa.out_max_logprob = (mode == DEER_SEL_ARGMAX_LOGPROB) ? out_max_logprob : nullptr;
     fa.out_lse = (mode == DEER_SEL_SOFTMAX) ? out_lse : nullptr;
-    lmhead_finalize_kernel<<<(M + 127) / 128, 128, 0, st>>>(fa);
+    lmhead_finalize_kernel<<<(M + 7) / 8, 256, 0, st>>>(fa);
     DEER_CUDA(cudaGetLastError());
     return DEER_OK;
 }

@@ -22,6 +22,8 @@ struct Partial {                 // per (vocabulary part, row): running selectio
     int32_t pad;
 };
 
+constexpr int32_t PARTIAL_ABORTED = -2;   // idx written by a block that gave up on a wait
+
 struct Params {
     const __nv_bfloat16* h;      // [M][hid]
     const __nv_bfloat16* w;      // [V][hid]

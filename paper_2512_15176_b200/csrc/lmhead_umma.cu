@@ -1,0 +1,416 @@
+// LM-head contraction with fused selection on the 5th-generation tensor cores:
+// z = h w^T (Eq. 5's verifier logits) with TMA-staged operands, tcgen05.mma
+// accumulating in tensor memory, and an epilogue that reduces every
+// accumulator row to (max, argmax, sum exp) without the logits touching HBM
+// unless they are asked for.
+//
+// Tile shape: the block rows of h sit on the 128 TMEM lanes (rows beyond M are
+// zero), the vocabulary on up to 256 accumulator columns.  Each thread block
+// owns a contiguous vocabulary range cut into T equal tiles of N = 16*g rows
+// (g <= 16), so that the ranges of all blocks differ by at most one 16*T-row
+// unit and no weight row is fetched twice.  Two accumulators (2 x 256 columns)
+// let the epilogue of tile t overlap the MMAs of tile t+1.
+//
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (+ TMEM owner),
+// warps 2..5 = epilogue (one TMEM lane quarter each).  All waits are bounded:
+// a wait that runs out raises the block's abort flag and a device status word,
+// every role leaves its loop, TMEM is freed, and the kernel returns.
+
+#include <cuda.h>
+
+#include "lmhead_mma.cuh"
+
+namespace lmhead {
+namespace umma {
+
+constexpr int BM = 128;
+constexpr int BK = 64;                      // 64 bf16 = 128 bytes = one swizzle row
+constexpr int MAXN = 256;
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;        // 16 KB
+constexpr int B_BYTES = MAXN * BK * 2;      // 32 KB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int THREADS = 192;
+constexpr int W_BOX_ROWS = 16;              // one TMA box of the weight = 16 vocabulary rows x 64 k
+constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;   // ~1 s of SM clocks before a wait gives up
+
+struct Args {
+    int M, hid, V;
+    int h_box_rows;          // rows of h one TMA box brings (<= 128, multiple of 8)
+    int T;                   // tiles per block
+    int n_units;             // vocabulary units of 16*T rows
+    int nparts;
+    int need_sum;            // 0: argmax only
+    float c2;                // log2(e) / T
+    const int32_t* draft_ids;
+    float* out_draft_logit;
+    float* out_logits;
+    Partial* part;           // [nparts][M]
+};
+
+// ---- PTX wrappers -------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: false if the block is aborting or about a second has passed (then the abort flag is raised).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t i = 1;; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(tm), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// K-major operand tile [rows][64] bf16, 128-byte swizzle: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);       // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                          // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                          // descriptor version (Blackwell)
+    d |= (uint64_t)2 << 61;                          // SWIZZLE_128B
+    return d;
+}
+// kind::f16 instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t make_idesc(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+
+#define TMEM_LD_X16(taddr, r)                                                                                         \
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];" \
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),       \
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]) \
+                 : "r"(taddr))
+
+// One 16-column slice of an accumulator row: optional store, draft-token pick, running selection.
+__device__ __forceinline__ void consume16(const uint32_t (&r)[16], int vbase, int V, bool row_ok, const Args& a, size_t zrow,
+                                          int draft, int grow, float& run_m, int32_t& run_i, float& run_s) {
+    if (!row_ok || vbase >= V) return;
+    const int nv = min(16, V - vbase);
+    float v[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v[j] = (j < nv) ? __uint_as_float(r[j]) : -INFINITY;
+    if (a.out_logits) {
+        float* dst = a.out_logits + zrow + vbase;
+        if (nv == 16 && ((zrow + vbase) & 3) == 0) {
+#pragma unroll
+            for (int j = 0; j < 16; j += 4) *reinterpret_cast<float4*>(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if (j < nv) dst[j] = v[j];
+        }
+    }
+    if (draft >= vbase && draft < vbase + nv) {
+        float dv = 0.f;
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+            if (draft - vbase == j) dv = v[j];
+        a.out_draft_logit[grow] = dv;
+    }
+    float cm = v[0];
+    int ci = 0;
+#pragma unroll
+    for (int j = 1; j < 16; ++j)
+        if (v[j] > cm) {
+            cm = v[j];
+            ci = j;
+        }
+    if (cm > run_m) {
+        if (a.need_sum) run_s *= exp2f((run_m - cm) * a.c2);
+        run_m = cm;
+        run_i = vbase + ci;
+    }
+    if (a.need_sum) {
+        const float nm = -run_m * a.c2;
+        float s = 0.f;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) s += exp2f(fmaf(v[j], a.c2, nm));
+        run_s += s;
+    }
+}
+
+__global__ void __launch_bounds__(THREADS, 1)
+lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ CUtensorMap tm_w, const Args a) {
+    extern __shared__ unsigned char smem_raw[];
+    // operand stages need 1024-byte alignment for the 128-byte swizzle
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+    // bars[0..S) full, [S..2S) empty, [2S..2S+2) accumulator full, [2S+2..2S+4) accumulator empty
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int m0 = blockIdx.x * BM;
+    const int part = blockIdx.y;
+    const int u0 = (int)((long)part * a.n_units / a.nparts);
+    const int u1 = (int)((long)(part + 1) * a.n_units / a.nparts);
+    const int g = u1 - u0;                       // 16-row granules per tile (<= 16)
+    const int N = g * 16;
+    const int row_base = u0 * a.T * 16;
+    const int n_tiles = (g > 0) ? a.T : 0;
+    const int KB = a.hid / BK;
+
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t bar_base = smem_u32(bars);
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
+    auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + 2 + b); };
+
+    // ---- set-up ---------------------------------------------------------------
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(tfull_bar(b), 1);
+            mbar_init(tempty_bar(b), 4);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // rows of the h tile that TMA never writes must read as zero
+    if (a.h_box_rows < BM) {
+        for (int s = 0; s < STAGES; ++s) {
+            uint4* p = reinterpret_cast<uint4*>(smem + s * STAGE_BYTES + a.h_box_rows * 128);
+            const int n16 = (BM - a.h_box_rows) * 128 / 16;
+            for (int i = tid; i < n16; i += THREADS) p[i] = make_uint4(0, 0, 0, 0);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0 && n_tiles > 0) {
+            const uint32_t stage_tx = (uint32_t)(a.h_box_rows * 128 + N * 128);
+            int it = 0;
+            bool ok = true;
+            for (int t = 0; t < n_tiles && ok; ++t) {
+                const int row0 = row_base + t * N;
+                for (int kb = 0; kb < KB; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+                    mbar_expect_tx(full_bar(s), stage_tx);
+                    const uint32_t sa = smem_base + s * STAGE_BYTES;
+                    tma_load_2d(sa, &tm_h, kb * BK, m0, full_bar(s));
+                    const uint32_t sb = sa + A_BYTES;
+                    for (int j = 0; j < g; ++j) tma_load_2d(sb + j * (W_BOX_ROWS * 128), &tm_w, kb * BK, row0 + j * W_BOX_ROWS, full_bar(s));
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0 && n_tiles > 0) {
+            const uint32_t idesc = make_idesc(N);
+            int it = 0;
+            bool ok = true;
+            for (int t = 0; t < n_tiles && ok; ++t) {
+                const int buf = t & 1;
+                const uint32_t aph = (uint32_t)(t >> 1) & 1u;
+                if (!mbar_wait(tempty_bar(buf), aph ^ 1u, abort_flag)) break;
+                tcgen05_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * MAXN);
+                for (int kb = 0; kb < KB; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                    if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+                    tcgen05_fence_after();
+                    const uint32_t sa = smem_base + s * STAGE_BYTES;
+                    const uint64_t ad = smem_desc_sw128(sa), bd = smem_desc_sw128(sa + A_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)     // 16 bf16 = 32 bytes = 2 descriptor units along K
+                        umma_bf16(d_tmem, ad + 2 * k, bd + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    umma_commit(empty_bar(s));            // stage reusable once these MMAs have read it
+                }
+                if (ok) umma_commit(tfull_bar(buf));      // accumulator complete
+            }
+        }
+    } else {
+        // ---------------- epilogue: 4 warps, one TMEM lane quarter each ----------------
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        const int grow = m0 + row;
+        const bool row_ok = grow < a.M;
+        const size_t zrow = (size_t)(row_ok ? grow : 0) * a.V;
+        const int draft = (row_ok && a.draft_ids && a.out_draft_logit) ? a.draft_ids[grow] : -1;
+        float run_m = -INFINITY, run_s = 0.f;
+        int32_t run_i = 0x7fffffff;
+        for (int t = 0; t < n_tiles; ++t) {
+            const int buf = t & 1;
+            const uint32_t aph = (uint32_t)(t >> 1) & 1u;
+            const bool got = mbar_wait(tfull_bar(buf), aph, abort_flag);
+            if (!__all_sync(0xffffffffu, got)) break;          // warp-uniform, so the aligned TMEM loads stay converged
+            tcgen05_fence_after();
+            const int row0 = row_base + t * N;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * MAXN);
+            for (int c = 0; c < N; c += 32) {
+                uint32_t r0[16], r1[16];
+                TMEM_LD_X16(taddr + c, r0);
+                const bool second = (c + 16 < N);
+                if (second) TMEM_LD_X16(taddr + c + 16, r1);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                consume16(r0, row0 + c, a.V, row_ok, a, zrow, draft, grow, run_m, run_i, run_s);
+                if (second) consume16(r1, row0 + c + 16, a.V, row_ok, a, zrow, draft, grow, run_m, run_i, run_s);
+            }
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(buf));
+        }
+        if (row_ok) {
+            Partial pr;
+            pr.m = run_m;
+            pr.idx = run_i;
+            pr.s = a.need_sum ? run_s : 1.f;
+            pr.pad = 0;
+            if (*abort_flag) pr.idx = PARTIAL_ABORTED;     // the finalisation turns this into ids of -2
+            a.part[(size_t)part * a.M + grow] = pr;
+        }
+    }
+
+    // ---- tear-down ------------------------------------------------------------
+    tcgen05_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        // give copies that are still in flight time to land before the block's shared memory goes away
+        for (int i = 0; i < 64; ++i) __nanosleep(10000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        __syncwarp();
+        tcgen05_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+    }
+}
+
+// ---- host side ------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 2-D bf16 tensor [rows][cols] (cols contiguous), box = box_rows x 64 columns, 128-byte swizzle.
+static int make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    DEER_CHECK_ARG(fn, DEER_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {BK, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    DEER_CHECK_ARG(r == CUDA_SUCCESS, DEER_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    return DEER_OK;
+}
+
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+}  // namespace umma
+
+bool umma_supported(int M, int hid, int V) { return M > 0 && hid % umma::BK == 0 && hid >= umma::BK && V >= 16; }
+
+// Launches the tcgen05 kernel; the partials it writes are merged by lmhead_finalize_kernel.
+// *nparts_out receives the number of vocabulary parts written.
+int launch_umma(const Params& p, int need_sum, int* nparts_out, cudaStream_t st) {
+    using namespace umma;
+    const int m_tiles = (p.M + BM - 1) / BM;
+    int nparts = 148 / m_tiles;
+    if (nparts < 1) nparts = 1;
+    const int gran = (p.V + 15) / 16;                    // 16-row granules of the vocabulary
+    if (nparts > gran) nparts = gran;
+    int T = (gran + nparts * 16 - 1) / (nparts * 16);    // tiles per block so that a tile has <= 16 granules
+    int n_units;
+    for (;; ++T) {
+        n_units = (gran + T - 1) / T;
+        if ((n_units + nparts - 1) / nparts <= 16) break;
+    }
+    Args a;
+    a.M = p.M;
+    a.hid = p.hid;
+    a.V = p.V;
+    a.h_box_rows = (p.M >= BM) ? BM : ((p.M + 7) / 8) * 8;
+    a.T = T;
+    a.n_units = n_units;
+    a.nparts = nparts;
+    a.need_sum = need_sum;
+    a.c2 = p.inv_t_log2;
+    a.draft_ids = p.draft_ids;
+    a.out_draft_logit = p.out_draft_logit;
+    a.out_logits = p.out_logits;
+    a.part = p.part;
+    CUtensorMap tm_h, tm_w;
+    int rc = make_map(&tm_h, p.h, (uint64_t)p.M, (uint64_t)p.hid, (uint32_t)a.h_box_rows);
+    if (rc != DEER_OK) return rc;
+    rc = make_map(&tm_w, p.w, (uint64_t)p.V, (uint64_t)p.hid, W_BOX_ROWS);
+    if (rc != DEER_OK) return rc;
+    DEER_CUDA(cudaFuncSetAttribute(lmhead_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+    dim3 grid(m_tiles, nparts);
+    lmhead_umma_kernel<<<grid, umma::THREADS, SMEM_BYTES, st>>>(tm_h, tm_w, a);
+    DEER_CUDA(cudaGetLastError());
+    *nparts_out = nparts;
+    return DEER_OK;
+}
+
+}  // namespace lmhead

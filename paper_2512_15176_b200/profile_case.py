@@ -1,0 +1,107 @@
+"""Run one library call a few times on a chosen shape -- the small, self-ending
+program that profiler captures are taken from.
+
+    python -m paper_2512_15176_b200.profile_case lmhead --M 32 --hid 4096 --V 32768 --iters 3
+    python -m paper_2512_15176_b200.profile_case attn --B 8 --Hq 32 --Hkv 8 --k 32 --ctx 8192 --iters 3
+    python -m paper_2512_15176_b200.profile_case qstats --B 4 --k 32 --V 151936 --iters 3
+
+Prints the average CUDA-event time per call and the achieved GB/s over the
+call's algorithmic bytes.
+"""
+from __future__ import annotations
+
+import argparse
+import math
+
+import numpy as np
+import torch
+
+from . import binding as L
+from . import workload as W
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("what", choices=["lmhead", "attn", "qstats"])
+    ap.add_argument("--M", type=int, default=32)
+    ap.add_argument("--hid", type=int, default=4096)
+    ap.add_argument("--V", type=int, default=32768)
+    ap.add_argument("--B", type=int, default=8)
+    ap.add_argument("--Hq", type=int, default=32)
+    ap.add_argument("--Hkv", type=int, default=8)
+    ap.add_argument("--D", type=int, default=128)
+    ap.add_argument("--k", type=int, default=32)
+    ap.add_argument("--ctx", type=int, default=8192)
+    ap.add_argument("--mode", default="argmax", choices=["argmax", "logprob", "softmax"])
+    ap.add_argument("--logits", action="store_true")
+    ap.add_argument("--bidir", action="store_true")
+    ap.add_argument("--iters", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=1)
+    a = ap.parse_args()
+    dev = "cuda"
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    flush_rd = torch.zeros(64 << 20, dtype=torch.int32, device=dev)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(a.iters)]
+
+    if a.what == "lmhead":
+        cfg = W.StepConfig("prof", 1, 1, 1, 64, 1, a.hid, a.V, (0, 0), seed=31).with_(B=a.M)
+        w = W.normal(31, "w", (a.V, a.hid), 0.02, device=dev)
+        h = W.hidden(cfg).to(dev)
+        ids = torch.empty(a.M, dtype=torch.int32, device=dev)
+        f = lambda: torch.empty(a.M, dtype=torch.float32, device=dev)
+        mlp, lse, dl = f(), f(), f()
+        Z = torch.empty(a.M, a.V, dtype=torch.float32, device=dev) if a.logits else None
+        drafts = torch.zeros(a.M, dtype=torch.int32, device=dev)
+        ws = torch.empty(L.deer_lmhead_workspace_bytes(a.M, a.hid, a.V), dtype=torch.uint8, device=dev)
+        mode = {"argmax": L.DEER_SEL_ARGMAX, "logprob": L.DEER_SEL_ARGMAX_LOGPROB, "softmax": L.DEER_SEL_SOFTMAX}[a.mode]
+        call = lambda: L.deer_lmhead_select(h, w, mode, 1.0, drafts, ids, mlp, lse, dl, Z, ws)
+        nbytes = a.V * a.hid * 2 + a.M * a.hid * 2 + a.M * 8 + (a.M * a.V * 4 if a.logits else 0)
+        flops = 2.0 * a.M * a.hid * a.V
+    elif a.what == "attn":
+        cfg = W.StepConfig("prof", a.B, a.Hq, a.Hkv, a.D, a.k, 64, 64, (a.ctx, a.ctx),
+                           mask=W.MASK_BIDIR if a.bidir else W.MASK_CAUSAL, seed=32)
+        lengths = W.seq_lengths(cfg)
+        lay = W.kv_layout(cfg, lengths)
+        kp, vp = W.kv_pools(cfg, lay.num_pages, device=dev, sigma=1.0)
+        kv = L.KVCache.from_layout(lay, kp, vp, dev)
+        q, kb, vb = (t.to(dev) for t in W.block_qkv(cfg, sigma=1.0))
+        out = torch.empty_like(q)
+        seq_ids = torch.arange(a.B, dtype=torch.int32, device=dev)
+        ws = torch.empty(L.deer_block_attn_workspace_bytes(a.B, a.k, a.Hq, a.Hkv, a.D, a.ctx), dtype=torch.uint8, device=dev)
+        call = lambda: L.deer_block_attn(kv, seq_ids, q, kb, vb, out, cfg.mask, 0, 1.0 / math.sqrt(a.D), a.ctx, ws)
+        nbytes = W.algorithmic_bytes(cfg, lengths)["attn"]
+        flops = float(W.algorithmic_flops(cfg, lengths)["attn"])
+    else:
+        M = a.B * a.k
+        ql = W.normal(33, "ql", (a.B, a.k, a.V), 1.0, dtype=torch.float32, device=dev)
+        zt = W.normal(33, "zt", (a.B, a.k, a.V), 1.0, dtype=torch.float32, device=dev)
+        drafts = torch.zeros(a.B, a.k, dtype=torch.int32, device=dev)
+        lse = torch.logsumexp(zt, dim=2).contiguous()
+        zd = zt[:, :, 0].contiguous()
+        u = torch.full((a.B, a.k), 0.5, device=dev)
+        r = torch.full((a.B,), 0.5, device=dev)
+        al = torch.empty(a.B, dtype=torch.int32, device=dev)
+        oi = torch.empty(a.B, a.k, dtype=torch.int32, device=dev)
+        no = torch.empty(a.B, dtype=torch.int32, device=dev)
+        ws = torch.empty(L.deer_accept_workspace_bytes(L.DEER_ACC_SAMPLE, a.B, a.k, a.V), dtype=torch.uint8, device=dev)
+        call = lambda: L.deer_accept(L.DEER_ACC_SAMPLE, a.B, a.k, a.V, drafts, None, zt, lse, zd, 1.0, ql, u, r, -1, al, oi, no, ws)
+        nbytes = M * a.V * 4
+        flops = 0.0
+
+    for _ in range(a.warmup):
+        call()
+    torch.cuda.synchronize()
+    for e0, e1 in ev:
+        flush.zero_()
+        flush_rd.max()          # read pass: leaves L2 full of clean lines
+        e0.record()
+        call()
+        e1.record()
+    torch.cuda.synchronize()
+    ms = float(np.mean([e0.elapsed_time(e1) for e0, e1 in ev]))
+    print(f"{a.what}: {ms * 1e3:.1f} us/call, {nbytes / ms / 1e6:.1f} GB/s over {nbytes} algorithmic bytes, "
+          f"{flops / ms / 1e9:.1f} TFLOP/s")
+
+
+if __name__ == "__main__":
+    main()
