@@ -4,12 +4,15 @@
 // accumulator row to (max, argmax, sum exp) without the logits touching HBM
 // unless they are asked for.
 //
-// Tile shape: the block rows of h sit on the 128 TMEM lanes (rows beyond M are
-// zero), the vocabulary on up to 256 accumulator columns.  Each thread block
-// owns a contiguous vocabulary range cut into T equal tiles of N = 16*g rows
-// (g <= 16), so that the ranges of all blocks differ by at most one 16*T-row
-// unit and no weight row is fetched twice.  Two accumulators (2 x 256 columns)
-// let the epilogue of tile t overlap the MMAs of tile t+1.
+// Tile shape: the block rows of h sit on the 128 TMEM lanes (lanes beyond the
+// rows that exist are never read back), the vocabulary on up to 256 accumulator
+// columns.  Each thread block owns a contiguous vocabulary range cut into T
+// equal tiles of N = 16*g rows (g <= 16), so that the ranges of all blocks
+// differ by at most one 16*T-row unit and no weight row is fetched twice; one
+// TMA box brings a whole N x 64 weight tile.  The operand ring is as deep as
+// shared memory allows (7 stages of 30 KB at 32 block rows), because the bytes
+// in flight per SM are what cover the HBM latency.  Two accumulators
+// (2 x 256 columns) let the epilogue of tile t overlap the MMAs of tile t+1.
 //
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (+ TMEM owner),
 // warps 2..5 = epilogue (one TMEM lane quarter each).  All waits are bounded:
@@ -26,17 +29,19 @@ namespace umma {
 constexpr int BM = 128;
 constexpr int BK = 64;                      // 64 bf16 = 128 bytes = one swizzle row
 constexpr int MAXN = 256;
-constexpr int STAGES = 4;
-constexpr int A_BYTES = BM * BK * 2;        // 16 KB
-constexpr int B_BYTES = MAXN * BK * 2;      // 32 KB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int MAX_STAGES = 8;
+constexpr int A_SPAN = BM * BK * 2;         // bytes one MMA reads for its 128-row operand (16 KB)
+constexpr int SMEM_BUDGET = 220 * 1024;     // operand ring; barriers and alignment slack come on top
 constexpr int THREADS = 192;
-constexpr int W_BOX_ROWS = 16;              // one TMA box of the weight = 16 vocabulary rows x 64 k
 constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;   // ~1 s of SM clocks before a wait gives up
 
 struct Args {
     int M, hid, V;
     int h_box_rows;          // rows of h one TMA box brings (<= 128, multiple of 8)
+    int a_bytes;             // bytes of the h tile in a stage (h_box_rows * 128, a multiple of 1024)
+    int stage_bytes;         // bytes of one stage: h tile + w tile, never less than the 16 KB an MMA reads for h
+    int stages;              // pipeline depth
+    int gmax;                // granules of the larger tile size (box of tm_w_hi); tm_w_lo has gmax - 1
     int T;                   // tiles per block
     int n_units;             // vocabulary units of 16*T rows
     int nparts;
@@ -172,13 +177,15 @@ __device__ __forceinline__ void consume16(const uint32_t (&r)[16], int vbase, in
 }
 
 __global__ void __launch_bounds__(THREADS, 1)
-lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ CUtensorMap tm_w, const Args a) {
+lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ CUtensorMap tm_w_hi,
+                   const __grid_constant__ CUtensorMap tm_w_lo, const Args a) {
     extern __shared__ unsigned char smem_raw[];
     // operand stages need 1024-byte alignment for the 128-byte swizzle
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
-    // bars[0..S) full, [S..2S) empty, [2S..2S+2) accumulator full, [2S+2..2S+4) accumulator empty
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+    const int stage_bytes = a.stage_bytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + a.stages * stage_bytes);
+    // bars[0..S) full, [S..2S) empty, [2S..2S+2) accumulator full, [2S+2..2S+4) accumulator empty   (S = MAX_STAGES)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * MAX_STAGES + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -186,7 +193,7 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
     const int part = blockIdx.y;
     const int u0 = (int)((long)part * a.n_units / a.nparts);
     const int u1 = (int)((long)(part + 1) * a.n_units / a.nparts);
-    const int g = u1 - u0;                       // 16-row granules per tile (<= 16)
+    const int g = u1 - u0;                       // 16-row granules per tile: gmax or gmax - 1
     const int N = g * 16;
     const int row_base = u0 * a.T * 16;
     const int n_tiles = (g > 0) ? a.T : 0;
@@ -195,13 +202,13 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t bar_base = smem_u32(bars);
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
-    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
-    auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
-    auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + 2 + b); };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (MAX_STAGES + s); };
+    auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * MAX_STAGES + b); };
+    auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * MAX_STAGES + 2 + b); };
 
     // ---- set-up ---------------------------------------------------------------
     if (tid == 0) {
-        for (int s = 0; s < STAGES; ++s) {
+        for (int s = 0; s < a.stages; ++s) {
             mbar_init(full_bar(s), 1);
             mbar_init(empty_bar(s), 1);
         }
@@ -212,15 +219,6 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // rows of the h tile that TMA never writes must read as zero
-    if (a.h_box_rows < BM) {
-        for (int s = 0; s < STAGES; ++s) {
-            uint4* p = reinterpret_cast<uint4*>(smem + s * STAGE_BYTES + a.h_box_rows * 128);
-            const int n16 = (BM - a.h_box_rows) * 128 / 16;
-            for (int i = tid; i < n16; i += THREADS) p[i] = make_uint4(0, 0, 0, 0);
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
@@ -230,23 +228,26 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    // Accumulator rows at or beyond h_box_rows are never read back, and row i of an MMA depends on row i
+    // of its 128-row operand only, so the h atom holds just h_box_rows rows: the rest of the 16 KB the
+    // MMA reads for that operand is whatever follows in the stage (the w atom), and lands in unused lanes.
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0 && n_tiles > 0) {
+            const CUtensorMap* tm_w = (g == a.gmax) ? &tm_w_hi : &tm_w_lo;
             const uint32_t stage_tx = (uint32_t)(a.h_box_rows * 128 + N * 128);
             int it = 0;
             bool ok = true;
             for (int t = 0; t < n_tiles && ok; ++t) {
                 const int row0 = row_base + t * N;
                 for (int kb = 0; kb < KB; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                    const int s = it % a.stages;
+                    const uint32_t ph = (uint32_t)(it / a.stages) & 1u;
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
                     mbar_expect_tx(full_bar(s), stage_tx);
-                    const uint32_t sa = smem_base + s * STAGE_BYTES;
+                    const uint32_t sa = smem_base + s * stage_bytes;
+                    tma_load_2d(sa + a.a_bytes, tm_w, kb * BK, row0, full_bar(s));     // the whole N-row tile in one box
                     tma_load_2d(sa, &tm_h, kb * BK, m0, full_bar(s));
-                    const uint32_t sb = sa + A_BYTES;
-                    for (int j = 0; j < g; ++j) tma_load_2d(sb + j * (W_BOX_ROWS * 128), &tm_w, kb * BK, row0 + j * W_BOX_ROWS, full_bar(s));
                 }
             }
         }
@@ -263,12 +264,12 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * MAXN);
                 for (int kb = 0; kb < KB; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                    const int s = it % a.stages;
+                    const uint32_t ph = (uint32_t)(it / a.stages) & 1u;
                     if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
                     tcgen05_fence_after();
-                    const uint32_t sa = smem_base + s * STAGE_BYTES;
-                    const uint64_t ad = smem_desc_sw128(sa), bd = smem_desc_sw128(sa + A_BYTES);
+                    const uint32_t sa = smem_base + s * stage_bytes;
+                    const uint64_t ad = smem_desc_sw128(sa), bd = smem_desc_sw128(sa + a.a_bytes);
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k)     // 16 bf16 = 32 bytes = 2 descriptor units along K
                         umma_bf16(d_tmem, ad + 2 * k, bd + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
@@ -365,8 +366,6 @@ static int make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t c
     return DEER_OK;
 }
 
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
-
 }  // namespace umma
 
 bool umma_supported(int M, int hid, int V) { return M > 0 && hid % umma::BK == 0 && hid >= umma::BK && V >= 16; }
@@ -391,6 +390,14 @@ int launch_umma(const Params& p, int need_sum, int* nparts_out, cudaStream_t st)
     a.hid = p.hid;
     a.V = p.V;
     a.h_box_rows = (p.M >= BM) ? BM : ((p.M + 7) / 8) * 8;
+    a.gmax = (n_units + nparts - 1) / nparts;
+    a.a_bytes = a.h_box_rows * 128;
+    // a stage is never shorter than the span an MMA reads for its 128-row operand
+    a.stage_bytes = a.a_bytes + a.gmax * 16 * 128;
+    if (a.stage_bytes < A_SPAN) a.stage_bytes = A_SPAN;
+    // as deep a ring as shared memory holds: the bytes in flight per SM are what hide the HBM latency
+    a.stages = SMEM_BUDGET / a.stage_bytes;
+    if (a.stages > MAX_STAGES) a.stages = MAX_STAGES;
     a.T = T;
     a.n_units = n_units;
     a.nparts = nparts;
@@ -400,14 +407,17 @@ int launch_umma(const Params& p, int need_sum, int* nparts_out, cudaStream_t st)
     a.out_draft_logit = p.out_draft_logit;
     a.out_logits = p.out_logits;
     a.part = p.part;
-    CUtensorMap tm_h, tm_w;
+    CUtensorMap tm_h, tm_w_hi, tm_w_lo;
     int rc = make_map(&tm_h, p.h, (uint64_t)p.M, (uint64_t)p.hid, (uint32_t)a.h_box_rows);
     if (rc != DEER_OK) return rc;
-    rc = make_map(&tm_w, p.w, (uint64_t)p.V, (uint64_t)p.hid, W_BOX_ROWS);
+    rc = make_map(&tm_w_hi, p.w, (uint64_t)p.V, (uint64_t)p.hid, (uint32_t)a.gmax * 16);
     if (rc != DEER_OK) return rc;
-    DEER_CUDA(cudaFuncSetAttribute(lmhead_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+    rc = make_map(&tm_w_lo, p.w, (uint64_t)p.V, (uint64_t)p.hid, (uint32_t)(a.gmax > 1 ? a.gmax - 1 : 1) * 16);
+    if (rc != DEER_OK) return rc;
+    const int smem_bytes = a.stages * a.stage_bytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    DEER_CUDA(cudaFuncSetAttribute(lmhead_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
     dim3 grid(m_tiles, nparts);
-    lmhead_umma_kernel<<<grid, umma::THREADS, SMEM_BYTES, st>>>(tm_h, tm_w, a);
+    lmhead_umma_kernel<<<grid, umma::THREADS, smem_bytes, st>>>(tm_h, tm_w_hi, tm_w_lo, a);
     DEER_CUDA(cudaGetLastError());
     *nparts_out = nparts;
     return DEER_OK;
