@@ -43,6 +43,7 @@ extern "C" {
 #define DEER_ERR_CUDA         4   /* a CUDA runtime call failed; see deer_last_error()        */
 #define DEER_ERR_WORKSPACE    5   /* workspace smaller than the *_workspace_bytes() figure    */
 #define DEER_ERR_BAD_PAGE     6   /* device status: a kernel met an unmapped/out-of-range page */
+#define DEER_ERR_TIMEOUT      7   /* device status: a bounded wait inside a kernel ran out      */
 
 #define DEER_MASK_CAUSAL 0   /* verifier: block row i sees block rows j <= i           */
 #define DEER_MASK_BIDIR  1   /* drafter single-step fill: every block row sees all k   */

@@ -11,29 +11,16 @@
 // straight from k_blk/v_blk as one more tile handled by the last chunk's block,
 // which also appends them to the cache when asked to.
 
-#include "common.cuh"
+#include <stdlib.h>
+#include <string.h>
 
-namespace {
+#include "attn.cuh"
+
+namespace attn {
 
 constexpr int ATT_ROWS = 128;     // query rows per thread block: 8 warps x 16
-constexpr int ATT_TILE = 64;      // tokens per pipeline stage (4 pages)
 constexpr int ATT_STAGES = 3;
 constexpr int ATT_THREADS = 256;
-constexpr float LOG2E = 1.4426950408889634f;
-
-struct AttnParams {
-    deer_kv_desc kv;
-    const int32_t* seq_ids;
-    const __nv_bfloat16* q;
-    const __nv_bfloat16* k_blk;
-    const __nv_bfloat16* v_blk;
-    float* part_o;     // [max_chunks][B*k*Hq][D]
-    float* part_lse;   // [max_chunks][B*k*Hq]   (log2 domain)
-    int B, k, Hq, G, R, row_tiles;
-    int mask, append;
-    float scale_log2;
-    int chunk, max_chunks, max_seq_len;
-};
 
 template <int D>
 __device__ __forceinline__ uint32_t tile_off(int row, int chunk16) {
@@ -333,38 +320,33 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(AttnParams p, __nv_bflo
     }
 }
 
-struct AttnPlan {
-    int chunk, max_chunks, row_tiles;
-};
-
-AttnPlan plan_attn(int B, int k, int Hq, int Hkv, int max_seq_len) {
-    AttnPlan pl;
-    const int R = (Hq / Hkv) * k;
-    pl.row_tiles = (R + ATT_ROWS - 1) / ATT_ROWS;
-    const long units = (long)B * Hkv * pl.row_tiles;
-    const long target_blocks = 2L * 148;
-    long per_unit = (target_blocks + units - 1) / units;
-    if (per_unit < 1) per_unit = 1;
-    long chunk = (max_seq_len + per_unit - 1) / per_unit;
-    chunk = ((chunk + ATT_TILE - 1) / ATT_TILE) * ATT_TILE;
-    if (chunk < 256) chunk = 256;
-    pl.chunk = (int)chunk;
-    pl.max_chunks = max_seq_len > 0 ? (int)((max_seq_len + chunk - 1) / chunk) : 1;
-    if (pl.max_chunks < 1) pl.max_chunks = 1;
-    return pl;
-}
-
 template <int D>
 constexpr int attn_smem_bytes() {
     return ATT_ROWS * D * 2 + 2 * ATT_STAGES * ATT_TILE * D * 2;
 }
 
-}  // namespace
+static int mma_row_tiles(int k, int G) { return (G * k + ATT_ROWS - 1) / ATT_ROWS; }
+
+// DEER_ATTN_IMPL=mma forces the warp-level kernel (used to cross-check the tcgen05 one).
+static bool use_umma(int D, int G, float scale) {
+    const char* force = getenv("DEER_ATTN_IMPL");
+    return umma_supported(D, G, scale) && !(force && strcmp(force, "mma") == 0);
+}
+
+}  // namespace attn
+
+using namespace attn;
 
 extern "C" size_t deer_block_attn_workspace_bytes(int B, int k, int Hq, int Hkv, int D, int max_seq_len) {
     if (B <= 0 || k <= 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || max_seq_len < 0) return 0;
-    const AttnPlan pl = plan_attn(B, k, Hq, Hkv, max_seq_len);
-    return (size_t)pl.max_chunks * B * k * Hq * (D + 1) * sizeof(float);
+    // room for whichever kernel variant the call ends up using
+    const int G = Hq / Hkv > 0 ? Hq / Hkv : 1;
+    int mc = plan_attn(B, Hkv, mma_row_tiles(k, G), max_seq_len).max_chunks;
+    if (D == 128 && G <= 128) {
+        const int mc2 = plan_attn(B, Hkv, umma_row_tiles(k, G), max_seq_len).max_chunks;
+        if (mc2 > mc) mc = mc2;
+    }
+    return (size_t)mc * B * k * Hq * (D + 1) * sizeof(float);
 }
 
 extern "C" int deer_block_attn(deer_kv* kv, const int32_t* seq_ids, const void* q, const void* k_blk, const void* v_blk,
@@ -384,7 +366,9 @@ extern "C" int deer_block_attn(deer_kv* kv, const int32_t* seq_ids, const void* 
     const size_t need = deer_block_attn_workspace_bytes(B, k, Hq, Hkv, D, max_seq_len);
     DEER_CHECK_ARG(workspace && workspace_bytes >= need, DEER_ERR_WORKSPACE,
                    "deer_block_attn: workspace of %zu bytes needed, %zu given", need, workspace_bytes);
-    const AttnPlan pl = plan_attn(B, k, Hq, Hkv, max_seq_len);
+    const int G = Hq / Hkv;
+    const bool umma = use_umma(D, G, scale);
+    const AttnPlan pl = plan_attn(B, Hkv, umma ? umma_row_tiles(k, G) : mma_row_tiles(k, G), max_seq_len);
     DEER_CHECK_ARG((long)Hkv * pl.row_tiles <= 65535, DEER_ERR_UNSUPPORTED, "deer_block_attn: too many KV heads");
 
     AttnParams p;
@@ -402,6 +386,7 @@ extern "C" int deer_block_attn(deer_kv* kv, const int32_t* seq_ids, const void* 
     p.G = Hq / Hkv;
     p.R = p.G * k;
     p.row_tiles = pl.row_tiles;
+    p.ipt = 0;
     p.mask = mask;
     p.append = append ? 1 : 0;
     p.scale_log2 = scale * LOG2E;
@@ -412,7 +397,11 @@ extern "C" int deer_block_attn(deer_kv* kv, const int32_t* seq_ids, const void* 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     dim3 grid(pl.max_chunks, Hkv * pl.row_tiles, B);
     const unsigned merge_blocks = (unsigned)((n_rows + 7) / 8);
-    if (D == 128) {
+    if (umma) {
+        const int rc = launch_umma(p, st);
+        if (rc != DEER_OK) return rc;
+        attn_merge_kernel<128><<<merge_blocks, 256, 0, st>>>(p, static_cast<__nv_bfloat16*>(out));
+    } else if (D == 128) {
         constexpr int SM = attn_smem_bytes<128>();
         DEER_CUDA(cudaFuncSetAttribute(block_attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM));
         block_attn_kernel<128><<<grid, ATT_THREADS, SM, st>>>(p);

@@ -1,0 +1,54 @@
+// Shared declarations of the block-attention kernels: launch parameters, the
+// split of a sequence's context into chunks, and the two kernel variants.
+#pragma once
+
+#include "common.cuh"
+
+namespace attn {
+
+constexpr int ATT_TILE = 64;      // tokens per pipeline stage (4 pages)
+constexpr float LOG2E = 1.4426950408889634f;
+
+struct AttnParams {
+    deer_kv_desc kv;
+    const int32_t* seq_ids;
+    const __nv_bfloat16* q;
+    const __nv_bfloat16* k_blk;
+    const __nv_bfloat16* v_blk;
+    float* part_o;     // [max_chunks][B*k*Hq][D]   normalised partial outputs of the context chunks
+    float* part_lse;   // [max_chunks][B*k*Hq]      their log2-sum-exp
+    int B, k, Hq, G, R, row_tiles;
+    int ipt;           // tcgen05 variant: block rows per row tile (each brings its G query heads)
+    int mask, append;
+    float scale_log2;
+    int chunk, max_chunks, max_seq_len;
+};
+
+struct AttnPlan {
+    int chunk, max_chunks, row_tiles;
+};
+
+// Cut a context of up to max_seq_len tokens into equal chunks so that about two waves of thread
+// blocks cover the (sequence, KV head, row tile) units.
+inline AttnPlan plan_attn(int B, int Hkv, int row_tiles, int max_seq_len) {
+    AttnPlan pl;
+    pl.row_tiles = row_tiles;
+    const long units = (long)B * Hkv * row_tiles;
+    const long target_blocks = 2L * 148;
+    long per_unit = (target_blocks + units - 1) / units;
+    if (per_unit < 1) per_unit = 1;
+    long chunk = (max_seq_len + per_unit - 1) / per_unit;
+    chunk = ((chunk + ATT_TILE - 1) / ATT_TILE) * ATT_TILE;
+    if (chunk < 256) chunk = 256;
+    pl.chunk = (int)chunk;
+    pl.max_chunks = max_seq_len > 0 ? (int)((max_seq_len + chunk - 1) / chunk) : 1;
+    if (pl.max_chunks < 1) pl.max_chunks = 1;
+    return pl;
+}
+
+// tcgen05 variant (head_dim 128): row tiles of floor(128 / G) block rows.
+bool umma_supported(int D, int G, float scale);
+int umma_row_tiles(int k, int G);
+int launch_umma(AttnParams p, cudaStream_t st);
+
+}  // namespace attn

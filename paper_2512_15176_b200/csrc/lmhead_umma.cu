@@ -19,12 +19,13 @@
 // a wait that runs out raises the block's abort flag and a device status word,
 // every role leaves its loop, TMEM is freed, and the kernel returns.
 
-#include <cuda.h>
-
 #include "lmhead_mma.cuh"
+#include "sm100.cuh"
 
 namespace lmhead {
 namespace umma {
+
+using namespace sm100;
 
 constexpr int BM = 128;
 constexpr int BK = 64;                      // 64 bf16 = 128 bytes = one swizzle row
@@ -33,7 +34,6 @@ constexpr int MAX_STAGES = 8;
 constexpr int A_SPAN = BM * BK * 2;         // bytes one MMA reads for its 128-row operand (16 KB)
 constexpr int SMEM_BUDGET = 220 * 1024;     // operand ring; barriers and alignment slack come on top
 constexpr int THREADS = 192;
-constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;   // ~1 s of SM clocks before a wait gives up
 
 struct Args {
     int M, hid, V;
@@ -52,81 +52,6 @@ struct Args {
     float* out_logits;
     Partial* part;           // [nparts][M]
 };
-
-// ---- PTX wrappers -------------------------------------------------------------
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait: false if the block is aborting or about a second has passed (then the abort flag is raised).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (uint32_t i = 1;; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 63u) == 0u) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
-        }
-    }
-    *abort_flag = 1;
-    return false;
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(tm), "r"(bar), "r"(x), "r"(y)
-        : "memory");
-}
-__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// K-major operand tile [rows][64] bf16, 128-byte swizzle: 8-row groups are 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);       // start address, 16-byte units
-    d |= (uint64_t)1 << 16;                          // leading byte offset (unused for swizzled K-major)
-    d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset between 8-row groups
-    d |= (uint64_t)1 << 46;                          // descriptor version (Blackwell)
-    d |= (uint64_t)2 << 61;                          // SWIZZLE_128B
-    return d;
-}
-// kind::f16 instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
-__device__ __forceinline__ uint32_t make_idesc(int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-}
-
-#define TMEM_LD_X16(taddr, r)                                                                                         \
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];" \
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),       \
-                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]) \
-                 : "r"(taddr))
 
 // One 16-column slice of an accumulator row: optional store, draft-token pick, running selection.
 __device__ __forceinline__ void consume16(const uint32_t (&r)[16], int vbase, int V, bool row_ok, const Args& a, size_t zrow,
@@ -217,11 +142,10 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
             mbar_init(tempty_bar(b), 4);
         }
         *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_init_fence();
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+        tmem_alloc(smem_u32(tmem_slot), 512);
     }
     tcgen05_fence_before();
     __syncthreads();
@@ -254,7 +178,7 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0 && n_tiles > 0) {
-            const uint32_t idesc = make_idesc(N);
+            const uint32_t idesc = make_idesc_bf16(N, 0);
             int it = 0;
             bool ok = true;
             for (int t = 0; t < n_tiles && ok; ++t) {
@@ -269,10 +193,10 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
                     if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
                     tcgen05_fence_after();
                     const uint32_t sa = smem_base + s * stage_bytes;
-                    const uint64_t ad = smem_desc_sw128(sa), bd = smem_desc_sw128(sa + a.a_bytes);
+                    const uint64_t ad = smem_desc_sw128_kmajor(sa), bd = smem_desc_sw128_kmajor(sa + a.a_bytes);
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k)     // 16 bf16 = 32 bytes = 2 descriptor units along K
-                        umma_bf16(d_tmem, ad + 2 * k, bd + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        umma_bf16_ss(d_tmem, ad + 2 * k, bd + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
                     umma_commit(empty_bar(s));            // stage reusable once these MMAs have read it
                 }
                 if (ok) umma_commit(tfull_bar(buf));      // accumulator complete
@@ -301,7 +225,7 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
                 TMEM_LD_X16(taddr + c, r0);
                 const bool second = (c + 16 < N);
                 if (second) TMEM_LD_X16(taddr + c + 16, r1);
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                tmem_wait_ld();
                 consume16(r0, row0 + c, a.V, row_ok, a, zrow, draft, grow, run_m, run_i, run_s);
                 if (second) consume16(r1, row0 + c + 16, a.V, row_ok, a, zrow, draft, grow, run_m, run_i, run_s);
             }
@@ -331,39 +255,17 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
     if (warp == 1) {
         __syncwarp();
         tcgen05_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+        tmem_dealloc(tmem_base, 512);
     }
 }
 
 // ---- host side ------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
-// 2-D bf16 tensor [rows][cols] (cols contiguous), box = box_rows x 64 columns, 128-byte swizzle.
+// 2-D bf16 tensor [rows][cols] (cols contiguous), box = box_rows x 64 columns.
 static int make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
-    EncodeTiledFn fn = encode_fn();
-    DEER_CHECK_ARG(fn, DEER_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
-    const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {cols * 2};
-    const cuuint32_t box[2] = {BK, box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    DEER_CHECK_ARG(r == CUDA_SUCCESS, DEER_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
-    return DEER_OK;
+    const uint64_t dims[2] = {cols, rows};
+    const uint64_t strides[1] = {cols * 2};
+    const uint32_t box[2] = {BK, box_rows};
+    return make_map_bf16(tm, base, 2, dims, strides, box);
 }
 
 }  // namespace umma
