@@ -7,16 +7,18 @@
 // layout below); S = Q K^T and O += P V are tcgen05 MMAs:
 //     S (128 x 64, fp32)  = Q [smem, K-major] x K tile [smem, K-major]
 //     O (128 x 128, fp32) += P [TMEM, bf16] x V tile [smem, MN-major]
-// S is double-buffered so that the MMAs of tile t+1 overlap the softmax of
-// tile t; P overwrites its own S buffer.  The softmax warps hold one row per
+// S and P are double-buffered so that the MMAs of tile t+1 overlap the softmax
+// of tile t.  A thread gets a tcgen05.mma accepted only every ~100 cycles
+// whatever its size, so three warps issue -- even S tiles, odd S tiles, O --
+// and their streams interleave on the tensor pipe.  The softmax warps hold one row per
 // thread (no shuffles), keep a running maximum that is only raised when a tile
 // exceeds it by 2^8 (the accumulator in TMEM is rescaled then, which is rare),
 // and emit a normalised partial output plus log2-sum-exp per chunk; the merge
 // kernel combines the chunks.
 //
-// Warp roles: warp 0 = TMA producer (all lanes share page ids by shuffle),
-// warp 1 = MMA issuer and TMEM owner, warps 2..5 = softmax (one TMEM lane
-// quarter each).  Every wait is bounded: a wait that runs out raises the
+// Warp roles: warp 0 = TMA producer, warps 1-2 = issuers of S = Q K^T (warp 1
+// owns the TMEM allocation), warp 3 = issuer of O += P V, warps 4..7 = softmax
+// (one TMEM lane quarter each).  Every wait is bounded: a wait that runs out raises the
 // block's abort flag and the cache's status word, every role leaves its loop,
 // TMEM is freed and the kernel returns.
 
@@ -35,9 +37,10 @@ constexpr int Q_BYTES = 2 * Q_HALF;            // 32 KB
 constexpr int KV_HALF = ATT_TILE * 128;        // [64 tokens][64 d] bf16 = 8 KB
 constexpr int K_BYTES = 2 * KV_HALF;           // 16 KB
 constexpr int SLOT_BYTES = 2 * K_BYTES;        // K tile then V tile
-constexpr int THREADS = 192;
-constexpr int TMEM_COLS = 256;                 // S0 [0,64)  S1 [64,128)  O [128,256)
-constexpr int O_COL = 128;
+constexpr int THREADS = 256;
+constexpr int TMEM_COLS = 512;                 // S0 [0,64)  S1 [64,128)  P0 [128,160)  P1 [160,192)  O [256,384)
+constexpr int P_COL = 128;
+constexpr int O_COL = 256;
 constexpr int N_BARS = 3 * NSLOT + 6;
 constexpr float RESCALE_STEP = 8.f;            // raise the running maximum only when a tile exceeds it by 2^8
 // Slot layout.  A K (or V) tile of 64 tokens x 128 dims is 16 KB of 1 KB swizzle atoms (8 tokens x 64 dims).
@@ -187,50 +190,60 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 if (lane < 8 && pj < 2) tma_load_3d(dst + pj * KV_HALF, is_v ? &tm_vb : &tm_kb, pj * 64, kvh, b * p.k, bar);
             }
         }
-    } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
+    } else if (warp <= 2) {
+        // ---------------- issuers of S = Q K^T: warp 1 takes the even tiles, warp 2 the odd ones ----------------
         if (lane == 0) {
             const uint32_t idesc_qk = make_idesc_bf16(ATT_TILE, 0);   // S: N = 64 tokens, both operands K-major
-            const uint32_t idesc_pv = make_idesc_bf16(HD, 1);         // O: N = 128 dims, V is MN-major
+            // Operand descriptors are built once; inside the loops only their 16-byte-unit address field moves
+            // (one issuing thread: every instruction between two MMAs is latency on the critical path).
+            const uint64_t q_desc = smem_desc_sw128_kmajor(q_addr);
+            const uint64_t k_desc_pre = smem_desc_sw128(ring_addr, 16, 2048), k_desc_blk = smem_desc_sw128(ring_addr, 16, 1024);
             bool ok = mbar_wait(q_full, 0u, abort_flag);
             // S[i & 1] = Q K_i^T: 8 k-steps of 16 dims, 4 per 64-wide half
             auto issue_qk = [&](int i) -> bool {
                 const int sl = i % NSLOT;
                 if (!mbar_wait(k_full(sl), (uint32_t)(i / NSLOT) & 1u, abort_flag)) return false;
                 tcgen05_fence_after();
-                const uint32_t kdst = ring_addr + sl * SLOT_BYTES;
                 const uint32_t d_tmem = tmem_base + (uint32_t)((i & 1) * ATT_TILE);
                 const bool blk = (i >= n_prefix_tiles);
-                const uint32_t half_off = blk ? KV_HALF : 1024, sbo = blk ? 1024 : 2048;
+                const uint64_t kd = (blk ? k_desc_blk : k_desc_pre) + (uint64_t)((sl * SLOT_BYTES) >> 4);
+                const uint64_t half16 = blk ? (KV_HALF >> 4) : (1024 >> 4);     // distance between the dim halves
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk) {
-                    const uint64_t ad = smem_desc_sw128_kmajor(q_addr + (kk >> 2) * Q_HALF + (kk & 3) * 32);
-                    const uint64_t bd = smem_desc_sw128(kdst + (kk >> 2) * half_off + (kk & 3) * 32, 16, sbo);
+                    const uint64_t ad = q_desc + (uint64_t)(((kk >> 2) * Q_HALF + (kk & 3) * 32) >> 4);
+                    const uint64_t bd = kd + ((kk >> 2) ? half16 : 0) + (uint64_t)(((kk & 3) * 32) >> 4);
                     umma_bf16_ss(d_tmem, ad, bd, idesc_qk, kk != 0 ? 1u : 0u);
                 }
                 umma_commit(s_full(i & 1));
                 return true;
             };
-            if (ok) ok = issue_qk(0);
-            for (int i = 0; i < n_tiles && ok; ++i) {
-                if (i + 1 < n_tiles) {
-                    if (!issue_qk(i + 1)) break;          // the tensor core works on S_{i+1} during the softmax of tile i
-                }
+            // S buffer i & 1 is free again once the softmax warps have read tile i-2 out of it: p_ready of that tile
+            for (int i = warp - 1; i < n_tiles && ok; i += 2) {
+                if (i >= 2 && !mbar_wait(p_ready(i & 1), (uint32_t)((i - 2) >> 1) & 1u, abort_flag)) break;
+                ok = issue_qk(i);
+            }
+        }
+    } else if (warp == 3) {
+        // ---------------- issuer of O += P V ----------------
+        if (lane == 0) {
+            const uint32_t idesc_pv = make_idesc_bf16(HD, 1);         // O: N = 128 dims, V is MN-major
+            const uint64_t v_desc_pre = smem_desc_sw128(ring_addr + K_BYTES, 1024, 2048);
+            const uint64_t v_desc_blk = smem_desc_sw128(ring_addr + K_BYTES, KV_HALF, 1024);
+            for (int i = 0; i < n_tiles; ++i) {
                 const int sl = i % NSLOT;
                 if (!mbar_wait(p_ready(i & 1), (uint32_t)(i >> 1) & 1u, abort_flag)) break;
                 if (!mbar_wait(v_full(sl), (uint32_t)(i / NSLOT) & 1u, abort_flag)) break;
                 tcgen05_fence_after();
-                const uint32_t vdst = ring_addr + sl * SLOT_BYTES + K_BYTES;
-                const uint32_t p_tmem = tmem_base + (uint32_t)((i & 1) * ATT_TILE);    // P_i lives in S_i's first 32 columns
+                const uint32_t p_tmem = tmem_base + (uint32_t)(P_COL + (i & 1) * (ATT_TILE / 2));
                 const bool blk = (i >= n_prefix_tiles);
+                // 16 tokens per MMA = two 8-token atoms; lbo = distance between the dim halves, sbo = between token atoms
+                const uint64_t vd = (blk ? v_desc_blk : v_desc_pre) + (uint64_t)((sl * SLOT_BYTES) >> 4);
+                const uint64_t step16 = blk ? (2048 >> 4) : (4096 >> 4);
 #pragma unroll
-                for (int kk = 0; kk < ATT_TILE / 16; ++kk) {
-                    // 16 tokens = two 8-token atoms; lbo = distance between the dim halves, sbo = between the token atoms
-                    const uint64_t bd = blk ? smem_desc_sw128(vdst + kk * 2048, KV_HALF, 1024)
-                                            : smem_desc_sw128(vdst + kk * 4096, 1024, 2048);
-                    umma_bf16_ts(tmem_base + O_COL, p_tmem + kk * 8, bd, idesc_pv, (i | kk) != 0 ? 1u : 0u);
-                }
-                umma_commit(slot_empty(sl));              // K/V slot reusable once these MMAs have read it
+                for (int kk = 0; kk < ATT_TILE / 16; ++kk)
+                    umma_bf16_ts(tmem_base + O_COL, p_tmem + kk * 8, vd + kk * step16, idesc_pv, (i | kk) != 0 ? 1u : 0u);
+                // S_i was complete before the softmax of tile i, hence before this point: both K and V are consumed
+                umma_commit(slot_empty(sl));
                 umma_commit(o_done);                      // phase i of o_done: O includes tile i
             }
         }
@@ -242,7 +255,7 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const int g = row % p.G;
         const bool row_valid = row < ni * p.G;
         const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
-        const int wtid = tid - 64;                        // 0..127 within the softmax warps
+        const int wtid = tid - 128;                       // 0..127 within the softmax warps
 
         // append the block's K/V rows to the cache (one thread block per (sequence, KV head))
         if (p.append && last && rt == 0) {
@@ -325,7 +338,7 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 l_run *= alpha;
                 m_run = m_new;
             }
-            // P = 2^(s * scale - m), two bf16 per TMEM column, over the first 32 columns of this S buffer
+            // P = 2^(s * scale - m), two bf16 per TMEM column, in this tile's P buffer
             uint32_t pr[ATT_TILE / 2];
             float sum4[4] = {0.f, 0.f, 0.f, 0.f};
             const float neg_m = -m_run;
@@ -342,7 +355,7 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 const bool od = mbar_wait(o_done, (uint32_t)(i - 1) & 1u, abort_flag);
                 if (!__all_sync(0xffffffffu, od)) { alive = false; break; }
             }
-            TMEM_ST_X32(t_lane + buf * ATT_TILE, pr);
+            TMEM_ST_X32(t_lane + P_COL + buf * (ATT_TILE / 2), pr);
             tmem_wait_st();
             if (tile_valid < ATT_TILE) {
                 // V rows beyond the valid tokens hold whatever was in memory; they meet P = 0, which must not
