@@ -341,12 +341,13 @@ extern "C" size_t deer_block_attn_workspace_bytes(int B, int k, int Hq, int Hkv,
     if (B <= 0 || k <= 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || max_seq_len < 0) return 0;
     // room for whichever kernel variant the call ends up using
     const int G = Hq / Hkv > 0 ? Hq / Hkv : 1;
-    int mc = plan_attn(B, Hkv, mma_row_tiles(k, G), max_seq_len).max_chunks;
+    const int mc = plan_attn(B, Hkv, mma_row_tiles(k, G), max_seq_len).max_chunks;
+    size_t bytes = (size_t)mc * B * k * Hq * (D + 1) * sizeof(float);
     if (D == 128 && G <= 128) {
-        const int mc2 = plan_attn(B, Hkv, umma_row_tiles(k, G), max_seq_len).max_chunks;
-        if (mc2 > mc) mc = mc2;
+        const size_t b2 = umma_workspace_bytes(B, k, Hq, Hkv, max_seq_len);
+        if (b2 > bytes) bytes = b2;
     }
-    return (size_t)mc * B * k * Hq * (D + 1) * sizeof(float);
+    return bytes;
 }
 
 extern "C" int deer_block_attn(deer_kv* kv, const int32_t* seq_ids, const void* q, const void* k_blk, const void* v_blk,
@@ -387,6 +388,10 @@ extern "C" int deer_block_attn(deer_kv* kv, const int32_t* seq_ids, const void* 
     p.R = p.G * k;
     p.row_tiles = pl.row_tiles;
     p.ipt = 0;
+    p.nc = 0;
+    p.unit_parts = nullptr;
+    p.total_tiles = nullptr;
+    p.out = nullptr;
     p.mask = mask;
     p.append = append ? 1 : 0;
     p.scale_log2 = scale * LOG2E;
@@ -398,9 +403,9 @@ extern "C" int deer_block_attn(deer_kv* kv, const int32_t* seq_ids, const void* 
     dim3 grid(pl.max_chunks, Hkv * pl.row_tiles, B);
     const unsigned merge_blocks = (unsigned)((n_rows + 7) / 8);
     if (umma) {
+        p.out = static_cast<__nv_bfloat16*>(out);
         const int rc = launch_umma(p, st);
         if (rc != DEER_OK) return rc;
-        attn_merge_kernel<128><<<merge_blocks, 256, 0, st>>>(p, static_cast<__nv_bfloat16*>(out));
     } else if (D == 128) {
         constexpr int SM = attn_smem_bytes<128>();
         DEER_CUDA(cudaFuncSetAttribute(block_attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM));

@@ -22,6 +22,10 @@ struct AttnParams {
     int mask, append;
     float scale_log2;
     int chunk, max_chunks, max_seq_len;
+    int nc;            // tcgen05 variant: thread blocks, each with an equal share of all KV tiles
+    long long* total_tiles;   // tcgen05 variant: tiles of all units together, written by the attention kernel
+    int2* unit_parts;  // tcgen05 variant: per unit, (first, last) block holding a piece of it; first < 0: nothing to merge
+    __nv_bfloat16* out;
 };
 
 struct AttnPlan {
@@ -46,9 +50,12 @@ inline AttnPlan plan_attn(int B, int Hkv, int row_tiles, int max_seq_len) {
     return pl;
 }
 
-// tcgen05 variant (head_dim 128): row tiles of floor(128 / G) block rows.
+// tcgen05 variant (head_dim 128): row tiles of floor(128 / G) block rows; the KV tiles of all
+// (sequence, KV head, row tile) units form one list that is cut into equal shares, one per thread block.
+// launch_umma runs the attention kernel and the merge kernel for the units that were cut.
 bool umma_supported(int D, int G, float scale);
 int umma_row_tiles(int k, int G);
+size_t umma_workspace_bytes(int B, int k, int Hq, int Hkv, int max_seq_len);
 int launch_umma(AttnParams p, cudaStream_t st);
 
 }  // namespace attn
