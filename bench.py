@@ -30,6 +30,10 @@ from paper_2512_15176_b200 import workload as W  # noqa: E402
 METRIC = "verified draft tokens/s per verify step"
 UNIT = "tokens/s"
 
+# DRAM bytes (read + write) of one lmhead_umma_kernel launch from ncu, per workload name; None = not captured for
+# the kernel as it stands.
+LMHEAD_TRAFFIC = {}
+
 
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -176,13 +180,15 @@ def run_ours(args, cfg):
     L.lib()          # fail loudly if the library has not been built
 
     peaks = load_peaks()
+    greedy = cfg.mode == "greedy"
     lengths = W.seq_lengths(cfg)
     lay = W.kv_layout(cfg, lengths)
-    kp, vp = W.kv_pools(cfg, lay.num_pages)
+    # pools of the larger workloads are drawn on the device (hundreds of MB); the values only feed the timing
+    kp, vp = W.kv_pools(cfg, lay.num_pages, device="cpu" if lay.num_pages * cfg.Hkv * cfg.D < (1 << 22) else str(dev))
     kv = L.KVCache.from_layout(lay, kp, vp, dev)
     saved = [t.clone() for t in (kv.page_table, kv.seq_len, kv.n_pages, kv.free_stack, kv.free_top)]
     w = W.lm_head(cfg).to(dev)
-    vs = VerifyStep(cfg, kv, w, int(lengths.max()), device=dev, store_logits=False)
+    vs = VerifyStep(cfg, kv, w, int(lengths.max()), device=dev, store_logits=None if cfg.mode == "sample" else False)
     q, kb, vb = W.block_qkv(cfg)
     h = W.hidden(cfg)
     vs.load(q, kb, vb, h)
@@ -193,11 +199,19 @@ def run_ours(args, cfg):
 
     # drafts planted against the head's own argmax (an untimed pre-pass; only the
     # timing inputs come from it, never an expected value of a test)
-    vs.lmhead()
-    torch.cuda.synchronize()
-    target = vs.target_ids.cpu().numpy()
-    drafts = W.plant_drafts(cfg, target, W.planted_prefix_lengths(cfg))
-    vs.load(draft_ids=drafts)
+    if cfg.mode == "sample":
+        ql = W.draft_logits(cfg)
+        drafts = W.sample_drafts(ql, cfg.seed)
+        vs.load(draft_ids=drafts, q_logits=ql, u=W.uniform_open(cfg.seed, "u", (cfg.B, cfg.k)),
+                r=W.uniform_open(cfg.seed, "r", (cfg.B,)))
+        del ql
+    else:
+        vs.lmhead()
+        torch.cuda.synchronize()
+        target = vs.target_ids.cpu().numpy()
+        drafts = W.plant_drafts(cfg, target, W.planted_prefix_lengths(cfg))
+        vs.load(draft_ids=drafts)
+    bidir = cfg.mask == W.MASK_BIDIR
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
     flush_rd = torch.zeros(64 << 20, dtype=torch.int32, device=dev)      # 256 MiB
 
@@ -212,15 +226,17 @@ def run_ours(args, cfg):
         flush_l2()
         if events is not None:
             events[0].record()
-        vs.reserve()
-        vs.attn(append=True)
+        if not bidir:
+            vs.reserve()
+        vs.attn(append=not bidir)
         if events is not None:
             events[1].record()
         vs.lmhead()
         if events is not None:
             events[2].record()
-        vs.accept()
-        vs.commit()
+        if not bidir:              # the drafter's block fill proposes; nothing is accepted or committed
+            vs.accept()
+            vs.commit()
         if events is not None:
             events[3].record()
 
@@ -249,30 +265,31 @@ def run_ours(args, cfg):
     status = L.deer_kv_status(kv)
     accepted = int(vs.accept_len.sum().item())
 
-    # ---- end to end: host buffers in, verdict out, every step -----------------
-    pin = lambda t: t.contiguous().pin_memory()
-    hq, hkb, hvb, hh = pin(q), pin(kb), pin(vb), pin(h)
-    hd = pin(torch.from_numpy(drafts))
-    ha = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
-    ho = torch.empty(cfg.B, cfg.k, dtype=torch.int32).pin_memory()
-    hn = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
-    sd = L.deer_step_dev(vs.q.data_ptr(), vs.k_blk.data_ptr(), vs.v_blk.data_ptr(), vs.attn_out.data_ptr(), vs.h.data_ptr(),
-                         vs.seq_ids.data_ptr(), vs.draft_ids.data_ptr(), vs.target_ids.data_ptr(), vs.accept_len.data_ptr(),
-                         vs.out_ids.data_ptr(), vs.n_out.data_ptr(), vs.attn_ws.data_ptr(), vs.attn_ws.numel(),
-                         vs.lm_ws.data_ptr(), vs.lm_ws.numel())
-    h2d = sum(t.numel() * t.element_size() for t in (hq, hkb, hvb, hh, hd))
-    d2h = sum(t.numel() * t.element_size() for t in (ha, ho, hn))
-    e2e_s = 0.0
-    for s in range(3 + args.steps):
-        restore()
-        flush_l2()
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        L.deer_verify_step_host(kv, sd, w, hq, hkb, hvb, hh, hd, cfg.B, cfg.k, cfg.Hq, cfg.hid, cfg.V, vs.scale,
-                                int(lengths.max()), ha, ho, hn)
-        dt = time.perf_counter() - t0
-        if s >= 3:
-            e2e_s += dt
+    # ---- end to end: host buffers in, verdict out, every step (the greedy verify step has such a call) ----
+    e2e_s, h2d, d2h = 0.0, 0, 0
+    if greedy:
+        pin = lambda t: t.contiguous().pin_memory()
+        hq, hkb, hvb, hh = pin(q), pin(kb), pin(vb), pin(h)
+        hd = pin(torch.from_numpy(drafts))
+        ha = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
+        ho = torch.empty(cfg.B, cfg.k, dtype=torch.int32).pin_memory()
+        hn = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
+        sd = L.deer_step_dev(vs.q.data_ptr(), vs.k_blk.data_ptr(), vs.v_blk.data_ptr(), vs.attn_out.data_ptr(), vs.h.data_ptr(),
+                             vs.seq_ids.data_ptr(), vs.draft_ids.data_ptr(), vs.target_ids.data_ptr(), vs.accept_len.data_ptr(),
+                             vs.out_ids.data_ptr(), vs.n_out.data_ptr(), vs.attn_ws.data_ptr(), vs.attn_ws.numel(),
+                             vs.lm_ws.data_ptr(), vs.lm_ws.numel())
+        h2d = sum(t.numel() * t.element_size() for t in (hq, hkb, hvb, hh, hd))
+        d2h = sum(t.numel() * t.element_size() for t in (ha, ho, hn))
+        for s in range(3 + args.steps):
+            restore()
+            flush_l2()
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            L.deer_verify_step_host(kv, sd, w, hq, hkb, hvb, hh, hd, cfg.B, cfg.k, cfg.Hq, cfg.hid, cfg.V, vs.scale,
+                                    int(lengths.max()), ha, ho, hn)
+            dt = time.perf_counter() - t0
+            if s >= 3:
+                e2e_s += dt
     e2e_s_t = torch.tensor([total_ms / 1e3, e2e_s], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(e2e_s_t, op=dist.ReduceOp.MAX)
@@ -286,30 +303,44 @@ def run_ours(args, cfg):
     value = tokens / total_s
     ab = W.algorithmic_bytes(cfg, lengths)
     fl = W.algorithmic_flops(cfg, lengths)
-    lm_avg_s = float(np.mean(lm_ms)) / 1e3
-    achieved = ab["lmhead"] / lm_avg_s / 1e9
-    floor_s = (ab["attn"] + ab["lmhead"] + ab["accept"]) / (peaks["hbm_gbs"] * 1e9)
+    hbm, tens = peaks["hbm_gbs"] * 1e9, peaks["bf16_tflops_sustained"] * 1e12
+    attn_s, lm_s = float(np.mean(attn_ms)) / 1e3, float(np.mean(lm_ms)) / 1e3
+    step_s = total_s / args.steps
+    # the dominant kernel is the LM head; it is HBM-bound below about hbm-ridge rows and tensor-bound above
+    lm_tensor_bound = fl["lmhead"] / tens > ab["lmhead"] / hbm
+    if lm_tensor_bound:
+        achieved, peak, unit, bound = fl["lmhead"] / lm_s / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s", "tensor"
+    else:
+        achieved, peak, unit, bound = ab["lmhead"] / lm_s / 1e9, peaks["hbm_gbs"], "GB/s", "hbm"
+    floor_s = (max(ab["attn"] / hbm, fl["attn"] / tens) + max(ab["lmhead"] / hbm, fl["lmhead"] / tens) + ab["accept"] / hbm)
+    accept_text = {"greedy": "greedy, planted Geometric(0.1) prefix capped at k",
+                   "argmax_logprob": "none (drafter block fill: argmax + max log-probability per position)",
+                   "sample": "rejection sampling at temperature %.2g with residual resampling" % cfg.temperature}[cfg.mode]
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-        "ms_per_step": total_s * 1e3 / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": cfg.name, "B": cfg.B, "k": cfg.k, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D,
-                   "ctx": [int(lengths.min()), int(lengths.max())], "hid": cfg.hid, "V": cfg.V, "mask": "causal",
-                   "accept": "greedy, planted Geometric(0.1) prefix capped at k", "parallelism": f"replicas x{world}",
-                   "l2": "flushed between steps by a 512 MiB write followed by a 256 MiB read; the 1.2 GB weight stream exceeds L2 by itself"},
-        "roofline": {"bound": "hbm", "kernel": "deer_lmhead_select", "achieved": achieved, "peak": peaks["hbm_gbs"],
-                     "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
-                     "bytes_per_launch": ab["lmhead"], "avg_launch_ms": lm_avg_s * 1e3,
-                     "step_frac_of_hbm_floor": floor_s / (total_s / args.steps),
-                     "attn_avg_ms": float(np.mean(attn_ms)), "attn_gbs": ab["attn"] / (float(np.mean(attn_ms)) / 1e3) / 1e9},
-        "e2e": {"value": cfg.M * args.steps * world / e2e_total, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": e2e_total * 1e3 / args.steps},
+                   "ctx": [int(lengths.min()), int(lengths.max())], "hid": cfg.hid, "V": cfg.V,
+                   "mask": "bidirectional" if bidir else "causal", "accept": accept_text, "parallelism": f"replicas x{world}",
+                   "l2": "flushed between steps by a 512 MiB write followed by a 256 MiB read; the weight stream exceeds L2 by itself"},
+        "roofline": {"bound": bound, "kernel": "deer_lmhead_select", "achieved": achieved, "peak": peak,
+                     "unit": unit, "frac": achieved / peak, "traffic": LMHEAD_TRAFFIC.get(cfg.name), "peak_source": peaks["source"],
+                     "bytes_per_launch": ab["lmhead"], "flops_per_launch": fl["lmhead"], "avg_launch_ms": lm_s * 1e3,
+                     "step_frac_of_roofline_floor": floor_s / step_s, "step_floor_ms": floor_s * 1e3},
+        "phases": {"attn_ms": attn_s * 1e3, "attn_gbs": ab["attn"] / attn_s / 1e9, "attn_frac_of_hbm": ab["attn"] / attn_s / hbm,
+                   "attn_tflops": fl["attn"] / attn_s / 1e12, "lmhead_ms": lm_s * 1e3, "lmhead_gbs": ab["lmhead"] / lm_s / 1e9,
+                   "lmhead_tflops": fl["lmhead"] / lm_s / 1e12, "accept_commit_ms": (step_s - attn_s - lm_s) * 1e3},
+        "e2e": ({"value": cfg.M * args.steps * world / e2e_total, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                 "ms_per_step": e2e_total * 1e3 / args.steps} if greedy else
+                {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+                 "note": "the host-buffer entry point covers the greedy verify step only"}),
         "gpu_launches": args.steps * vs.launches_per_step(),
         "clocks": clocks,
         "kv_status": status, "accepted_tokens_last_step": accepted, "wall_s_timed_loop": wall,
         "flops_per_step": fl["total"],
     }
-    if world == 1 and not args.no_cpu_baseline:
+    if world == 1 and greedy and not args.no_cpu_baseline:
         sec, toks, sample = oracle_step_seconds(cfg, 1)
         line["cpu_baseline"] = {"value": toks / sec, "unit": UNIT, "cores": len(os.sched_getaffinity(0)), "kind": "oracle",
                                 "sample": sample}
@@ -328,8 +359,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     cfg = W.config(args.config)
-    if cfg.mode != "greedy":
-        raise SystemExit("bench.py times the greedy verify step (workload 0 or 1)")
+    if args.impl == "reference" and cfg.mode != "greedy":
+        raise SystemExit("the oracle arm times the greedy verify step (workload 0 or 1)")
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

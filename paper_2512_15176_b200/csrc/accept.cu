@@ -13,9 +13,8 @@
 
 namespace {
 
-constexpr int NS = 8;              // vocabulary slices per rejected row
-constexpr int RES_THREADS = 512;
-constexpr int LOC_THREADS = 1024;
+constexpr int NS = 32;             // vocabulary slices per rejected row
+constexpr int RES_THREADS = 256;
 
 // ---------------------------------------------------------------- greedy
 __global__ void accept_greedy_kernel(int B, int k, const int32_t* __restrict__ draft, const int32_t* __restrict__ target,
@@ -107,7 +106,8 @@ __global__ void __launch_bounds__(128) accept_scan_kernel(int B, int k, const in
                                                           float inv_t, const float* __restrict__ lse_q,
                                                           const float* __restrict__ zq_draft, const float* __restrict__ u,
                                                           int32_t* __restrict__ accept_len, int32_t* __restrict__ out_ids,
-                                                          int32_t* __restrict__ n_out, int32_t* __restrict__ rej_pos) {
+                                                          int32_t* __restrict__ n_out, int32_t* __restrict__ rej_pos,
+                                                          int32_t* __restrict__ done) {
     const int b = blockIdx.x * 4 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (b >= B) return;
@@ -126,10 +126,14 @@ __global__ void __launch_bounds__(128) accept_scan_kernel(int B, int k, const in
         accept_len[b] = a;
         n_out[b] = a < k ? a + 1 : k;
         rej_pos[b] = a < k ? a : -1;
+        done[b] = 0;                    // slices of the residual pass finished so far
     }
 }
 
 // ---------------------------------------------------------------- sample (c)
+// The residual of the one rejected row of a sequence.  Probabilities are recomputed from the fp32 logits in
+// fp64 wherever they are needed instead of being stored: p(v) = exp(z_p/T - lse_p) / Sp with Sp the fp64 sum of the
+// numerators (lse_p is only fp32-accurate), likewise q.
 struct ResidualArgs {
     int B, k, V, slice;
     const int32_t* rej_pos;
@@ -139,9 +143,8 @@ struct ResidualArgs {
     const float* lse_q;
     double temperature;
     const float* r;
-    double* e_p;                  // [B][V]  exp(z_p/T - lse_p)
-    double* e_q;                  // [B][V]
-    double* sums;                 // [B][NS][4]: sum e_p, sum e_q, sum residual, unused
+    double* sums;                 // [B][NS][4]: sum e_p, sum e_q, residual mass of the slice, unused
+    int32_t* done;                // [B] slices finished (zeroed by the scan kernel)
     int32_t* out_ids;
     int32_t eos_id;
     int32_t* accept_len;
@@ -160,8 +163,21 @@ __device__ __forceinline__ double block_sum(double v, double* sh) {
     return t;
 }
 
-// Pass 1: unnormalised probabilities of the rejected row in fp64, and their slice sums.
-__global__ void __launch_bounds__(RES_THREADS) residual_exp_kernel(ResidualArgs a) {
+// Algorithm 1's EOS break: nothing is emitted after the first EOS (one thread per sequence).
+__device__ void cut_at_eos(const ResidualArgs& a, int b) {
+    int32_t* o = a.out_ids + (size_t)b * a.k;
+    const int n = a.n_out[b];
+    for (int j = 0; j < n; ++j)
+        if (o[j] == a.eos_id) {
+            for (int t = j + 1; t < n; ++t) o[t] = -1;
+            a.n_out[b] = j + 1;
+            a.accept_len[b] = min(a.accept_len[b], j + 1);
+            break;
+        }
+}
+
+// Pass 1: the fp64 normalisers, one (slice, sequence) per block.
+__global__ void __launch_bounds__(RES_THREADS) residual_norm_kernel(ResidualArgs a) {
     __shared__ double sh[32];
     const int b = blockIdx.y, sl = blockIdx.x;
     const int i = a.rej_pos[b];
@@ -169,16 +185,12 @@ __global__ void __launch_bounds__(RES_THREADS) residual_exp_kernel(ResidualArgs 
     const size_t row = (size_t)b * a.k + i;
     const float* zp = a.target_logits + row * a.V;
     const float* zq = a.draft_logits + row * a.V;
-    const double lp = (double)a.lse_p[row], lq = (double)a.lse_q[row], T = a.temperature;
+    const double lp = (double)a.lse_p[row], lq = (double)a.lse_q[row], it = 1.0 / a.temperature;
     const int v0 = sl * a.slice, v1 = min(a.V, v0 + a.slice);
     double sp = 0.0, sq = 0.0;
     for (int v = v0 + threadIdx.x; v < v1; v += RES_THREADS) {
-        const double ep = exp((double)zp[v] / T - lp);
-        const double eq = exp((double)zq[v] - lq);
-        a.e_p[(size_t)b * a.V + v] = ep;
-        a.e_q[(size_t)b * a.V + v] = eq;
-        sp += ep;
-        sq += eq;
+        sp += exp((double)zp[v] * it - lp);
+        sq += exp((double)zq[v] - lq);
     }
     sp = block_sum(sp, sh);
     sq = block_sum(sq, sh);
@@ -188,113 +200,113 @@ __global__ void __launch_bounds__(RES_THREADS) residual_exp_kernel(ResidualArgs 
     }
 }
 
-// Pass 2: residual mass of each slice.
-__global__ void __launch_bounds__(RES_THREADS) residual_mass_kernel(ResidualArgs a) {
+// Pass 2: residual mass of each slice; the block that finishes a sequence's last slice then draws the token:
+// inverse CDF in vocabulary order, the smallest v whose cumulative residual reaches r * (total residual mass),
+// from p itself if that mass is 0.
+__global__ void __launch_bounds__(RES_THREADS) residual_pick_kernel(ResidualArgs a) {
     __shared__ double sh[32];
+    __shared__ double warp_pref[RES_THREADS / 32];
+    __shared__ int s_last, s_hit;
     const int b = blockIdx.y, sl = blockIdx.x;
-    if (a.rej_pos[b] < 0) return;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int i = a.rej_pos[b];
+    if (i < 0) {
+        if (sl == 0 && tid == 0 && a.eos_id >= 0) cut_at_eos(a, b);
+        return;
+    }
+    const size_t row = (size_t)b * a.k + i;
+    const float* zp = a.target_logits + row * a.V;
+    const float* zq = a.draft_logits + row * a.V;
+    const double lp = (double)a.lse_p[row], lq = (double)a.lse_q[row], it = 1.0 / a.temperature;
     double Sp = 0.0, Sq = 0.0;
     for (int j = 0; j < NS; ++j) {
         Sp += a.sums[((size_t)b * NS + j) * 4 + 0];
         Sq += a.sums[((size_t)b * NS + j) * 4 + 1];
     }
     const double ip = 1.0 / Sp, iq = 1.0 / Sq;
-    const int v0 = sl * a.slice, v1 = min(a.V, v0 + a.slice);
-    double acc = 0.0;
-    for (int v = v0 + threadIdx.x; v < v1; v += RES_THREADS) {
-        const double res = a.e_p[(size_t)b * a.V + v] * ip - a.e_q[(size_t)b * a.V + v] * iq;
-        acc += res > 0.0 ? res : 0.0;
-    }
-    acc = block_sum(acc, sh);
-    if (threadIdx.x == 0) a.sums[((size_t)b * NS + sl) * 4 + 2] = acc;
-}
-
-// Pass 3: inverse CDF in vocabulary order: the smallest v whose cumulative
-// residual reaches r * (total residual mass); from p itself if that mass is 0.
-__global__ void __launch_bounds__(LOC_THREADS) residual_locate_kernel(ResidualArgs a) {
-    __shared__ double seg[LOC_THREADS];
-    __shared__ int found_v;
-    const int b = blockIdx.x;
-    const int i = a.rej_pos[b];
-    const int tid = threadIdx.x;
-    if (i >= 0) {
-        double Sp = 0.0, Sq = 0.0, S = 0.0;
-        for (int j = 0; j < NS; ++j) {
-            Sp += a.sums[((size_t)b * NS + j) * 4 + 0];
-            Sq += a.sums[((size_t)b * NS + j) * 4 + 1];
-            S += a.sums[((size_t)b * NS + j) * 4 + 2];
-        }
-        const bool use_p = !(S > 0.0);
-        const double ip = 1.0 / Sp, iq = 1.0 / Sq;
-        const double total = use_p ? 1.0 : S;
-        const double target = (double)a.r[b] * total;
-        // slice that contains the target
-        double base = 0.0;
-        int sl = 0;
-        for (; sl < NS - 1; ++sl) {
-            const double m = use_p ? a.sums[((size_t)b * NS + sl) * 4 + 0] * ip : a.sums[((size_t)b * NS + sl) * 4 + 2];
-            if (base + m >= target) break;
-            base += m;
-        }
+    auto prob_p = [&](int v) { return exp((double)zp[v] * it - lp) * ip; };
+    auto resid = [&](int v) {
+        const double res = prob_p(v) - exp((double)zq[v] - lq) * iq;
+        return res > 0.0 ? res : 0.0;
+    };
+    {
         const int v0 = sl * a.slice, v1 = min(a.V, v0 + a.slice);
-        const int per = (v1 - v0 + LOC_THREADS - 1) / LOC_THREADS;
-        const int s0 = min(v1, v0 + tid * per), s1 = min(v1, s0 + per);
-        const double* ep = a.e_p + (size_t)b * a.V;
-        const double* eq = a.e_q + (size_t)b * a.V;
-        auto weight = [&](int v) -> double {
-            if (use_p) return ep[v] * ip;
-            const double res = ep[v] * ip - eq[v] * iq;
-            return res > 0.0 ? res : 0.0;
-        };
-        double mine = 0.0;
-        for (int v = s0; v < s1; ++v) mine += weight(v);
-        seg[tid] = mine;
-        if (tid == 0) found_v = -1;
-        __syncthreads();
+        double acc = 0.0;
+        for (int v = v0 + tid; v < v1; v += RES_THREADS) acc += resid(v);
+        acc = block_sum(acc, sh);
         if (tid == 0) {
-            // sequential walk over the 1024 segment sums, then inside the one segment
-            double cum = base;
-            int t = 0;
-            for (; t < LOC_THREADS - 1; ++t) {
-                if (cum + seg[t] >= target) break;
-                cum += seg[t];
+            a.sums[((size_t)b * NS + sl) * 4 + 2] = acc;
+            __threadfence();
+            s_last = (atomicAdd(a.done + b, 1) == NS - 1) ? 1 : 0;
+        }
+        __syncthreads();
+        if (!s_last) return;
+        __threadfence();
+    }
+    // ---- the last block of the sequence: locate the slice, then the token inside it ----
+    const volatile double* vs = a.sums;
+    double S = 0.0;
+    for (int j = 0; j < NS; ++j) S += vs[((size_t)b * NS + j) * 4 + 2];
+    const bool use_p = !(S > 0.0);
+    const double target = (double)a.r[b] * (use_p ? 1.0 : S);
+    double base = 0.0;
+    int hs = 0;
+    for (; hs < NS - 1; ++hs) {
+        const double m = use_p ? vs[((size_t)b * NS + hs) * 4 + 0] * ip : vs[((size_t)b * NS + hs) * 4 + 2];
+        if (base + m >= target) break;
+        base += m;
+    }
+    auto weight = [&](int v) { return use_p ? prob_p(v) : resid(v); };
+    const int v0 = hs * a.slice, v1 = min(a.V, v0 + a.slice);
+    const int per = (v1 - v0 + RES_THREADS - 1) / RES_THREADS;      // contiguous tokens per thread
+    const int c0 = min(v1, v0 + tid * per), c1 = min(v1, c0 + per);
+    double mine = 0.0;
+    for (int v = c0; v < c1; ++v) mine += weight(v);
+    // exclusive prefix of the threads' sums in token order
+    double incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (tid == 0) s_hit = -1;
+    if (lane == 31) warp_pref[warp] = incl;
+    __syncthreads();
+    double wbase = base;
+    for (int w = 0; w < warp; ++w) wbase += warp_pref[w];
+    const double before = wbase + incl - mine, upto = wbase + incl;
+    if (before < target && upto >= target) {
+        // the one thread whose tokens straddle the target walks them
+        double cum = before;
+        int hit = -1;
+        for (int v = c0; v < c1; ++v) {
+            cum += weight(v);
+            if (cum >= target) {
+                hit = v;
+                break;
             }
-            const int q0 = min(v1, v0 + t * per), q1 = min(v1, q0 + per);
-            int hit = -1;
-            for (int v = q0; v < q1; ++v) {
-                cum += weight(v);
-                if (cum >= target) {
+        }
+        if (hit < 0)                                   // rounding left the walk just short: last token with weight
+            for (int v = c1 - 1; v >= c0; --v)
+                if (weight(v) > 0.0) {
                     hit = v;
                     break;
                 }
-            }
-            if (hit < 0) {
-                // rounding left the running sum just short: take the last token with positive weight
-                for (int v = a.V - 1; v >= 0; --v)
-                    if (weight(v) > 0.0) {
-                        hit = v;
-                        break;
-                    }
-            }
-            found_v = hit;
-        }
-        __syncthreads();
-        if (tid == 0) a.out_ids[(size_t)b * a.k + i] = found_v;
+        s_hit = hit;
     }
-    // Algorithm 1's EOS break: nothing is emitted after the first EOS
-    if (a.eos_id >= 0) {
-        __syncthreads();
-        if (tid == 0) {
-            int32_t* o = a.out_ids + (size_t)b * a.k;
-            const int n = a.n_out[b];
-            for (int j = 0; j < n; ++j)
-                if (o[j] == a.eos_id) {
-                    for (int t = j + 1; t < n; ++t) o[t] = -1;
-                    a.n_out[b] = j + 1;
-                    a.accept_len[b] = min(a.accept_len[b], j + 1);
+    __syncthreads();
+    if (tid == 0) {
+        int hit = s_hit;
+        if (hit < 0) {
+            // the target lies beyond the last cumulative sum by rounding: take the last token with positive weight
+            for (int v = a.V - 1; v >= 0; --v)
+                if (weight(v) > 0.0) {
+                    hit = v;
                     break;
                 }
         }
+        a.out_ids[(size_t)b * a.k + i] = hit;
+        if (a.eos_id >= 0) cut_at_eos(a, b);
     }
 }
 
@@ -302,9 +314,8 @@ struct SampleWs {
     float* lse_q;
     float* zq_draft;
     int32_t* rej_pos;
-    double* e_p;
-    double* e_q;
     double* sums;
+    int32_t* done;
     size_t bytes;
 };
 
@@ -321,9 +332,8 @@ SampleWs carve(void* base, int B, int k, int V) {
     w.lse_q = static_cast<float*>(take((size_t)B * k * sizeof(float)));
     w.zq_draft = static_cast<float*>(take((size_t)B * k * sizeof(float)));
     w.rej_pos = static_cast<int32_t*>(take((size_t)B * sizeof(int32_t)));
-    w.e_p = static_cast<double*>(take((size_t)B * V * sizeof(double)));
-    w.e_q = static_cast<double*>(take((size_t)B * V * sizeof(double)));
     w.sums = static_cast<double*>(take((size_t)B * NS * 4 * sizeof(double)));
+    w.done = static_cast<int32_t*>(take((size_t)B * sizeof(int32_t)));
     w.bytes = off;
     return w;
 }
@@ -365,7 +375,8 @@ extern "C" int deer_accept(int mode, int B, int k, int V, const int32_t* draft_i
     draft_row_stats_kernel<<<B * k, 256, 0, st>>>(V, draft_logits, draft_ids, w.lse_q, w.zq_draft);
     DEER_CUDA(cudaGetLastError());
     accept_scan_kernel<<<(B + 3) / 4, 128, 0, st>>>(B, k, draft_ids, target_lse, target_draft_logit, 1.f / temperature,
-                                                     w.lse_q, w.zq_draft, u, accept_len, out_ids, n_out, w.rej_pos);
+                                                     w.lse_q, w.zq_draft, u, accept_len, out_ids, n_out, w.rej_pos,
+                                                     w.done);
     DEER_CUDA(cudaGetLastError());
 
     ResidualArgs a;
@@ -380,18 +391,15 @@ extern "C" int deer_accept(int mode, int B, int k, int V, const int32_t* draft_i
     a.lse_q = w.lse_q;
     a.temperature = (double)temperature;
     a.r = r;
-    a.e_p = w.e_p;
-    a.e_q = w.e_q;
     a.sums = w.sums;
+    a.done = w.done;
     a.out_ids = out_ids;
     a.eos_id = eos_id;
     a.accept_len = accept_len;
     a.n_out = n_out;
-    residual_exp_kernel<<<dim3(NS, B), RES_THREADS, 0, st>>>(a);
+    residual_norm_kernel<<<dim3(NS, B), RES_THREADS, 0, st>>>(a);
     DEER_CUDA(cudaGetLastError());
-    residual_mass_kernel<<<dim3(NS, B), RES_THREADS, 0, st>>>(a);
-    DEER_CUDA(cudaGetLastError());
-    residual_locate_kernel<<<B, LOC_THREADS, 0, st>>>(a);
+    residual_pick_kernel<<<dim3(NS, B), RES_THREADS, 0, st>>>(a);
     DEER_CUDA(cudaGetLastError());
     return DEER_OK;
 }

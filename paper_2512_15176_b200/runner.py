@@ -117,4 +117,4 @@ class VerifyStep:
     def launches_per_step(self) -> int:
         if self.cfg.mask == MASK_BIDIR:
             return 4
-        return 2 + 2 + 2 + (5 if self.cfg.mode == "sample" else 1)
+        return 2 + 2 + 2 + (4 if self.cfg.mode == "sample" else 1)

@@ -54,10 +54,42 @@ def test_tiny_config(stress):
     (2, 32, 32, 4, 128, [300, 1031]),         # 256 rows per KV head -> two row tiles
     (1, 5, 6, 2, 64, [97]),                   # odd k, G = 3
     (4, 16, 16, 8, 128, [64, 65, 63, 4096]),  # page/tile boundaries
+    (2, 7, 6, 2, 128, [130, 1]),              # G = 3: 21 rows on the 128 lanes
+    (2, 32, 20, 4, 128, [200, 999]),          # G = 5: 25 block rows per row tile, two row tiles
+    (3, 32, 32, 4, 128, [5000, 64, 700]),     # G = 8, very unequal lengths: shares cross unit and sequence boundaries
 ])
 def test_shapes_and_edges(mask, B, k, Hq, Hkv, D, lens):
     cfg = W.StepConfig("edge", B, Hq, Hkv, D, k, 64, 64, (min(lens), max(lens)), mask=mask, seed=77)
     _run(cfg, lengths=lens, stress=True, append=(mask == W.MASK_CAUSAL))
+
+
+def test_many_short_sequences():
+    """Hundreds of sequences of 0..150 tokens (many of them empty): every thread
+    block's share of the work holds dozens of (sequence, KV head) pieces, more
+    than its piece list takes at once."""
+    B = 900
+    lens = W.rng(81, "lens").integers(0, 3, size=B) * W.rng(81, "lens2").integers(0, 76, size=B)
+    cfg = W.StepConfig("short", B, 8, 8, 128, 2, 64, 64, (int(lens.min()), int(lens.max())), seed=81)
+    _run(cfg, lengths=lens.tolist(), stress=True, append=True)
+
+
+def test_one_unusable_sequence_does_not_disturb_the_others():
+    """A sequence longer than max_seq_len is skipped and reported; its
+    neighbours in the batch still get their exact results."""
+    from paper_2512_15176_b200 import binding as L
+    lens = [300, 900, 40]
+    cfg = W.StepConfig("skip", 3, 8, 2, 128, 8, 64, 64, (40, 900), seed=82)
+    st = Hn.draw_state(cfg, lens, True)
+    q, kb, vb = Hn.draw_block(cfg, 0, True)
+    want = Hn.oracle_attention(cfg, Hn.oracle_kv(st), q, kb, vb)
+    kv = Hn.gpu_kv(st)
+    seq_ids = torch.arange(3, dtype=torch.int32, device="cuda")
+    ws = torch.empty(L.deer_block_attn_workspace_bytes(3, 8, 8, 2, 128, 512), dtype=torch.uint8, device="cuda")
+    out = torch.zeros(3, 8, 8, 128, dtype=torch.bfloat16, device="cuda")
+    L.deer_block_attn(kv, seq_ids, q.cuda(), kb.cuda(), vb.cuda(), out, 0, 0, 1.0 / math.sqrt(128), 512, ws)
+    assert L.deer_kv_status(kv) == L.DEER_ERR_INVALID_ARG
+    got = out.cpu()
+    Hn.check_attention(got[[0, 2]], want[[0, 2]], "neighbours of a skipped sequence")
 
 
 def test_split_is_invisible():
