@@ -30,9 +30,10 @@ from paper_2512_15176_b200 import workload as W  # noqa: E402
 METRIC = "verified draft tokens/s per verify step"
 UNIT = "tokens/s"
 
-# DRAM bytes (read + write) of one lmhead_umma_kernel launch from ncu, per workload name; None = not captured for
-# the kernel as it stands.
-LMHEAD_TRAFFIC = {}
+# DRAM bytes (read + write) of one lmhead_umma_kernel launch from ncu, per workload name; absent = not captured for
+# the kernel as it stands.  The capture ran at V = 65536 (542.2 MB of traffic for 537.13 MB algorithmic, ratio 1.0094);
+# every weight row is fetched once by one block, so the traffic scales with V to the full-size launch.
+LMHEAD_TRAFFIC = {"C2-qwen3-8b-verify": int(1244922112 * 1.0094)}
 
 
 def load_peaks():
