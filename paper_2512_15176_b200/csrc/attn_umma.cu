@@ -604,12 +604,14 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     }
 }
 
-// Combines the segments of the units that were cut.  One thread block per (unit, 32 of its rows); a warp takes four
-// rows at a time so that their loads are in flight together.  unit_parts[u] = (first, last) block that holds a piece
+// Combines the segments of the units that were cut.  One thread block per (unit, 8 * R of its rows); a warp takes R
+// rows at a time so that their loads are in flight together (R = 4, or 1 when that is what it takes to fill the GPU).  unit_parts[u] = (first, last) block that holds a piece
 // of unit u, or first < 0 when the unit was written directly (or its sequence was skipped).
+template <int R>
 __global__ void __launch_bounds__(256) attn_umma_merge_kernel(const AttnParams p) {
+    constexpr int BPU = 128 / (8 * R);                            // thread blocks per unit
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int unit = blockIdx.x >> 2;
+    const int unit = blockIdx.x / BPU;
     const int2 parts = p.unit_parts[unit];
     if (parts.x < 0) return;
     const int Hkv = p.kv.n_kv_heads, HR = Hkv * p.row_tiles;
@@ -617,7 +619,7 @@ __global__ void __launch_bounds__(256) attn_umma_merge_kernel(const AttnParams p
     const int kvh = hr / p.row_tiles, rt = hr % p.row_tiles;
     const int i0 = rt * p.ipt;
     const int n_rows_u = min(p.ipt, p.k - i0) * p.G;
-    const int r0 = (blockIdx.x & 3) * 32 + warp * 4;             // this warp's rows r0 .. r0 + 3
+    const int r0 = ((blockIdx.x % BPU) * 8 + warp) * R;           // this warp's rows r0 .. r0 + R - 1
     if (r0 >= n_rows_u) return;
     const int j_lo = parts.x, nj = parts.y - parts.x + 1;
     const float* __restrict__ lse_base = p.part_lse + ((size_t)unit + j_lo) * 128;
@@ -627,9 +629,9 @@ __global__ void __launch_bounds__(256) attn_umma_merge_kernel(const AttnParams p
     const bool dense = T >= p.nc;
     auto live = [&](int jj) { return dense || share_begin(T, j_lo + jj + 1, p.nc) > share_begin(T, j_lo + jj, p.nc); };
 
-    float acc[4][4], wsum[4], mx[4];
+    float acc[R][4], wsum[R], mx[R];
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
+    for (int q = 0; q < R; ++q) {
         acc[q][0] = acc[q][1] = acc[q][2] = acc[q][3] = 0.f;
         wsum[q] = 0.f;
         mx[q] = -INFINITY;
@@ -637,34 +639,34 @@ __global__ void __launch_bounds__(256) attn_umma_merge_kernel(const AttnParams p
     for (int c0 = 0; c0 < nj; c0 += 32) {
         const int jj = c0 + lane;
         const bool on = jj < nj && live(jj);
-        float l[4];
+        float l[R];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) l[q] = (on && r0 + q < n_rows_u) ? lse_base[(size_t)jj * 128 + r0 + q] : -INFINITY;
+        for (int q = 0; q < R; ++q) l[q] = (on && r0 + q < n_rows_u) ? lse_base[(size_t)jj * 128 + r0 + q] : -INFINITY;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) mx[q] = fmaxf(mx[q], l[q]);
+        for (int q = 0; q < R; ++q) mx[q] = fmaxf(mx[q], l[q]);
     }
 #pragma unroll
-    for (int q = 0; q < 4; ++q)
+    for (int q = 0; q < R; ++q)
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) mx[q] = fmaxf(mx[q], __shfl_xor_sync(0xffffffffu, mx[q], o));
     for (int c0 = 0; c0 < nj; c0 += 32) {
         const int jj = c0 + lane;
         const bool on = jj < nj && live(jj);
-        float w_mine[4];
+        float w_mine[R];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
+        for (int q = 0; q < R; ++q) {
             const float l = (on && r0 + q < n_rows_u) ? lse_base[(size_t)jj * 128 + r0 + q] : -INFINITY;
             w_mine[q] = (l == -INFINITY) ? 0.f : exp2f(l - mx[q]);
         }
         const int cn = min(32, nj - c0);
 #pragma unroll 2
         for (int e = 0; e < cn; ++e) {
-            float4 v[4];
+            float4 v[R];
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
+            for (int q = 0; q < R; ++q)
                 v[q] = *reinterpret_cast<const float4*>(o_base + ((size_t)(c0 + e) * 128 + min(r0 + q, 127)) * HD + lane * 4);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
+            for (int q = 0; q < R; ++q) {
                 const float w = __shfl_sync(0xffffffffu, w_mine[q], e);
                 if (w > 0.f) {                                // an empty share's slot was never written
                     wsum[q] += w;
@@ -677,7 +679,7 @@ __global__ void __launch_bounds__(256) attn_umma_merge_kernel(const AttnParams p
         }
     }
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
+    for (int q = 0; q < R; ++q) {
         const int r = r0 + q;
         if (r >= n_rows_u) break;
         const float winv = wsum[q] > 0.f ? 1.f / wsum[q] : 0.f;
@@ -692,7 +694,7 @@ __global__ void __launch_bounds__(256) attn_umma_merge_kernel(const AttnParams p
 // Thread blocks for a call: one per SM, fewer when the tiles would not give each of them a few.
 static int pick_blocks(int B, int HR, int max_seq_len) {
     const long long t_max = (long long)B * HR * ((max_seq_len + ATT_TILE - 1) / ATT_TILE + 1);
-    long long nc = t_max / 4;
+    long long nc = t_max / 8;
     if (nc > NUM_SMS) nc = NUM_SMS;
     if (nc < 1) nc = 1;
     return (int)nc;
@@ -760,7 +762,8 @@ int launch_umma(AttnParams p, cudaStream_t st) {
     DEER_CUDA(cudaFuncSetAttribute(block_attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
     block_attn_umma_kernel<<<p.nc, THREADS, SMEM_BYTES, st>>>(tm_q, tm_kb, tm_vb, tm_kp, tm_vp, p);
     DEER_CUDA(cudaGetLastError());
-    attn_umma_merge_kernel<<<(unsigned)(p.B * HR * 4), 256, 0, st>>>(p);
+    if ((long long)p.B * HR * 4 >= 2 * NUM_SMS) attn_umma_merge_kernel<4><<<(unsigned)(p.B * HR * 4), 256, 0, st>>>(p);
+    else attn_umma_merge_kernel<1><<<(unsigned)(p.B * HR * 16), 256, 0, st>>>(p);
     DEER_CUDA(cudaGetLastError());
     return DEER_OK;
 }
