@@ -552,6 +552,7 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         }
                     }
                     tcgen05_fence_before();
+                    if (wtid == 0) p.unit_parts[unit] = make_int2(-1, -1);      // nothing for the merge kernel to do
                     continue;
                 }
                 // partial result: O / l and the log2-sum-exp, in slot (unit index + block index)
@@ -605,17 +606,19 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 }
 
 // Combines the segments of the units that were cut.  One thread block per (unit, 8 * R of its rows); a warp takes R
-// rows at a time so that their loads are in flight together (R = 4, or 1 when that is what it takes to fill the GPU).  unit_parts[u] = (first, last) block that holds a piece
-// of unit u, or first < 0 when the unit was written directly (or its sequence was skipped).
+// rows at a time so that their loads are in flight together (R = 4, or 1 when that is what it takes to fill the GPU).
+// unit_parts[u] = (first, last) block that holds a piece of unit u, or first < 0 when the unit was written directly.
 template <int R>
 __global__ void __launch_bounds__(256) attn_umma_merge_kernel(const AttnParams p) {
     constexpr int BPU = 128 / (8 * R);                            // thread blocks per unit
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int unit = blockIdx.x / BPU;
-    const int2 parts = p.unit_parts[unit];
-    if (parts.x < 0) return;
     const int Hkv = p.kv.n_kv_heads, HR = Hkv * p.row_tiles;
     const int b = unit / HR, hr = unit % HR;
+    // the entry of a unit is written by the block that holds the unit's first tile; a skipped sequence has no tiles
+    if (seq_tiles(p, b, nullptr, nullptr) == 0) return;
+    const int2 parts = p.unit_parts[unit];
+    if (parts.x < 0) return;
     const int kvh = hr / p.row_tiles, rt = hr % p.row_tiles;
     const int i0 = rt * p.ipt;
     const int n_rows_u = min(p.ipt, p.k - i0) * p.G;
@@ -728,7 +731,6 @@ int launch_umma(AttnParams p, cudaStream_t st) {
     p.part_lse = p.part_o + slots * 128 * HD;
     p.total_tiles = reinterpret_cast<long long*>(p.part_lse + slots * 128);      // 8-byte aligned: slots * 128 * 129 floats
     p.unit_parts = reinterpret_cast<int2*>(p.total_tiles + 1);
-    DEER_CUDA(cudaMemsetAsync(p.unit_parts, 0xFF, (size_t)p.B * HR * sizeof(int2), st));     // "no pieces to merge"
     const int box_i = p.ipt < p.k ? p.ipt : p.k;
     const uint64_t rows = (uint64_t)p.B * p.k;
 
