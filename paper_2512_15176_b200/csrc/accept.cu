@@ -131,9 +131,9 @@ __global__ void __launch_bounds__(128) accept_scan_kernel(int B, int k, const in
 }
 
 // ---------------------------------------------------------------- sample (c)
-// The residual of the one rejected row of a sequence.  Probabilities are recomputed from the fp32 logits in
-// fp64 wherever they are needed instead of being stored: p(v) = exp(z_p/T - lse_p) / Sp with Sp the fp64 sum of the
-// numerators (lse_p is only fp32-accurate), likewise q.
+// The residual of the one rejected row of a sequence, in fp64: p(v) = exp(z_p/T - lse_p) / Sp with Sp the fp64 sum of
+// the numerators (lse_p is only fp32-accurate), likewise q.  The numerators are computed once (the fp64 exponential is
+// what this path costs) and kept in the workspace for the second pass.
 struct ResidualArgs {
     int B, k, V, slice;
     const int32_t* rej_pos;
@@ -143,6 +143,8 @@ struct ResidualArgs {
     const float* lse_q;
     double temperature;
     const float* r;
+    double* e_p;                  // [B][V]  exp(z_p/T - lse_p) of the rejected row
+    double* e_q;                  // [B][V]  exp(z_q - lse_q)
     double* sums;                 // [B][NS][4]: sum e_p, sum e_q, residual mass of the slice, unused
     int32_t* done;                // [B] slices finished (zeroed by the scan kernel)
     int32_t* out_ids;
@@ -188,9 +190,14 @@ __global__ void __launch_bounds__(RES_THREADS) residual_norm_kernel(ResidualArgs
     const double lp = (double)a.lse_p[row], lq = (double)a.lse_q[row], it = 1.0 / a.temperature;
     const int v0 = sl * a.slice, v1 = min(a.V, v0 + a.slice);
     double sp = 0.0, sq = 0.0;
+    double* ep = a.e_p + (size_t)b * a.V;
+    double* eq = a.e_q + (size_t)b * a.V;
     for (int v = v0 + threadIdx.x; v < v1; v += RES_THREADS) {
-        sp += exp((double)zp[v] * it - lp);
-        sq += exp((double)zq[v] - lq);
+        const double x = exp((double)zp[v] * it - lp), y = exp((double)zq[v] - lq);
+        ep[v] = x;
+        eq[v] = y;
+        sp += x;
+        sq += y;
     }
     sp = block_sum(sp, sh);
     sq = block_sum(sq, sh);
@@ -214,19 +221,17 @@ __global__ void __launch_bounds__(RES_THREADS) residual_pick_kernel(ResidualArgs
         if (sl == 0 && tid == 0 && a.eos_id >= 0) cut_at_eos(a, b);
         return;
     }
-    const size_t row = (size_t)b * a.k + i;
-    const float* zp = a.target_logits + row * a.V;
-    const float* zq = a.draft_logits + row * a.V;
-    const double lp = (double)a.lse_p[row], lq = (double)a.lse_q[row], it = 1.0 / a.temperature;
+    const double* ep = a.e_p + (size_t)b * a.V;
+    const double* eq = a.e_q + (size_t)b * a.V;
     double Sp = 0.0, Sq = 0.0;
     for (int j = 0; j < NS; ++j) {
         Sp += a.sums[((size_t)b * NS + j) * 4 + 0];
         Sq += a.sums[((size_t)b * NS + j) * 4 + 1];
     }
     const double ip = 1.0 / Sp, iq = 1.0 / Sq;
-    auto prob_p = [&](int v) { return exp((double)zp[v] * it - lp) * ip; };
+    auto prob_p = [&](int v) { return ep[v] * ip; };
     auto resid = [&](int v) {
-        const double res = prob_p(v) - exp((double)zq[v] - lq) * iq;
+        const double res = ep[v] * ip - eq[v] * iq;
         return res > 0.0 ? res : 0.0;
     };
     {
@@ -314,6 +319,8 @@ struct SampleWs {
     float* lse_q;
     float* zq_draft;
     int32_t* rej_pos;
+    double* e_p;
+    double* e_q;
     double* sums;
     int32_t* done;
     size_t bytes;
@@ -332,6 +339,8 @@ SampleWs carve(void* base, int B, int k, int V) {
     w.lse_q = static_cast<float*>(take((size_t)B * k * sizeof(float)));
     w.zq_draft = static_cast<float*>(take((size_t)B * k * sizeof(float)));
     w.rej_pos = static_cast<int32_t*>(take((size_t)B * sizeof(int32_t)));
+    w.e_p = static_cast<double*>(take((size_t)B * V * sizeof(double)));
+    w.e_q = static_cast<double*>(take((size_t)B * V * sizeof(double)));
     w.sums = static_cast<double*>(take((size_t)B * NS * 4 * sizeof(double)));
     w.done = static_cast<int32_t*>(take((size_t)B * sizeof(int32_t)));
     w.bytes = off;
@@ -391,6 +400,8 @@ extern "C" int deer_accept(int mode, int B, int k, int V, const int32_t* draft_i
     a.lse_q = w.lse_q;
     a.temperature = (double)temperature;
     a.r = r;
+    a.e_p = w.e_p;
+    a.e_q = w.e_q;
     a.sums = w.sums;
     a.done = w.done;
     a.out_ids = out_ids;
