@@ -247,18 +247,21 @@ def run_ours(args, cfg):
     for _ in range(max(args.warmup, 3)):
         one_step()
     torch.cuda.synchronize()
+    graph, gev = None, None
     if not args.no_graph:
-        # The step's launches are replayed from CUDA graphs (one per phase, so that events can sit between them):
+        # The whole step is replayed from one CUDA graph, with timing events recorded inside it between the phases:
         # the host's launch work no longer paces the GPU.  The calls and their arguments are exactly the ones above.
-        graphs = []
-        for ph in phases:
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g):
+        gev = [torch.cuda.Event(enable_timing=True, external=True) for _ in range(4)]
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for i, ph in enumerate(phases):
+                gev[i].record()
                 ph()
-            graphs.append(g)
-        phases = [g.replay for g in graphs]
+            gev[3].record()
         for _ in range(3):
-            one_step()
+            restore()
+            flush_l2()
+            graph.replay()
         torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
@@ -266,18 +269,28 @@ def run_ours(args, cfg):
     if rank == 0:
         sampler.start()
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    marks = []          # per step: ms from the step's start to the end of each phase
     torch.cuda.synchronize()
     wall0 = time.perf_counter()
     for s in range(args.steps):
-        one_step(evs[s])
+        if graph is None:
+            one_step(evs[s])
+        else:
+            restore()
+            flush_l2()
+            graph.replay()
+            torch.cuda.synchronize()          # the graph's events are re-recorded by the next replay: read them now
+            marks.append([gev[0].elapsed_time(gev[i]) for i in (1, 2, 3)])
     torch.cuda.synchronize()
     wall = time.perf_counter() - wall0
     if world > 1:
         dist.barrier()
     clocks = sampler.stop() if rank == 0 else None
-    step_ms = [e[0].elapsed_time(e[3]) for e in evs]
-    attn_ms = [e[0].elapsed_time(e[1]) for e in evs]
-    lm_ms = [e[1].elapsed_time(e[2]) for e in evs]
+    if graph is None:
+        marks = [[e[0].elapsed_time(e[i]) for i in (1, 2, 3)] for e in evs]
+    step_ms = [m[2] for m in marks]
+    attn_ms = [m[0] for m in marks]
+    lm_ms = [m[1] - m[0] for m in marks]
     total_ms = float(sum(step_ms))
     status = L.deer_kv_status(kv)
     accepted = int(vs.accept_len.sum().item())
@@ -340,7 +353,7 @@ def run_ours(args, cfg):
         "config": {"workload": cfg.name, "B": cfg.B, "k": cfg.k, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D,
                    "ctx": [int(lengths.min()), int(lengths.max())], "hid": cfg.hid, "V": cfg.V,
                    "mask": "bidirectional" if bidir else "causal", "accept": accept_text, "parallelism": f"replicas x{world}",
-                   "launch": "host launches" if args.no_graph else "three CUDA graphs per step (attention phase, LM head, acceptance + commit)",
+                   "launch": "host launches" if args.no_graph else "one CUDA graph per step, timing events recorded inside it",
                    "l2": "flushed between steps by a 512 MiB write followed by a 256 MiB read; the weight stream exceeds L2 by itself"},
         "roofline": {"bound": bound, "kernel": "deer_lmhead_select", "achieved": achieved, "peak": peak,
                      "unit": unit, "frac": achieved / peak, "traffic": LMHEAD_TRAFFIC.get(cfg.name), "peak_source": peaks["source"],
