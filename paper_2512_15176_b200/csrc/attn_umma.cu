@@ -190,7 +190,13 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 
     // ---- this block's share of the flattened tile list ----
     long long T = 0;
-    for (int b = lane; b < p.B; b += 32) T += seq_tiles(p, b, nullptr, nullptr);
+    for (int b = lane; b < p.B; b += 32) {
+        const int tiles = seq_tiles(p, b, nullptr, nullptr);
+        T += tiles;
+        // a sequence that cannot be used has no tiles, so no block will write its units' merge entries: do it here
+        if (tiles == 0 && j == 0 && warp == 0)
+            for (int hr = 0; hr < HR; ++hr) p.unit_parts[(size_t)b * HR + hr] = make_int2(-1, -1);
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) T += __shfl_xor_sync(0xffffffffu, T, o);
     T *= HR;
@@ -615,8 +621,7 @@ __global__ void __launch_bounds__(256) attn_umma_merge_kernel(const AttnParams p
     const int unit = blockIdx.x / BPU;
     const int Hkv = p.kv.n_kv_heads, HR = Hkv * p.row_tiles;
     const int b = unit / HR, hr = unit % HR;
-    // the entry of a unit is written by the block that holds the unit's first tile; a skipped sequence has no tiles
-    if (seq_tiles(p, b, nullptr, nullptr) == 0) return;
+    // written by the block that holds the unit's first tile (by block 0 for a sequence that was skipped)
     const int2 parts = p.unit_parts[unit];
     if (parts.x < 0) return;
     const int kvh = hr / p.row_tiles, rt = hr % p.row_tiles;
