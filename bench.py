@@ -100,6 +100,16 @@ class ClockSampler:
                 "samples": len(self.sm), "power_w_max": max(self.power) if self.power else None}
 
 
+def max_over_ranks(values, device, world):
+    """Element-wise maximum of ``values`` over all ranks (the replicas are independent, so the job's time is the
+    slowest rank's); with one rank the values themselves."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
 def dist_env():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -320,10 +330,7 @@ def run_ours(args, cfg):
             dt = time.perf_counter() - t0
             if s >= 3:
                 e2e_s += dt
-    e2e_s_t = torch.tensor([total_ms / 1e3, e2e_s], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(e2e_s_t, op=dist.ReduceOp.MAX)
-    total_s, e2e_total = float(e2e_s_t[0]), float(e2e_s_t[1])
+    total_s, e2e_total = max_over_ranks([total_ms / 1e3, e2e_s], dev, world)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
