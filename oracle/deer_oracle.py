@@ -285,3 +285,42 @@ class PagedKV:
         n = int(self.seq_len[s])
         return (gather_prefix(self.k_pool, self.page_table[s], n, self.page_size),
                 gather_prefix(self.v_pool, self.page_table[s], n, self.page_size))
+
+
+# --------------------------------------------------------------------------
+# (5) Algorithm 1's outer loop: "while the last token is not EOS ... append the
+#     chosen tokens to the prefix ... update j <- length(x)".  One call of
+#     emit() is the book-keeping of one pass of that loop for every sequence:
+#     what was chosen in this block joins the sequence's output, the sequence
+#     ends at an EOS or at a length limit, and only the accepted draft tokens
+#     that were really emitted stay in the KV cache.
+# --------------------------------------------------------------------------
+
+class DecodeState:
+    """Output tokens of every sequence over the passes of the loop."""
+
+    def __init__(self, B, max_new):
+        self.max_new = int(max_new)
+        self.tokens = np.full((B, max_new), -1, dtype=np.int32)
+        self.n_tokens = np.zeros(B, dtype=np.int32)
+        self.finished = np.zeros(B, dtype=np.int32)
+
+    def emit(self, accept_len, out_ids, n_out, eos_id=-1):
+        """Append this block's chosen tokens (``out_ids[b][:n_out[b]]``, already cut
+        after an EOS by the acceptance rule).  A sequence that has finished emits
+        nothing and keeps nothing.  Returns keep [B]: cache rows to commit."""
+        B = self.tokens.shape[0]
+        keep = np.zeros(B, dtype=np.int32)
+        for b in range(B):
+            if self.finished[b]:
+                continue
+            room = self.max_new - int(self.n_tokens[b])
+            m = min(int(n_out[b]), room)
+            for i in range(m):
+                self.tokens[b, self.n_tokens[b] + i] = out_ids[b][i]
+            self.n_tokens[b] += m
+            keep[b] = min(int(accept_len[b]), m)
+            hit_eos = eos_id >= 0 and any(int(out_ids[b][i]) == eos_id for i in range(m))
+            if hit_eos or self.n_tokens[b] >= self.max_new:
+                self.finished[b] = 1
+        return keep
