@@ -228,6 +228,26 @@ int deer_accept(int mode, int B, int k, int V,
                 void* workspace, size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------
+ * (5) Book-keeping of one pass of Algorithm 1's outer loop ("while the last
+ * token is not EOS": the tokens chosen in this block are appended to the
+ * output, "update j <- length(x)").  For every sequence that has not finished:
+ * out_ids[b][0 .. n_out[b]) (deer_accept's output, already cut after an EOS) is
+ * appended to tokens[b] as far as max_new allows; the sequence finishes when an
+ * appended token equals eos_id (eos_id < 0 disables) or when it holds max_new
+ * tokens; keep[b] = min(accept_len[b], tokens appended) is what
+ * deer_kv_commit should keep.  A finished sequence appends nothing and gets
+ * keep[b] = 0, so it may stay in the batch of later passes.
+ *   accept_len, n_out  i32 [B];  out_ids  i32 [B][k]
+ *   tokens    i32 [B][max_new]  output tokens so far (caller fills it with -1 before the first pass)
+ *   n_tokens  i32 [B]           their number           (caller zeroes it before the first pass)
+ *   finished  i32 [B]           0 / 1                  (caller zeroes it before the first pass)
+ *   keep      i32 [B]           out
+ * ---------------------------------------------------------------------- */
+int deer_emit(int B, int k, const int32_t* accept_len, const int32_t* out_ids, const int32_t* n_out,
+              int32_t eos_id, int32_t max_new, int32_t* tokens, int32_t* n_tokens, int32_t* finished,
+              int32_t* keep, void* stream);
+
+/* ------------------------------------------------------------------------
  * One whole greedy verify step with HOST inputs and outputs (Algorithm 1, one
  * iteration of the while loop on the verifier side): copies the block's
  * q/k_blk/v_blk, hidden states and draft ids from host memory to the device

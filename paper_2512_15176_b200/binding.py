@@ -25,7 +25,7 @@ EXPORTS = [
     "deer_last_error", "deer_kv_create", "deer_kv_destroy", "deer_kv_reserve", "deer_kv_commit", "deer_kv_status",
     "deer_block_attn_workspace_bytes", "deer_block_attn", "deer_lmhead_workspace_bytes", "deer_lmhead_select",
     "deer_accept_workspace_bytes", "deer_accept", "deer_verify_step_host",
-    "deer_lmhead_static_max_rows", "deer_lmhead_select_static",
+    "deer_lmhead_static_max_rows", "deer_lmhead_select_static", "deer_emit",
 ]
 
 
@@ -85,6 +85,8 @@ def lib() -> ctypes.CDLL:
     L.deer_accept.argtypes = [c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_float,
                               c_void_p, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t,
                               c_void_p]
+    L.deer_emit.argtypes = [c_int, c_int, c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p,
+                            c_void_p]
     L.deer_verify_step_host.argtypes = [c_void_p, POINTER(deer_step_dev), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                         c_void_p, c_int, c_int, c_int, c_int, c_int, c_float, c_int, c_void_p, c_void_p,
                                         c_void_p, c_void_p]
@@ -224,6 +226,12 @@ def deer_accept(mode, B, k, V, draft_ids, target_ids, target_logits, target_lse,
                              _ptr(accept_len), _ptr(out_ids), _ptr(n_out), _ptr(workspace),
                              workspace.numel() * workspace.element_size() if workspace is not None else 0,
                              _stream(stream)))
+
+
+def deer_emit(accept_len, out_ids, n_out, eos_id, tokens, n_tokens, finished, keep, stream=None):
+    B, k = out_ids.shape
+    _check(lib().deer_emit(B, k, _ptr(accept_len), _ptr(out_ids), _ptr(n_out), int(eos_id), tokens.shape[1], _ptr(tokens),
+                           _ptr(n_tokens), _ptr(finished), _ptr(keep), _stream(stream)))
 
 
 def deer_verify_step_host(kv: KVCache, dev: deer_step_dev, w, q_host, k_blk_host, v_blk_host, h_host, draft_ids_host,

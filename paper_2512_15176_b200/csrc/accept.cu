@@ -315,6 +315,35 @@ __global__ void __launch_bounds__(RES_THREADS) residual_pick_kernel(ResidualArgs
     }
 }
 
+// ---------------------------------------------------------------- loop book-keeping
+// One thread per sequence: append this block's chosen tokens to the sequence's output, decide whether the
+// sequence has finished (EOS or length limit), and how many cache rows survive (Algorithm 1's outer loop).
+__global__ void emit_kernel(int B, int k, const int32_t* __restrict__ accept_len, const int32_t* __restrict__ out_ids,
+                            const int32_t* __restrict__ n_out, int32_t eos_id, int32_t max_new, int32_t* __restrict__ tokens,
+                            int32_t* __restrict__ n_tokens, int32_t* __restrict__ finished, int32_t* __restrict__ keep) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    if (finished[b]) {
+        keep[b] = 0;
+        return;
+    }
+    const int have = n_tokens[b];
+    int m = n_out[b];
+    m = m < 0 ? 0 : (m > k ? k : m);
+    if (m > max_new - have) m = max_new - have;
+    if (m < 0) m = 0;
+    bool eos = false;
+    for (int i = 0; i < m; ++i) {
+        const int32_t t = out_ids[(size_t)b * k + i];
+        tokens[(size_t)b * max_new + have + i] = t;
+        eos |= (eos_id >= 0 && t == eos_id);
+    }
+    n_tokens[b] = have + m;
+    const int a = accept_len[b];
+    keep[b] = a < m ? (a < 0 ? 0 : a) : m;
+    if (eos || have + m >= max_new) finished[b] = 1;
+}
+
 struct SampleWs {
     float* lse_q;
     float* zq_draft;
@@ -348,6 +377,19 @@ SampleWs carve(void* base, int B, int k, int V) {
 }
 
 }  // namespace
+
+extern "C" int deer_emit(int B, int k, const int32_t* accept_len, const int32_t* out_ids, const int32_t* n_out, int32_t eos_id,
+                         int32_t max_new, int32_t* tokens, int32_t* n_tokens, int32_t* finished, int32_t* keep, void* stream) {
+    DEER_CHECK_ARG(accept_len && out_ids && n_out && (tokens || max_new == 0) && n_tokens && finished && keep, DEER_ERR_INVALID_ARG,
+                   "deer_emit: null argument");
+    DEER_CHECK_ARG(k >= 1 && k <= DEER_MAX_BLOCK, DEER_ERR_UNSUPPORTED, "deer_emit: k must be in [1, 32]");
+    DEER_CHECK_ARG(B >= 0 && max_new >= 0, DEER_ERR_INVALID_ARG, "deer_emit: B and max_new must not be negative");
+    if (B == 0) return DEER_OK;
+    emit_kernel<<<(B + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(B, k, accept_len, out_ids, n_out, eos_id, max_new,
+                                                                               tokens, n_tokens, finished, keep);
+    DEER_CUDA(cudaGetLastError());
+    return DEER_OK;
+}
 
 extern "C" size_t deer_accept_workspace_bytes(int mode, int B, int k, int V) {
     if (mode != DEER_ACC_SAMPLE || B <= 0 || k <= 0 || V <= 0) return 0;

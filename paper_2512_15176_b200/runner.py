@@ -53,6 +53,7 @@ class VerifyStep:
         self.lm_ws = _ws(L.deer_lmhead_workspace_bytes(M, cfg.hid, V), dev)
         self.acc_ws = _ws(L.deer_accept_workspace_bytes(L.DEER_ACC_SAMPLE if sample else L.DEER_ACC_GREEDY, B, k, V), dev)
         self.scale = 1.0 / math.sqrt(D)
+        self.eos_id = -1                # Algorithm 1's EOS break inside a block; < 0 disables
 
     # ---- inputs -------------------------------------------------------------
     def load(self, q=None, k_blk=None, v_blk=None, h=None, draft_ids=None, q_logits=None, u=None, r=None):
@@ -91,11 +92,11 @@ class VerifyStep:
         c = self.cfg
         if c.mode == "sample":
             L.deer_accept(L.DEER_ACC_SAMPLE, c.B, c.k, c.V, self.draft_ids, None, self.logits, self.lse, self.draft_logit,
-                          c.temperature, self.q_logits, self.u, self.r, -1, self.accept_len, self.out_ids, self.n_out,
+                          c.temperature, self.q_logits, self.u, self.r, self.eos_id, self.accept_len, self.out_ids, self.n_out,
                           self.acc_ws)
         else:
             L.deer_accept(L.DEER_ACC_GREEDY, c.B, c.k, c.V, self.draft_ids, self.target_ids, None, None, None, 1.0, None,
-                          None, None, -1, self.accept_len, self.out_ids, self.n_out, None)
+                          None, None, self.eos_id, self.accept_len, self.out_ids, self.n_out, None)
 
     def commit(self):
         L.deer_kv_commit(self.kv, self.seq_ids, self.accept_len, self.cfg.k)
@@ -118,3 +119,29 @@ class VerifyStep:
         if self.cfg.mask == MASK_BIDIR:
             return 4
         return 2 + 2 + 2 + (4 if self.cfg.mode == "sample" else 1)
+
+
+class DecodeLoop:
+    """Algorithm 1's outer loop over a batch: every pass runs one verify step
+    and then ``deer_emit`` -- the chosen tokens join each sequence's output,
+    a sequence ends at an EOS or at ``max_new`` tokens, and the cache keeps only
+    the accepted drafts that were emitted.  Nothing synchronises with the host
+    between passes; finished sequences stay in the batch and are ignored."""
+
+    def __init__(self, step: VerifyStep, eos_id: int, max_new: int):
+        self.vs, self.eos_id = step, int(eos_id)
+        step.eos_id = int(eos_id)
+        B, dev = step.cfg.B, step.q.device
+        self.tokens = torch.full((B, max_new), -1, dtype=torch.int32, device=dev)
+        self.n_tokens = torch.zeros(B, dtype=torch.int32, device=dev)
+        self.finished = torch.zeros(B, dtype=torch.int32, device=dev)
+        self.keep = torch.zeros(B, dtype=torch.int32, device=dev)
+
+    def one_pass(self):
+        vs = self.vs
+        vs.reserve()
+        vs.attn(append=True)
+        vs.lmhead()
+        vs.accept()
+        L.deer_emit(vs.accept_len, vs.out_ids, vs.n_out, self.eos_id, self.tokens, self.n_tokens, self.finished, self.keep)
+        L.deer_kv_commit(vs.kv, vs.seq_ids, self.keep, vs.cfg.k)
