@@ -396,8 +396,18 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every call from the host instead of replaying CUDA graphs")
+    ap.add_argument("--sweep-point", default=None, metavar="B,CTX,K,MASK",
+                    help="time one point of the sweep instead of a fixed workload: batch, context (ragged lengths in "
+                         "[CTX/2, CTX]), block size, causal|bidir")
     args = ap.parse_args()
-    cfg = W.config(args.config)
+    if args.sweep_point:
+        b, ctx, k, mask = args.sweep_point.split(",")
+        cfg = W.sweep_config(int(b), int(ctx), int(k), W.MASK_BIDIR if mask == "bidir" else W.MASK_CAUSAL, steps=1)
+        if mask == "bidir":
+            cfg = cfg.with_(mode="argmax_logprob")
+        args.no_cpu_baseline = True
+    else:
+        cfg = W.config(args.config)
     if args.impl == "reference" and cfg.mode != "greedy":
         raise SystemExit("the oracle arm times the greedy verify step (workload 0 or 1)")
     if args.impl == "reference":
