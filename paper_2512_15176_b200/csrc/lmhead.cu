@@ -11,7 +11,7 @@
 namespace lmhead {
 
 bool umma_supported(int M, int hid, int V);
-int launch_umma(const Params& p, int need_sum, int* nparts_out, cudaStream_t st);
+int launch_umma(const Params& p, int need_sum, bool allow_pair, int* nparts_out, cudaStream_t st);
 
 struct FinalizeArgs {
     const Partial* part;
@@ -125,12 +125,14 @@ extern "C" int deer_lmhead_select(const void* h, const void* w, int M, int hid, 
     p.out_logits = out_logits;
     p.part = static_cast<Partial*>(workspace);
     p.nparts = pl.nparts;
-    // DEER_LMHEAD_IMPL=mma forces the warp-level kernel (used to cross-check the tcgen05 one)
+    // DEER_LMHEAD_IMPL=mma forces the warp-level kernel, =single the one-block tcgen05 kernel at every M
+    // (used to cross-check the kernels against each other)
     const char* force = getenv("DEER_LMHEAD_IMPL");
     const bool use_umma = umma_supported(M, hid, V) && !(force && strcmp(force, "mma") == 0);
+    const bool allow_pair = !(force && strcmp(force, "single") == 0);
     int nparts = pl.nparts;
     int rc;
-    if (use_umma) rc = launch_umma(p, mode != DEER_SEL_ARGMAX, &nparts, st);
+    if (use_umma) rc = launch_umma(p, mode != DEER_SEL_ARGMAX, allow_pair, &nparts, st);
     else if (pl.bm == 32) rc = launch<32>(p, pl, st);
     else if (pl.bm == 64) rc = launch<64>(p, pl, st);
     else rc = launch<128>(p, pl, st);

@@ -259,6 +259,169 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
     }
 }
 
+// ---- CTA-pair variant (more than 128 block rows) ------------------------------------
+// Two thread blocks of a cluster share every weight tile: one tcgen05.mma with cta_group::2 covers 256 block
+// rows (128 per block, in that block's tensor memory) and reads half of the N-row weight tile from each
+// block's shared memory, so each block stages 16 KB of h and N/2 rows of w per 64-wide step instead of all N:
+// a third less L2 -> shared-memory traffic per flop, which is what bounds the single-block kernel at these
+// sizes.  Block 0 of the pair issues the MMAs.  Its `full` barriers count the bytes of both blocks' loads (the
+// peer's TMA completes on the leader's barrier); `empty` and `accumulator full` arrive in both blocks through
+// one multicast commit; both blocks' epilogue warps arrive on the leader's `accumulator empty`.
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
+lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ CUtensorMap tm_w_hi,
+                        const __grid_constant__ CUtensorMap tm_w_lo, const Args a) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int stage_bytes = a.stage_bytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + a.stages * stage_bytes);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * MAX_STAGES + 4);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = cluster_ctarank();
+    const bool leader = (rank == 0);
+    const int m0 = (int)(blockIdx.x >> 1) * (2 * BM) + (int)rank * BM;
+    const int part = blockIdx.y;
+    const int u0 = (int)((long)part * a.n_units / a.nparts);
+    const int u1 = (int)((long)(part + 1) * a.n_units / a.nparts);
+    const int g = u1 - u0;
+    const int N = g * 16;
+    const int half = g * 8;                      // rows of the weight tile this block stages
+    const int row_base = u0 * a.T * 16;
+    const int n_tiles = (g > 0) ? a.T : 0;
+    const int KB = a.hid / BK;
+
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t bar_base = smem_u32(bars);
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (MAX_STAGES + s); };
+    auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * MAX_STAGES + b); };
+    auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * MAX_STAGES + 2 + b); };
+
+    if (tid == 0) {
+        for (int s = 0; s < a.stages; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(tfull_bar(b), 1);
+            mbar_init(tempty_bar(b), 8);         // four epilogue warps in each of the two blocks
+        }
+        *abort_flag = 0;
+        mbar_init_fence();
+    }
+    if (warp == 1) tmem_alloc_pair(smem_u32(tmem_slot), 512);
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync();                              // the peer's barriers exist before anything signals them
+    tcgen05_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ---------------- TMA producer (each block: its 128 rows of h, its half of the weight tile) ----------------
+        if (lane == 0 && n_tiles > 0) {
+            const CUtensorMap* tm_w = (g == a.gmax) ? &tm_w_hi : &tm_w_lo;
+            const uint32_t stage_tx = 2u * (uint32_t)(A_SPAN + half * 128);
+            int it = 0;
+            bool ok = true;
+            for (int t = 0; t < n_tiles && ok; ++t) {
+                const int row0 = row_base + t * N + (int)rank * half;
+                for (int kb = 0; kb < KB; ++kb, ++it) {
+                    const int s = it % a.stages;
+                    const uint32_t ph = (uint32_t)(it / a.stages) & 1u;
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+                    if (leader) mbar_expect_tx(full_bar(s), stage_tx);
+                    const uint32_t lead_full = map_to_cta(full_bar(s), 0);
+                    const uint32_t sa = smem_base + s * stage_bytes;
+                    tma_load_2d_pair(sa + A_SPAN, tm_w, kb * BK, row0, lead_full);
+                    tma_load_2d_pair(sa, &tm_h, kb * BK, m0, lead_full);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer (leader block only) ----------------
+        if (leader && lane == 0 && n_tiles > 0) {
+            const uint32_t idesc = make_idesc_bf16_pair(N);
+            int it = 0;
+            bool ok = true;
+            for (int t = 0; t < n_tiles && ok; ++t) {
+                const int buf = t & 1;
+                const uint32_t aph = (uint32_t)(t >> 1) & 1u;
+                if (!mbar_wait(tempty_bar(buf), aph ^ 1u, abort_flag)) break;
+                tcgen05_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * MAXN);
+                for (int kb = 0; kb < KB; ++kb, ++it) {
+                    const int s = it % a.stages;
+                    const uint32_t ph = (uint32_t)(it / a.stages) & 1u;
+                    if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+                    tcgen05_fence_after();
+                    const uint32_t sa = smem_base + s * stage_bytes;
+                    const uint64_t ad = smem_desc_sw128_kmajor(sa), bd = smem_desc_sw128_kmajor(sa + A_SPAN);
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)
+                        umma_bf16_ss_pair(d_tmem, ad + 2 * k, bd + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    umma_commit_pair(empty_bar(s), 3);
+                }
+                if (ok) umma_commit_pair(tfull_bar(buf), 3);
+            }
+        }
+    } else {
+        // ---------------- epilogue: 4 warps in each block, one TMEM lane quarter each ----------------
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        const int grow = m0 + row;
+        const bool row_ok = grow < a.M;
+        const size_t zrow = (size_t)(row_ok ? grow : 0) * a.V;
+        const int draft = (row_ok && a.draft_ids && a.out_draft_logit) ? a.draft_ids[grow] : -1;
+        float run_m = -INFINITY, run_s = 0.f;
+        int32_t run_i = 0x7fffffff;
+        for (int t = 0; t < n_tiles; ++t) {
+            const int buf = t & 1;
+            const uint32_t aph = (uint32_t)(t >> 1) & 1u;
+            const bool got = mbar_wait(tfull_bar(buf), aph, abort_flag);
+            if (!__all_sync(0xffffffffu, got)) break;
+            tcgen05_fence_after();
+            const int row0 = row_base + t * N;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * MAXN);
+            for (int c = 0; c < N; c += 32) {
+                uint32_t r0[16], r1[16];
+                TMEM_LD_X16(taddr + c, r0);
+                const bool second = (c + 16 < N);
+                if (second) TMEM_LD_X16(taddr + c + 16, r1);
+                tmem_wait_ld();
+                consume16(r0, row0 + c, a.V, row_ok, a, zrow, draft, grow, run_m, run_i, run_s);
+                if (second) consume16(r1, row0 + c + 16, a.V, row_ok, a, zrow, draft, grow, run_m, run_i, run_s);
+            }
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(buf), 0));
+        }
+        if (row_ok) {
+            Partial pr;
+            pr.m = run_m;
+            pr.idx = run_i;
+            pr.s = a.need_sum ? run_s : 1.f;
+            pr.pad = 0;
+            if (*abort_flag) pr.idx = PARTIAL_ABORTED;
+            a.part[(size_t)part * a.M + grow] = pr;
+        }
+    }
+
+    // ---- tear-down: neither block leaves while the other may still signal it or read its shared memory ----
+    tcgen05_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(10000);
+        __syncthreads();
+    }
+    cluster_sync();
+    if (warp == 1) {
+        __syncwarp();
+        tcgen05_fence_after();
+        tmem_dealloc_pair(tmem_base, 512);
+    }
+}
+
 // ---- host side ------------------------------------------------------------------
 // 2-D bf16 tensor [rows][cols] (cols contiguous), box = box_rows x 64 columns.
 static int make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
@@ -274,9 +437,11 @@ bool umma_supported(int M, int hid, int V) { return M > 0 && hid % umma::BK == 0
 
 // Launches the tcgen05 kernel; the partials it writes are merged by lmhead_finalize_kernel.
 // *nparts_out receives the number of vocabulary parts written.
-int launch_umma(const Params& p, int need_sum, int* nparts_out, cudaStream_t st) {
+int launch_umma(const Params& p, int need_sum, bool allow_pair, int* nparts_out, cudaStream_t st) {
     using namespace umma;
-    const int m_tiles = (p.M + BM - 1) / BM;
+    // more than 128 block rows: pairs of blocks share the weight tiles (256 rows per pair)
+    const bool pair = allow_pair && p.M > BM;
+    const int m_tiles = pair ? 2 * ((p.M + 2 * BM - 1) / (2 * BM)) : (p.M + BM - 1) / BM;
     int nparts = 148 / m_tiles;
     if (nparts < 1) nparts = 1;
     const int gran = (p.V + 15) / 16;                    // 16-row granules of the vocabulary
@@ -294,8 +459,9 @@ int launch_umma(const Params& p, int need_sum, int* nparts_out, cudaStream_t st)
     a.h_box_rows = (p.M >= BM) ? BM : ((p.M + 7) / 8) * 8;
     a.gmax = (n_units + nparts - 1) / nparts;
     a.a_bytes = a.h_box_rows * 128;
+    const int w_rows = pair ? 8 : 16;                    // weight rows per granule that one block stages
     // a stage is never shorter than the span an MMA reads for its 128-row operand
-    a.stage_bytes = a.a_bytes + a.gmax * 16 * 128;
+    a.stage_bytes = a.a_bytes + a.gmax * w_rows * 128;
     if (a.stage_bytes < A_SPAN) a.stage_bytes = A_SPAN;
     // as deep a ring as shared memory holds: the bytes in flight per SM are what hide the HBM latency
     a.stages = SMEM_BUDGET / a.stage_bytes;
@@ -312,14 +478,19 @@ int launch_umma(const Params& p, int need_sum, int* nparts_out, cudaStream_t st)
     CUtensorMap tm_h, tm_w_hi, tm_w_lo;
     int rc = make_map(&tm_h, p.h, (uint64_t)p.M, (uint64_t)p.hid, (uint32_t)a.h_box_rows);
     if (rc != DEER_OK) return rc;
-    rc = make_map(&tm_w_hi, p.w, (uint64_t)p.V, (uint64_t)p.hid, (uint32_t)a.gmax * 16);
+    rc = make_map(&tm_w_hi, p.w, (uint64_t)p.V, (uint64_t)p.hid, (uint32_t)(a.gmax * w_rows));
     if (rc != DEER_OK) return rc;
-    rc = make_map(&tm_w_lo, p.w, (uint64_t)p.V, (uint64_t)p.hid, (uint32_t)(a.gmax > 1 ? a.gmax - 1 : 1) * 16);
+    rc = make_map(&tm_w_lo, p.w, (uint64_t)p.V, (uint64_t)p.hid, (uint32_t)((a.gmax > 1 ? a.gmax - 1 : 1) * w_rows));
     if (rc != DEER_OK) return rc;
     const int smem_bytes = a.stages * a.stage_bytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
-    DEER_CUDA(cudaFuncSetAttribute(lmhead_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
     dim3 grid(m_tiles, nparts);
-    lmhead_umma_kernel<<<grid, umma::THREADS, smem_bytes, st>>>(tm_h, tm_w_hi, tm_w_lo, a);
+    if (pair) {
+        DEER_CUDA(cudaFuncSetAttribute(lmhead_umma_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
+        lmhead_umma_pair_kernel<<<grid, umma::THREADS, smem_bytes, st>>>(tm_h, tm_w_hi, tm_w_lo, a);
+    } else {
+        DEER_CUDA(cudaFuncSetAttribute(lmhead_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
+        lmhead_umma_kernel<<<grid, umma::THREADS, smem_bytes, st>>>(tm_h, tm_w_hi, tm_w_lo, a);
+    }
     DEER_CUDA(cudaGetLastError());
     *nparts_out = nparts;
     return DEER_OK;

@@ -35,6 +35,8 @@ def _select(h, w, mode, T=1.0, drafts=None, logits=False):
     (100, 192, 3000),      # 128-row tile with a ragged tail
     (256, 128, 2048),      # two 128-row tiles
     (300, 64, 777),
+    (384, 128, 4000),      # three 128-row tiles: the second block pair's peer has no rows at all
+    (520, 256, 9000),      # three block pairs, the last with 8 rows
 ])
 def test_all_outputs_small(M, hid, V):
     from paper_2512_15176_b200 import binding as L
