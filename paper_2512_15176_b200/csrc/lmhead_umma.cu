@@ -33,6 +33,7 @@ constexpr int MAXN = 256;
 constexpr int MAX_STAGES = 8;
 constexpr int A_SPAN = BM * BK * 2;         // bytes one MMA reads for its 128-row operand (16 KB)
 constexpr int SMEM_BUDGET = 220 * 1024;     // operand ring; barriers and alignment slack come on top
+constexpr int SMEM_LIMIT = 227 * 1024;      // dynamic shared memory one block may have
 constexpr int THREADS = 192;
 
 struct Args {
@@ -46,6 +47,7 @@ struct Args {
     int n_units;             // vocabulary units of 16*T rows
     int nparts;
     int need_sum;            // 0: argmax only
+    int z_tma;               // 1: the logits leave through TMA stores from a staging area behind the operand ring
     float c2;                // log2(e) / T
     const int32_t* draft_ids;
     float* out_draft_logit;
@@ -55,13 +57,13 @@ struct Args {
 
 // One 16-column slice of an accumulator row: optional store, draft-token pick, running selection.
 __device__ __forceinline__ void consume16(const uint32_t (&r)[16], int vbase, int V, bool row_ok, const Args& a, size_t zrow,
-                                          int draft, int grow, float& run_m, int32_t& run_i, float& run_s) {
+                                          int draft, int grow, bool store, float& run_m, int32_t& run_i, float& run_s) {
     if (!row_ok || vbase >= V) return;
     const int nv = min(16, V - vbase);
     float v[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) v[j] = (j < nv) ? __uint_as_float(r[j]) : -INFINITY;
-    if (a.out_logits) {
+    if (store) {
         float* dst = a.out_logits + zrow + vbase;
         if (nv == 16 && ((zrow + vbase) & 3) == 0) {
 #pragma unroll
@@ -101,14 +103,94 @@ __device__ __forceinline__ void consume16(const uint32_t (&r)[16], int vbase, in
     }
 }
 
+constexpr int STAGING_BYTES = 4 * 2 * 4096;   // per epilogue warp two 32-row x 32-column fp32 boxes
+
+// The epilogue of both kernels: warp `quarter` owns TMEM lanes 32*quarter.. (block rows m0 + 32*quarter..).
+// Every accumulator row is reduced to (max, lowest argmax, sum exp); the logits, when asked for, go to a
+// staging box in the TMA 128-byte swizzle (16-byte chunk index XOR row mod 8: the 32 rows of a warp then hit
+// distinct banks) and leave as one 32 x 32 TMA store per column group -- full 128-byte lines per row where
+// per-thread stores would write 16 bytes of each of 32 rows.  A column group of 16 (odd g) and a vocabulary
+// whose row pitch is not a multiple of 16 bytes use plain stores.
+template <bool PAIR>
+__device__ __forceinline__ void epilogue(const Args& a, const CUtensorMap* tm_z, int quarter, int lane, int m0, int part,
+                                         int row_base, int N, int n_tiles, uint32_t tmem_base, uint32_t tfull0,
+                                         uint32_t tempty0, uint32_t staging, volatile int* abort_flag) {
+    const int row = quarter * 32 + lane;
+    const int grow = m0 + row;
+    const bool row_ok = grow < a.M;
+    const size_t zrow = (size_t)(row_ok ? grow : 0) * a.V;
+    const int draft = (row_ok && a.draft_ids && a.out_draft_logit) ? a.draft_ids[grow] : -1;
+    const bool z_any = a.out_logits != nullptr;
+    const bool z_box = a.z_tma && (m0 + quarter * 32 < a.M);      // warp-uniform
+    const uint32_t stg = staging + (uint32_t)quarter * 8192u;
+    const uint32_t stg_row = (uint32_t)lane * 128u, sw = (uint32_t)(lane & 7);
+    int stg_i = 0;
+    float run_m = -INFINITY, run_s = 0.f;
+    int32_t run_i = 0x7fffffff;
+    for (int t = 0; t < n_tiles; ++t) {
+        const int buf = t & 1;
+        const uint32_t aph = (uint32_t)(t >> 1) & 1u;
+        const bool got = mbar_wait(tfull0 + 8u * buf, aph, abort_flag);
+        if (!__all_sync(0xffffffffu, got)) break;          // warp-uniform, so the aligned TMEM loads stay converged
+        tcgen05_fence_after();
+        const int row0 = row_base + t * N;
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * MAXN);
+        for (int c = 0; c < N; c += 32) {
+            uint32_t r0[16], r1[16];
+            TMEM_LD_X16(taddr + c, r0);
+            const bool second = (c + 16 < N);
+            if (second) TMEM_LD_X16(taddr + c + 16, r1);
+            tmem_wait_ld();
+            const bool box = z_box && second && (row0 + c < a.V);
+            const bool direct = z_any && !box;
+            consume16(r0, row0 + c, a.V, row_ok, a, zrow, draft, grow, direct, run_m, run_i, run_s);
+            if (second) consume16(r1, row0 + c + 16, a.V, row_ok, a, zrow, draft, grow, direct, run_m, run_i, run_s);
+            if (box) {
+                // the store issued from this buffer two groups ago has read it
+                if (lane == 0) bulk_wait_read<1>();
+                __syncwarp();
+                const uint32_t b = stg + (uint32_t)stg_i * 4096u + stg_row;
+                stg_i ^= 1;
+#pragma unroll
+                for (uint32_t j = 0; j < 4; ++j) {
+                    st_shared_v4(b + ((j ^ sw) << 4), r0[4 * j], r0[4 * j + 1], r0[4 * j + 2], r0[4 * j + 3]);
+                    st_shared_v4(b + (((j + 4) ^ sw) << 4), r1[4 * j], r1[4 * j + 1], r1[4 * j + 2], r1[4 * j + 3]);
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_2d(tm_z, b - stg_row, row0 + c, m0 + quarter * 32);   // rows >= M, columns >= V are clipped
+                    bulk_commit();
+                }
+            }
+        }
+        tcgen05_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+            if (PAIR) mbar_arrive_cluster(map_to_cta(tempty0 + 8u * buf, 0));
+            else mbar_arrive(tempty0 + 8u * buf);
+        }
+    }
+    if (lane == 0) bulk_wait<0>();               // the staging area outlives every store that reads it
+    if (row_ok) {
+        Partial pr;
+        pr.m = run_m;
+        pr.idx = run_i;
+        pr.s = a.need_sum ? run_s : 1.f;
+        pr.pad = 0;
+        if (*abort_flag) pr.idx = PARTIAL_ABORTED;     // the finalisation turns this into ids of -2
+        a.part[(size_t)part * a.M + grow] = pr;
+    }
+}
+
 __global__ void __launch_bounds__(THREADS, 1)
 lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ CUtensorMap tm_w_hi,
-                   const __grid_constant__ CUtensorMap tm_w_lo, const Args a) {
+                   const __grid_constant__ CUtensorMap tm_w_lo, const __grid_constant__ CUtensorMap tm_z, const Args a) {
     extern __shared__ unsigned char smem_raw[];
     // operand stages need 1024-byte alignment for the 128-byte swizzle
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int stage_bytes = a.stage_bytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + a.stages * stage_bytes);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + a.stages * stage_bytes + (a.z_tma ? STAGING_BYTES : 0));
     // bars[0..S) full, [S..2S) empty, [2S..2S+2) accumulator full, [2S+2..2S+4) accumulator empty   (S = MAX_STAGES)
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * MAX_STAGES + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -204,44 +286,8 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
         }
     } else {
         // ---------------- epilogue: 4 warps, one TMEM lane quarter each ----------------
-        const int quarter = warp & 3;
-        const int row = quarter * 32 + lane;
-        const int grow = m0 + row;
-        const bool row_ok = grow < a.M;
-        const size_t zrow = (size_t)(row_ok ? grow : 0) * a.V;
-        const int draft = (row_ok && a.draft_ids && a.out_draft_logit) ? a.draft_ids[grow] : -1;
-        float run_m = -INFINITY, run_s = 0.f;
-        int32_t run_i = 0x7fffffff;
-        for (int t = 0; t < n_tiles; ++t) {
-            const int buf = t & 1;
-            const uint32_t aph = (uint32_t)(t >> 1) & 1u;
-            const bool got = mbar_wait(tfull_bar(buf), aph, abort_flag);
-            if (!__all_sync(0xffffffffu, got)) break;          // warp-uniform, so the aligned TMEM loads stay converged
-            tcgen05_fence_after();
-            const int row0 = row_base + t * N;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * MAXN);
-            for (int c = 0; c < N; c += 32) {
-                uint32_t r0[16], r1[16];
-                TMEM_LD_X16(taddr + c, r0);
-                const bool second = (c + 16 < N);
-                if (second) TMEM_LD_X16(taddr + c + 16, r1);
-                tmem_wait_ld();
-                consume16(r0, row0 + c, a.V, row_ok, a, zrow, draft, grow, run_m, run_i, run_s);
-                if (second) consume16(r1, row0 + c + 16, a.V, row_ok, a, zrow, draft, grow, run_m, run_i, run_s);
-            }
-            tcgen05_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(buf));
-        }
-        if (row_ok) {
-            Partial pr;
-            pr.m = run_m;
-            pr.idx = run_i;
-            pr.s = a.need_sum ? run_s : 1.f;
-            pr.pad = 0;
-            if (*abort_flag) pr.idx = PARTIAL_ABORTED;     // the finalisation turns this into ids of -2
-            a.part[(size_t)part * a.M + grow] = pr;
-        }
+        epilogue<false>(a, &tm_z, warp & 3, lane, m0, part, row_base, N, n_tiles, tmem_base, tfull_bar(0), tempty_bar(0),
+                        smem_base + (uint32_t)(a.stages * stage_bytes), abort_flag);
     }
 
     // ---- tear-down ------------------------------------------------------------
@@ -269,11 +315,11 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
 // one multicast commit; both blocks' epilogue warps arrive on the leader's `accumulator empty`.
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ CUtensorMap tm_w_hi,
-                        const __grid_constant__ CUtensorMap tm_w_lo, const Args a) {
+                        const __grid_constant__ CUtensorMap tm_w_lo, const __grid_constant__ CUtensorMap tm_z, const Args a) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int stage_bytes = a.stage_bytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + a.stages * stage_bytes);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + a.stages * stage_bytes + (a.z_tma ? STAGING_BYTES : 0));
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * MAX_STAGES + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -367,44 +413,8 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
         }
     } else {
         // ---------------- epilogue: 4 warps in each block, one TMEM lane quarter each ----------------
-        const int quarter = warp & 3;
-        const int row = quarter * 32 + lane;
-        const int grow = m0 + row;
-        const bool row_ok = grow < a.M;
-        const size_t zrow = (size_t)(row_ok ? grow : 0) * a.V;
-        const int draft = (row_ok && a.draft_ids && a.out_draft_logit) ? a.draft_ids[grow] : -1;
-        float run_m = -INFINITY, run_s = 0.f;
-        int32_t run_i = 0x7fffffff;
-        for (int t = 0; t < n_tiles; ++t) {
-            const int buf = t & 1;
-            const uint32_t aph = (uint32_t)(t >> 1) & 1u;
-            const bool got = mbar_wait(tfull_bar(buf), aph, abort_flag);
-            if (!__all_sync(0xffffffffu, got)) break;
-            tcgen05_fence_after();
-            const int row0 = row_base + t * N;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * MAXN);
-            for (int c = 0; c < N; c += 32) {
-                uint32_t r0[16], r1[16];
-                TMEM_LD_X16(taddr + c, r0);
-                const bool second = (c + 16 < N);
-                if (second) TMEM_LD_X16(taddr + c + 16, r1);
-                tmem_wait_ld();
-                consume16(r0, row0 + c, a.V, row_ok, a, zrow, draft, grow, run_m, run_i, run_s);
-                if (second) consume16(r1, row0 + c + 16, a.V, row_ok, a, zrow, draft, grow, run_m, run_i, run_s);
-            }
-            tcgen05_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(buf), 0));
-        }
-        if (row_ok) {
-            Partial pr;
-            pr.m = run_m;
-            pr.idx = run_i;
-            pr.s = a.need_sum ? run_s : 1.f;
-            pr.pad = 0;
-            if (*abort_flag) pr.idx = PARTIAL_ABORTED;
-            a.part[(size_t)part * a.M + grow] = pr;
-        }
+        epilogue<true>(a, &tm_z, warp & 3, lane, m0, part, row_base, N, n_tiles, tmem_base, tfull_bar(0), tempty_bar(0),
+                       smem_base + (uint32_t)(a.stages * stage_bytes), abort_flag);
     }
 
     // ---- tear-down: neither block leaves while the other may still signal it or read its shared memory ----
@@ -424,7 +434,7 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
 
 // ---- host side ------------------------------------------------------------------
 // 2-D bf16 tensor [rows][cols] (cols contiguous), box = box_rows x 64 columns.
-static int make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+static int make_operand_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
     const uint64_t dims[2] = {cols, rows};
     const uint64_t strides[1] = {cols * 2};
     const uint32_t box[2] = {BK, box_rows};
@@ -463,8 +473,10 @@ int launch_umma(const Params& p, int need_sum, bool allow_pair, int* nparts_out,
     // a stage is never shorter than the span an MMA reads for its 128-row operand
     a.stage_bytes = a.a_bytes + a.gmax * w_rows * 128;
     if (a.stage_bytes < A_SPAN) a.stage_bytes = A_SPAN;
+    // logits through TMA stores need a row pitch that is a multiple of 16 bytes
+    a.z_tma = (p.out_logits != nullptr && p.V % 4 == 0) ? 1 : 0;
     // as deep a ring as shared memory holds: the bytes in flight per SM are what hide the HBM latency
-    a.stages = SMEM_BUDGET / a.stage_bytes;
+    a.stages = (a.z_tma ? SMEM_LIMIT - 1280 - STAGING_BYTES : SMEM_BUDGET) / a.stage_bytes;
     if (a.stages > MAX_STAGES) a.stages = MAX_STAGES;
     a.T = T;
     a.n_units = n_units;
@@ -476,20 +488,28 @@ int launch_umma(const Params& p, int need_sum, bool allow_pair, int* nparts_out,
     a.out_logits = p.out_logits;
     a.part = p.part;
     CUtensorMap tm_h, tm_w_hi, tm_w_lo;
-    int rc = make_map(&tm_h, p.h, (uint64_t)p.M, (uint64_t)p.hid, (uint32_t)a.h_box_rows);
+    int rc = make_operand_map(&tm_h, p.h, (uint64_t)p.M, (uint64_t)p.hid, (uint32_t)a.h_box_rows);
     if (rc != DEER_OK) return rc;
-    rc = make_map(&tm_w_hi, p.w, (uint64_t)p.V, (uint64_t)p.hid, (uint32_t)(a.gmax * w_rows));
+    rc = make_operand_map(&tm_w_hi, p.w, (uint64_t)p.V, (uint64_t)p.hid, (uint32_t)(a.gmax * w_rows));
     if (rc != DEER_OK) return rc;
-    rc = make_map(&tm_w_lo, p.w, (uint64_t)p.V, (uint64_t)p.hid, (uint32_t)((a.gmax > 1 ? a.gmax - 1 : 1) * w_rows));
+    rc = make_operand_map(&tm_w_lo, p.w, (uint64_t)p.V, (uint64_t)p.hid, (uint32_t)((a.gmax > 1 ? a.gmax - 1 : 1) * w_rows));
     if (rc != DEER_OK) return rc;
-    const int smem_bytes = a.stages * a.stage_bytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    CUtensorMap tm_z = tm_h;                             // a valid map even when it is not used
+    if (a.z_tma) {
+        const uint64_t dims[2] = {(uint64_t)p.V, (uint64_t)p.M};
+        const uint64_t strides[1] = {(uint64_t)p.V * 4};
+        const uint32_t box[2] = {32, 32};
+        rc = make_map_f32(&tm_z, p.out_logits, 2, dims, strides, box);
+        if (rc != DEER_OK) return rc;
+    }
+    const int smem_bytes = a.stages * a.stage_bytes + (a.z_tma ? STAGING_BYTES : 0) + 1024 /*alignment slack*/ + 256 /*barriers*/;
     dim3 grid(m_tiles, nparts);
     if (pair) {
         DEER_CUDA(cudaFuncSetAttribute(lmhead_umma_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
-        lmhead_umma_pair_kernel<<<grid, umma::THREADS, smem_bytes, st>>>(tm_h, tm_w_hi, tm_w_lo, a);
+        lmhead_umma_pair_kernel<<<grid, umma::THREADS, smem_bytes, st>>>(tm_h, tm_w_hi, tm_w_lo, tm_z, a);
     } else {
         DEER_CUDA(cudaFuncSetAttribute(lmhead_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
-        lmhead_umma_kernel<<<grid, umma::THREADS, smem_bytes, st>>>(tm_h, tm_w_hi, tm_w_lo, a);
+        lmhead_umma_kernel<<<grid, umma::THREADS, smem_bytes, st>>>(tm_h, tm_w_hi, tm_w_lo, tm_z, a);
     }
     DEER_CUDA(cudaGetLastError());
     *nparts_out = nparts;

@@ -76,6 +76,25 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* tm,
         ::"r"(dst), "l"(tm), "r"(bar), "r"(x), "r"(y), "r"(z), "r"(w), "r"(v)
         : "memory");
 }
+// ---- TMA tile stores (shared -> global), tracked by the issuing thread's bulk groups ----
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(tm), "r"(src), "r"(x), "r"(y)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Returns once at most N of this thread's latest bulk groups still have to read their shared-memory source.
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+// Returns once at most N of this thread's latest bulk groups are incomplete.
+template <int N>
+__device__ __forceinline__ void bulk_wait() {
+    asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* tm) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
 }
@@ -243,10 +262,10 @@ inline EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// bf16 tensor of `rank` dimensions (dims[0] contiguous), 128-byte swizzle, out-of-range elements read as zero.
-// strides_bytes[i] is the byte stride of dimension i + 1; box[0] * 2 must be 128.
-inline int make_map_bf16(CUtensorMap* tm, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-                         const uint32_t* box) {
+// Tensor of `rank` dimensions (dims[0] contiguous), 128-byte swizzle, out-of-range elements read as zero (and
+// are not written by a store).  strides_bytes[i] is the byte stride of dimension i + 1; box[0] must span 128 bytes.
+inline int make_map(CUtensorMap* tm, CUtensorMapDataType dtype, const void* base, int rank, const uint64_t* dims,
+                    const uint64_t* strides_bytes, const uint32_t* box) {
     EncodeTiledFn fn = encode_fn();
     DEER_CHECK_ARG(fn, DEER_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
     cuuint64_t d[5], s[4];
@@ -257,11 +276,19 @@ inline int make_map_bf16(CUtensorMap* tm, const void* base, int rank, const uint
         e[i] = 1;
         if (i + 1 < rank) s[i] = strides_bytes[i];
     }
-    const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), d, s, b, e,
+    const CUresult r = fn(tm, dtype, (cuuint32_t)rank, const_cast<void*>(base), d, s, b, e,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     DEER_CHECK_ARG(r == CUDA_SUCCESS, DEER_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
     return DEER_OK;
+}
+inline int make_map_bf16(CUtensorMap* tm, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                         const uint32_t* box) {
+    return make_map(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, base, rank, dims, strides_bytes, box);
+}
+inline int make_map_f32(CUtensorMap* tm, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                        const uint32_t* box) {
+    return make_map(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, base, rank, dims, strides_bytes, box);
 }
 
 }  // namespace sm100
