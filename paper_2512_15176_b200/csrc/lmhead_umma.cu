@@ -6,13 +6,15 @@
 //
 // Tile shape: the block rows of h sit on the 128 TMEM lanes (lanes beyond the
 // rows that exist are never read back), the vocabulary on up to 256 accumulator
-// columns.  Each thread block owns a contiguous vocabulary range cut into T
-// equal tiles of N = 16*g rows (g <= 16), so that the ranges of all blocks
-// differ by at most one 16*T-row unit and no weight row is fetched twice; one
-// TMA box brings a whole N x 64 weight tile.  The operand ring is as deep as
-// shared memory allows (7 stages of 30 KB at 32 block rows), because the bytes
-// in flight per SM are what cover the HBM latency.  Two accumulators
-// (2 x 256 columns) let the epilogue of tile t overlap the MMAs of tile t+1.
+// columns.  The vocabulary is counted in granules of 16 rows; each thread block
+// owns a contiguous range of them (the ranges differ by at most one granule) and
+// cuts it into T tiles of g or g - 1 granules (N = 16*g <= 256), so no weight row
+// is fetched twice and one TMA box brings a whole N x 64 weight tile.  The operand
+// ring is as deep as shared memory allows (7 stages of 30 KB at 32 block rows),
+// because the bytes in flight per SM are what cover the HBM latency.  Two
+// accumulators (2 x 256 columns) let the epilogue of tile t overlap the MMAs of
+// tile t+1.  With more than 128 block rows, pairs of blocks share the weight
+// tiles through cta_group::2 MMAs (second kernel below).
 //
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (+ TMEM owner),
 // warps 2..5 = epilogue (one TMEM lane quarter each).  All waits are bounded:
@@ -43,8 +45,8 @@ struct Args {
     int stage_bytes;         // bytes of one stage: h tile + w tile, never less than the 16 KB an MMA reads for h
     int stages;              // pipeline depth
     int gmax;                // granules of the larger tile size (box of tm_w_hi); tm_w_lo has gmax - 1
-    int T;                   // tiles per block
-    int n_units;             // vocabulary units of 16*T rows
+    int T;                   // tiles per block (fewer only where a block has fewer granules than that)
+    int gran;                // 16-row granules of the vocabulary
     int nparts;
     int need_sum;            // 0: argmax only
     int z_tma;               // 1: the logits leave through TMA stores from a staging area behind the operand ring
@@ -103,6 +105,27 @@ __device__ __forceinline__ void consume16(const uint32_t (&r)[16], int vbase, in
     }
 }
 
+// Block `part` owns the granules [part * gran / nparts, (part + 1) * gran / nparts): the counts differ by at most
+// one between blocks.  Its range is cut into T tiles of `base` or `base + 1` granules (the first `extra` tiles are
+// the larger ones); over all blocks only the two sizes gmax - 1 and gmax occur.
+struct Tiles {
+    int g0, base, extra, n;
+};
+__device__ __forceinline__ Tiles block_tiles(const Args& a, int part) {
+    const int lo = (int)((long)part * a.gran / a.nparts), hi = (int)((long)(part + 1) * a.gran / a.nparts);
+    Tiles tl;
+    tl.g0 = lo;
+    tl.base = (hi - lo) / a.T;
+    tl.extra = (hi - lo) % a.T;
+    tl.n = tl.base > 0 ? a.T : tl.extra;
+    return tl;
+}
+// First vocabulary row and granule count of tile t.
+__device__ __forceinline__ void tile_span(const Tiles& tl, int t, int& row0, int& g) {
+    g = tl.base + (t < tl.extra ? 1 : 0);
+    row0 = (tl.g0 + t * tl.base + min(t, tl.extra)) * 16;
+}
+
 constexpr int STAGING_BYTES = 4 * 2 * 4096;   // per epilogue warp two 32-row x 32-column fp32 boxes
 
 // The epilogue of both kernels: warp `quarter` owns TMEM lanes 32*quarter.. (block rows m0 + 32*quarter..).
@@ -113,7 +136,7 @@ constexpr int STAGING_BYTES = 4 * 2 * 4096;   // per epilogue warp two 32-row x 
 // whose row pitch is not a multiple of 16 bytes use plain stores.
 template <bool PAIR>
 __device__ __forceinline__ void epilogue(const Args& a, const CUtensorMap* tm_z, int quarter, int lane, int m0, int part,
-                                         int row_base, int N, int n_tiles, uint32_t tmem_base, uint32_t tfull0,
+                                         const Tiles& tl, uint32_t tmem_base, uint32_t tfull0,
                                          uint32_t tempty0, uint32_t staging, volatile int* abort_flag) {
     const int row = quarter * 32 + lane;
     const int grow = m0 + row;
@@ -127,13 +150,15 @@ __device__ __forceinline__ void epilogue(const Args& a, const CUtensorMap* tm_z,
     int stg_i = 0;
     float run_m = -INFINITY, run_s = 0.f;
     int32_t run_i = 0x7fffffff;
-    for (int t = 0; t < n_tiles; ++t) {
+    for (int t = 0; t < tl.n; ++t) {
         const int buf = t & 1;
         const uint32_t aph = (uint32_t)(t >> 1) & 1u;
         const bool got = mbar_wait(tfull0 + 8u * buf, aph, abort_flag);
         if (!__all_sync(0xffffffffu, got)) break;          // warp-uniform, so the aligned TMEM loads stay converged
         tcgen05_fence_after();
-        const int row0 = row_base + t * N;
+        int row0, g;
+        tile_span(tl, t, row0, g);
+        const int N = g * 16;
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * MAXN);
         for (int c = 0; c < N; c += 32) {
             uint32_t r0[16], r1[16];
@@ -198,12 +223,8 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int m0 = blockIdx.x * BM;
     const int part = blockIdx.y;
-    const int u0 = (int)((long)part * a.n_units / a.nparts);
-    const int u1 = (int)((long)(part + 1) * a.n_units / a.nparts);
-    const int g = u1 - u0;                       // 16-row granules per tile: gmax or gmax - 1
-    const int N = g * 16;
-    const int row_base = u0 * a.T * 16;
-    const int n_tiles = (g > 0) ? a.T : 0;
+    const Tiles tl = block_tiles(a, part);
+    const int n_tiles = tl.n;
     const int KB = a.hid / BK;
 
     const uint32_t smem_base = smem_u32(smem);
@@ -240,12 +261,13 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0 && n_tiles > 0) {
-            const CUtensorMap* tm_w = (g == a.gmax) ? &tm_w_hi : &tm_w_lo;
-            const uint32_t stage_tx = (uint32_t)(a.h_box_rows * 128 + N * 128);
             int it = 0;
             bool ok = true;
             for (int t = 0; t < n_tiles && ok; ++t) {
-                const int row0 = row_base + t * N;
+                int row0, g;
+                tile_span(tl, t, row0, g);
+                const CUtensorMap* tm_w = (g == a.gmax) ? &tm_w_hi : &tm_w_lo;
+                const uint32_t stage_tx = (uint32_t)(a.h_box_rows * 128 + g * 16 * 128);
                 for (int kb = 0; kb < KB; ++kb, ++it) {
                     const int s = it % a.stages;
                     const uint32_t ph = (uint32_t)(it / a.stages) & 1u;
@@ -260,10 +282,12 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0 && n_tiles > 0) {
-            const uint32_t idesc = make_idesc_bf16(N, 0);
             int it = 0;
             bool ok = true;
             for (int t = 0; t < n_tiles && ok; ++t) {
+                int row0, g;
+                tile_span(tl, t, row0, g);
+                const uint32_t idesc = make_idesc_bf16(g * 16, 0);
                 const int buf = t & 1;
                 const uint32_t aph = (uint32_t)(t >> 1) & 1u;
                 if (!mbar_wait(tempty_bar(buf), aph ^ 1u, abort_flag)) break;
@@ -286,7 +310,7 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
         }
     } else {
         // ---------------- epilogue: 4 warps, one TMEM lane quarter each ----------------
-        epilogue<false>(a, &tm_z, warp & 3, lane, m0, part, row_base, N, n_tiles, tmem_base, tfull_bar(0), tempty_bar(0),
+        epilogue<false>(a, &tm_z, warp & 3, lane, m0, part, tl, tmem_base, tfull_bar(0), tempty_bar(0),
                         smem_base + (uint32_t)(a.stages * stage_bytes), abort_flag);
     }
 
@@ -328,13 +352,8 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
     const bool leader = (rank == 0);
     const int m0 = (int)(blockIdx.x >> 1) * (2 * BM) + (int)rank * BM;
     const int part = blockIdx.y;
-    const int u0 = (int)((long)part * a.n_units / a.nparts);
-    const int u1 = (int)((long)(part + 1) * a.n_units / a.nparts);
-    const int g = u1 - u0;
-    const int N = g * 16;
-    const int half = g * 8;                      // rows of the weight tile this block stages
-    const int row_base = u0 * a.T * 16;
-    const int n_tiles = (g > 0) ? a.T : 0;
+    const Tiles tl = block_tiles(a, part);
+    const int n_tiles = tl.n;
     const int KB = a.hid / BK;
 
     const uint32_t smem_base = smem_u32(smem);
@@ -366,12 +385,15 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
     if (warp == 0) {
         // ---------------- TMA producer (each block: its 128 rows of h, its half of the weight tile) ----------------
         if (lane == 0 && n_tiles > 0) {
-            const CUtensorMap* tm_w = (g == a.gmax) ? &tm_w_hi : &tm_w_lo;
-            const uint32_t stage_tx = 2u * (uint32_t)(A_SPAN + half * 128);
             int it = 0;
             bool ok = true;
             for (int t = 0; t < n_tiles && ok; ++t) {
-                const int row0 = row_base + t * N + (int)rank * half;
+                int row0, g;
+                tile_span(tl, t, row0, g);
+                const int half = g * 8;                  // rows of the weight tile this block stages
+                row0 += (int)rank * half;
+                const CUtensorMap* tm_w = (g == a.gmax) ? &tm_w_hi : &tm_w_lo;
+                const uint32_t stage_tx = 2u * (uint32_t)(A_SPAN + half * 128);
                 for (int kb = 0; kb < KB; ++kb, ++it) {
                     const int s = it % a.stages;
                     const uint32_t ph = (uint32_t)(it / a.stages) & 1u;
@@ -387,10 +409,12 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
     } else if (warp == 1) {
         // ---------------- MMA issuer (leader block only) ----------------
         if (leader && lane == 0 && n_tiles > 0) {
-            const uint32_t idesc = make_idesc_bf16_pair(N);
             int it = 0;
             bool ok = true;
             for (int t = 0; t < n_tiles && ok; ++t) {
+                int row0, g;
+                tile_span(tl, t, row0, g);
+                const uint32_t idesc = make_idesc_bf16_pair(g * 16);
                 const int buf = t & 1;
                 const uint32_t aph = (uint32_t)(t >> 1) & 1u;
                 if (!mbar_wait(tempty_bar(buf), aph ^ 1u, abort_flag)) break;
@@ -413,7 +437,7 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
         }
     } else {
         // ---------------- epilogue: 4 warps in each block, one TMEM lane quarter each ----------------
-        epilogue<true>(a, &tm_z, warp & 3, lane, m0, part, row_base, N, n_tiles, tmem_base, tfull_bar(0), tempty_bar(0),
+        epilogue<true>(a, &tm_z, warp & 3, lane, m0, part, tl, tmem_base, tfull_bar(0), tempty_bar(0),
                        smem_base + (uint32_t)(a.stages * stage_bytes), abort_flag);
     }
 
@@ -456,18 +480,14 @@ int launch_umma(const Params& p, int need_sum, bool allow_pair, int* nparts_out,
     if (nparts < 1) nparts = 1;
     const int gran = (p.V + 15) / 16;                    // 16-row granules of the vocabulary
     if (nparts > gran) nparts = gran;
-    int T = (gran + nparts * 16 - 1) / (nparts * 16);    // tiles per block so that a tile has <= 16 granules
-    int n_units;
-    for (;; ++T) {
-        n_units = (gran + T - 1) / T;
-        if ((n_units + nparts - 1) / nparts <= 16) break;
-    }
+    const int cmax = (gran + nparts - 1) / nparts;       // granules of the largest block
+    const int T = (cmax + 15) / 16;                      // tiles per block so that a tile has <= 16 granules
     Args a;
     a.M = p.M;
     a.hid = p.hid;
     a.V = p.V;
     a.h_box_rows = (p.M >= BM) ? BM : ((p.M + 7) / 8) * 8;
-    a.gmax = (n_units + nparts - 1) / nparts;
+    a.gmax = (cmax + T - 1) / T;
     a.a_bytes = a.h_box_rows * 128;
     const int w_rows = pair ? 8 : 16;                    // weight rows per granule that one block stages
     // a stage is never shorter than the span an MMA reads for its 128-row operand
@@ -479,7 +499,7 @@ int launch_umma(const Params& p, int need_sum, bool allow_pair, int* nparts_out,
     a.stages = (a.z_tma ? SMEM_LIMIT - 1280 - STAGING_BYTES : SMEM_BUDGET) / a.stage_bytes;
     if (a.stages > MAX_STAGES) a.stages = MAX_STAGES;
     a.T = T;
-    a.n_units = n_units;
+    a.gran = gran;
     a.nparts = nparts;
     a.need_sum = need_sum;
     a.c2 = p.inv_t_log2;
