@@ -178,7 +178,8 @@ __device__ void cut_at_eos(const ResidualArgs& a, int b) {
         }
 }
 
-// Pass 1: the fp64 normalisers, one (slice, sequence) per block.
+// Pass 1: the fp64 normalisers, one (slice, sequence) per block.  Four tokens per thread and step where the
+// rows are 16-byte aligned, so that eight exponentials are in flight per thread.
 __global__ void __launch_bounds__(RES_THREADS) residual_norm_kernel(ResidualArgs a) {
     __shared__ double sh[32];
     const int b = blockIdx.y, sl = blockIdx.x;
@@ -192,7 +193,26 @@ __global__ void __launch_bounds__(RES_THREADS) residual_norm_kernel(ResidualArgs
     double sp = 0.0, sq = 0.0;
     double* ep = a.e_p + (size_t)b * a.V;
     double* eq = a.e_q + (size_t)b * a.V;
-    for (int v = v0 + threadIdx.x; v < v1; v += RES_THREADS) {
+    int v = v0 + threadIdx.x;
+    if ((a.V & 3) == 0) {
+        // v0 and V are multiples of 4, so v1 - v0 is as well
+        for (int q = v0 + 4 * threadIdx.x; q < v1; q += 4 * RES_THREADS) {
+            const float4 p4 = __ldg(reinterpret_cast<const float4*>(zp + q));
+            const float4 q4 = __ldg(reinterpret_cast<const float4*>(zq + q));
+            const double x0 = exp((double)p4.x * it - lp), x1 = exp((double)p4.y * it - lp);
+            const double x2 = exp((double)p4.z * it - lp), x3 = exp((double)p4.w * it - lp);
+            const double y0 = exp((double)q4.x - lq), y1 = exp((double)q4.y - lq);
+            const double y2 = exp((double)q4.z - lq), y3 = exp((double)q4.w - lq);
+            *reinterpret_cast<double2*>(ep + q) = make_double2(x0, x1);
+            *reinterpret_cast<double2*>(ep + q + 2) = make_double2(x2, x3);
+            *reinterpret_cast<double2*>(eq + q) = make_double2(y0, y1);
+            *reinterpret_cast<double2*>(eq + q + 2) = make_double2(y2, y3);
+            sp += (x0 + x1) + (x2 + x3);
+            sq += (y0 + y1) + (y2 + y3);
+        }
+        v = v1;
+    }
+    for (; v < v1; v += RES_THREADS) {
         const double x = exp((double)zp[v] * it - lp), y = exp((double)zq[v] - lq);
         ep[v] = x;
         eq[v] = y;
@@ -211,8 +231,10 @@ __global__ void __launch_bounds__(RES_THREADS) residual_norm_kernel(ResidualArgs
 // inverse CDF in vocabulary order, the smallest v whose cumulative residual reaches r * (total residual mass),
 // from p itself if that mass is 0.
 __global__ void __launch_bounds__(RES_THREADS) residual_pick_kernel(ResidualArgs a) {
+    constexpr int NW = RES_THREADS / 32;
     __shared__ double sh[32];
-    __shared__ double warp_pref[RES_THREADS / 32];
+    __shared__ double s_mass[NS], s_psum[NS];
+    __shared__ double warp_tot[NW];
     __shared__ int s_last, s_hit;
     const int b = blockIdx.y, sl = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -224,20 +246,30 @@ __global__ void __launch_bounds__(RES_THREADS) residual_pick_kernel(ResidualArgs
     const double* ep = a.e_p + (size_t)b * a.V;
     const double* eq = a.e_q + (size_t)b * a.V;
     double Sp = 0.0, Sq = 0.0;
+#pragma unroll
     for (int j = 0; j < NS; ++j) {
         Sp += a.sums[((size_t)b * NS + j) * 4 + 0];
         Sq += a.sums[((size_t)b * NS + j) * 4 + 1];
     }
     const double ip = 1.0 / Sp, iq = 1.0 / Sq;
-    auto prob_p = [&](int v) { return ep[v] * ip; };
-    auto resid = [&](int v) {
-        const double res = ep[v] * ip - eq[v] * iq;
+    auto resid2 = [&](double x, double y) {
+        const double res = x * ip - y * iq;
         return res > 0.0 ? res : 0.0;
     };
     {
         const int v0 = sl * a.slice, v1 = min(a.V, v0 + a.slice);
         double acc = 0.0;
-        for (int v = v0 + tid; v < v1; v += RES_THREADS) acc += resid(v);
+        int v = v0 + tid;
+        if ((a.V & 1) == 0) {
+            // slices start at multiples of 4 and V is even: pairs stay inside the slice and 16-byte aligned
+            for (int q = v0 + 2 * tid; q < v1; q += 2 * RES_THREADS) {
+                const double2 x = *reinterpret_cast<const double2*>(ep + q);
+                const double2 y = *reinterpret_cast<const double2*>(eq + q);
+                acc += resid2(x.x, y.x) + resid2(x.y, y.y);
+            }
+            v = v1;
+        }
+        for (; v < v1; v += RES_THREADS) acc += resid2(ep[v], eq[v]);
         acc = block_sum(acc, sh);
         if (tid == 0) {
             a.sums[((size_t)b * NS + sl) * 4 + 2] = acc;
@@ -250,61 +282,70 @@ __global__ void __launch_bounds__(RES_THREADS) residual_pick_kernel(ResidualArgs
     }
     // ---- the last block of the sequence: locate the slice, then the token inside it ----
     const volatile double* vs = a.sums;
+    if (tid < NS) {
+        s_mass[tid] = vs[((size_t)b * NS + tid) * 4 + 2];
+        s_psum[tid] = vs[((size_t)b * NS + tid) * 4 + 0];
+    }
+    __syncthreads();
     double S = 0.0;
-    for (int j = 0; j < NS; ++j) S += vs[((size_t)b * NS + j) * 4 + 2];
+#pragma unroll
+    for (int j = 0; j < NS; ++j) S += s_mass[j];
     const bool use_p = !(S > 0.0);
     const double target = (double)a.r[b] * (use_p ? 1.0 : S);
     double base = 0.0;
     int hs = 0;
     for (; hs < NS - 1; ++hs) {
-        const double m = use_p ? vs[((size_t)b * NS + hs) * 4 + 0] * ip : vs[((size_t)b * NS + hs) * 4 + 2];
+        const double m = use_p ? s_psum[hs] * ip : s_mass[hs];
         if (base + m >= target) break;
         base += m;
     }
-    auto weight = [&](int v) { return use_p ? prob_p(v) : resid(v); };
+    auto weight = [&](int v) { return use_p ? ep[v] * ip : resid2(ep[v], eq[v]); };
+    // Warp w owns a contiguous span of the slice, walked 32 consecutive tokens at a time (coalesced).
     const int v0 = hs * a.slice, v1 = min(a.V, v0 + a.slice);
-    const int per = (v1 - v0 + RES_THREADS - 1) / RES_THREADS;      // contiguous tokens per thread
-    const int c0 = min(v1, v0 + tid * per), c1 = min(v1, c0 + per);
+    const int span = ((v1 - v0 + NW - 1) / NW + 31) / 32 * 32;
+    const int w0 = min(v1, v0 + warp * span), w1 = min(v1, w0 + span);
     double mine = 0.0;
-    for (int v = c0; v < c1; ++v) mine += weight(v);
-    // exclusive prefix of the threads' sums in token order
-    double incl = mine;
+    for (int v = w0 + lane; v < w1; v += 32) mine += weight(v);
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const double t = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += t;
-    }
+    for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
     if (tid == 0) s_hit = -1;
-    if (lane == 31) warp_pref[warp] = incl;
+    if (lane == 0) warp_tot[warp] = mine;
     __syncthreads();
-    double wbase = base;
-    for (int w = 0; w < warp; ++w) wbase += warp_pref[w];
-    const double before = wbase + incl - mine, upto = wbase + incl;
-    if (before < target && upto >= target) {
-        // the one thread whose tokens straddle the target walks them
+    double before = base;
+    for (int w = 0; w < warp; ++w) before += warp_tot[w];
+    if (before < target && before + mine >= target) {
+        // the one warp whose span straddles the target: running inclusive scans of 32 tokens
         double cum = before;
         int hit = -1;
-        for (int v = c0; v < c1; ++v) {
-            cum += weight(v);
-            if (cum >= target) {
-                hit = v;
-                break;
+        for (int c = w0; c < w1 && hit < 0; c += 32) {
+            const int v = c + lane;
+            const double wv = v < w1 ? weight(v) : 0.0;
+            double incl = wv;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const double t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
+            }
+            const unsigned reach = __ballot_sync(0xffffffffu, v < w1 && cum + incl >= target);
+            if (reach) hit = c + __ffs(reach) - 1;
+            cum += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        if (hit < 0) {
+            // rounding left the walk just short of the warp's total: last token of the span with weight
+            for (int c = ((w1 - w0 - 1) / 32) * 32 + w0; c >= w0 && hit < 0; c -= 32) {
+                const int v = c + lane;
+                const unsigned pos = __ballot_sync(0xffffffffu, v < w1 && weight(v) > 0.0);
+                if (pos) hit = c + 31 - __clz(pos);
             }
         }
-        if (hit < 0)                                   // rounding left the walk just short: last token with weight
-            for (int v = c1 - 1; v >= c0; --v)
-                if (weight(v) > 0.0) {
-                    hit = v;
-                    break;
-                }
-        s_hit = hit;
+        if (lane == 0) s_hit = hit;
     }
     __syncthreads();
     if (tid == 0) {
         int hit = s_hit;
         if (hit < 0) {
-            // the target lies beyond the last cumulative sum by rounding: take the last token with positive weight
-            for (int v = a.V - 1; v >= 0; --v)
+            // the target lies beyond the slice's last cumulative sum by rounding: the last token with weight up to there
+            for (int v = v1 - 1; v >= 0; --v)
                 if (weight(v) > 0.0) {
                     hit = v;
                     break;

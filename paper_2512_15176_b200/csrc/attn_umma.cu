@@ -9,7 +9,12 @@
 // crosses unit boundaries, and each (unit, block) piece is a segment.  A unit
 // that lies inside one share is written straight to the output; otherwise each
 // segment emits a normalised partial output plus its log2-sum-exp, and a small
-// merge kernel combines the segments of the units that were split.
+// merge kernel combines the segments of the units that were split.  With more
+// than one row tile per KV head (G * k > 128) the list holds one entry per
+// (sequence, KV head) and the thread blocks come in groups of row_tiles: the
+// blocks of a group walk the same share, each for its own row tile, so they
+// stream the same KV tiles at the same time and the second read is an L2 hit
+// rather than a second pass over HBM a hundred megabytes later.
 //
 // Pipeline.  KV pages stream through a ring of 64-token slots filled by TMA,
 // one 4 KB box per page (slot layout below).  S = Q K^T and O += P V are
@@ -101,8 +106,8 @@ __device__ __forceinline__ long long share_begin(long long T, int j, int nc) { r
 
 // Warp-collective: lists up to MAX_SEGS segments of the flattened tile range [cursor, end) into segs[], in order.
 // Returns their number; *cursor_out is where the next round starts (== end when the share is exhausted).
-__device__ int build_segments(const AttnParams& p, int HR, long long cursor, long long end, Seg* segs, long long* cursor_out,
-                              int lane) {
+__device__ int build_segments(const AttnParams& p, int HL, int rt, long long cursor, long long end, Seg* segs,
+                              long long* cursor_out, int lane) {
     int n_seg = 0;
     long long base = 0;                                   // flattened position of sequence b0's first tile
     long long next_cursor = end;
@@ -112,7 +117,7 @@ __device__ int build_segments(const AttnParams& p, int HR, long long cursor, lon
         int n = 0, s = 0;
         const int tiles = (b < p.B) ? seq_tiles(p, b, &n, &s) : 0;
         if (b < p.B && tiles == 0) deer_report(p.kv.status, DEER_ERR_INVALID_ARG);
-        const long long span = (long long)tiles * HR;     // tiles this sequence contributes
+        const long long span = (long long)tiles * HL;     // tiles this sequence contributes to the list
         long long incl = span;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -141,7 +146,7 @@ __device__ int build_segments(const AttnParams& p, int HR, long long cursor, lon
             if (idx < MAX_SEGS) {
                 Seg sg;
                 sg.b = b;
-                sg.hr = hr;
+                sg.hr = hr * p.row_tiles + rt;
                 sg.t_a = cursor > u0 ? (int)(cursor - u0) : 0;
                 sg.t_b = end < u0 + tiles ? (int)(end - u0) : tiles;
                 sg.n = n;
@@ -187,6 +192,8 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const int Hkv = p.kv.n_kv_heads;
     const int HR = Hkv * p.row_tiles;                          // units per sequence
     const int j = blockIdx.x;
+    const int jg = j / p.row_tiles, rt_blk = j % p.row_tiles;  // group of blocks that walk the same share; my row tile
+    const int ncg = p.nc / p.row_tiles;                        // groups (nc is a multiple of row_tiles)
 
     // ---- this block's share of the flattened tile list ----
     long long T = 0;
@@ -199,8 +206,8 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) T += __shfl_xor_sync(0xffffffffu, T, o);
-    T *= HR;
-    const long long share_lo = share_begin(T, j, p.nc), share_hi = share_begin(T, j + 1, p.nc);
+    T *= Hkv;                                                  // list entries: (sequence, KV head) x tiles
+    const long long share_lo = share_begin(T, jg, ncg), share_hi = share_begin(T, jg + 1, ncg);
     if (j == 0 && tid == 0) *p.total_tiles = T;                // for the merge kernel
     if (share_hi <= share_lo) return;                          // nothing to do (fewer tiles than blocks)
 
@@ -249,7 +256,7 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         // ---- list the next segments of the share (warp 0), then every role walks the list ----
         if (warp == 0) {
             long long next;
-            const int ns = build_segments(p, HR, cursor, share_hi, segs, &next, lane);
+            const int ns = build_segments(p, Hkv, rt_blk, cursor, share_hi, segs, &next, lane);
             if (lane == 0) {
                 *sh_nseg = ns;
                 *sh_cursor = next;
@@ -561,9 +568,9 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     if (wtid == 0) p.unit_parts[unit] = make_int2(-1, -1);      // nothing for the merge kernel to do
                     continue;
                 }
-                // partial result: O / l and the log2-sum-exp, in slot (unit index + block index)
+                // partial result: O / l and the log2-sum-exp, in slot ((sequence, KV head) index + group index, row tile)
                 {
-                    const size_t slot = unit + j;
+                    const size_t slot = ((size_t)g.b * Hkv + kvh + jg) * p.row_tiles + rt;
                     float* dst = p.part_o + (slot * 128 + row) * HD;
 #pragma unroll
                     for (int cc = 0; cc < HD / 32; ++cc) {
@@ -584,8 +591,8 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 // the segment that holds the unit's first tile tells the merge kernel which blocks share the unit
                 if (g.t_a == 0 && wtid == 0) {
                     const int tiles_u = last_tile + 1;
-                    const int j_lo = (int)(((g.u0 + 1) * p.nc + T - 1) / T) - 1;           // last block starting at or before u0
-                    const int j_hi = (int)(((g.u0 + tiles_u) * p.nc + T - 1) / T) - 1;     // last block starting inside the unit
+                    const int j_lo = (int)(((g.u0 + 1) * ncg + T - 1) / T) - 1;           // last group starting at or before u0
+                    const int j_hi = (int)(((g.u0 + tiles_u) * ncg + T - 1) / T) - 1;     // last group starting inside the unit
                     p.unit_parts[unit] = make_int2(j_lo, j_hi);
                 }
             }
@@ -613,7 +620,8 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 
 // Combines the segments of the units that were cut.  One thread block per (unit, 8 * R of its rows); a warp takes R
 // rows at a time so that their loads are in flight together (R = 4, or 1 when that is what it takes to fill the GPU).
-// unit_parts[u] = (first, last) block that holds a piece of unit u, or first < 0 when the unit was written directly.
+// unit_parts[u] = (first, last) block group that holds a piece of unit u, or first < 0 when the unit was written
+// directly.
 template <int R>
 __global__ void __launch_bounds__(256) attn_umma_merge_kernel(const AttnParams p) {
     constexpr int BPU = 128 / (8 * R);                            // thread blocks per unit
@@ -630,12 +638,16 @@ __global__ void __launch_bounds__(256) attn_umma_merge_kernel(const AttnParams p
     const int r0 = ((blockIdx.x % BPU) * 8 + warp) * R;           // this warp's rows r0 .. r0 + R - 1
     if (r0 >= n_rows_u) return;
     const int j_lo = parts.x, nj = parts.y - parts.x + 1;
-    const float* __restrict__ lse_base = p.part_lse + ((size_t)unit + j_lo) * 128;
-    const float* __restrict__ o_base = p.part_o + ((size_t)unit + j_lo) * 128 * HD;
-    // with fewer tiles than blocks some shares are empty: their slots were never written
+    const int RT = p.row_tiles, ncg = p.nc / RT;
+    // the pieces of a unit sit RT slots apart
+    const size_t slot0 = ((size_t)b * Hkv + kvh + j_lo) * RT + rt;
+    const float* __restrict__ lse_base = p.part_lse + slot0 * 128;
+    const float* __restrict__ o_base = p.part_o + slot0 * 128 * HD;
+    const size_t lse_step = (size_t)RT * 128, o_step = (size_t)RT * 128 * HD;
+    // with fewer tiles than groups some shares are empty: their slots were never written
     const long long T = *p.total_tiles;
-    const bool dense = T >= p.nc;
-    auto live = [&](int jj) { return dense || share_begin(T, j_lo + jj + 1, p.nc) > share_begin(T, j_lo + jj, p.nc); };
+    const bool dense = T >= ncg;
+    auto live = [&](int jj) { return dense || share_begin(T, j_lo + jj + 1, ncg) > share_begin(T, j_lo + jj, ncg); };
 
     float acc[R][4], wsum[R], mx[R];
 #pragma unroll
@@ -649,7 +661,7 @@ __global__ void __launch_bounds__(256) attn_umma_merge_kernel(const AttnParams p
         const bool on = jj < nj && live(jj);
         float l[R];
 #pragma unroll
-        for (int q = 0; q < R; ++q) l[q] = (on && r0 + q < n_rows_u) ? lse_base[(size_t)jj * 128 + r0 + q] : -INFINITY;
+        for (int q = 0; q < R; ++q) l[q] = (on && r0 + q < n_rows_u) ? lse_base[(size_t)jj * lse_step + r0 + q] : -INFINITY;
 #pragma unroll
         for (int q = 0; q < R; ++q) mx[q] = fmaxf(mx[q], l[q]);
     }
@@ -663,7 +675,7 @@ __global__ void __launch_bounds__(256) attn_umma_merge_kernel(const AttnParams p
         float w_mine[R];
 #pragma unroll
         for (int q = 0; q < R; ++q) {
-            const float l = (on && r0 + q < n_rows_u) ? lse_base[(size_t)jj * 128 + r0 + q] : -INFINITY;
+            const float l = (on && r0 + q < n_rows_u) ? lse_base[(size_t)jj * lse_step + r0 + q] : -INFINITY;
             w_mine[q] = (l == -INFINITY) ? 0.f : exp2f(l - mx[q]);
         }
         const int cn = min(32, nj - c0);
@@ -672,7 +684,7 @@ __global__ void __launch_bounds__(256) attn_umma_merge_kernel(const AttnParams p
             float4 v[R];
 #pragma unroll
             for (int q = 0; q < R; ++q)
-                v[q] = *reinterpret_cast<const float4*>(o_base + ((size_t)(c0 + e) * 128 + min(r0 + q, 127)) * HD + lane * 4);
+                v[q] = *reinterpret_cast<const float4*>(o_base + (size_t)(c0 + e) * o_step + (size_t)min(r0 + q, 127) * HD + lane * 4);
 #pragma unroll
             for (int q = 0; q < R; ++q) {
                 const float w = __shfl_sync(0xffffffffu, w_mine[q], e);
@@ -700,11 +712,13 @@ __global__ void __launch_bounds__(256) attn_umma_merge_kernel(const AttnParams p
 }
 
 // Thread blocks for a call: one per SM, fewer when the tiles would not give each of them a few.
-static int pick_blocks(int B, int HR, int max_seq_len) {
+static int pick_blocks(int B, int HR, int HKV, int max_seq_len) {
     const long long t_max = (long long)B * HR * ((max_seq_len + ATT_TILE - 1) / ATT_TILE + 1);
     long long nc = t_max / 8;
     if (nc > NUM_SMS) nc = NUM_SMS;
-    if (nc < 1) nc = 1;
+    const int rt = HR / HKV > 0 ? HR / HKV : 1;
+    nc = nc / rt * rt;                                    // whole groups of row_tiles blocks
+    if (nc < rt) nc = rt;
     return (int)nc;
 }
 
@@ -720,7 +734,7 @@ int umma_row_tiles(int k, int G) {
 size_t umma_workspace_bytes(int B, int k, int Hq, int Hkv, int max_seq_len) {
     const int G = Hq / Hkv > 0 ? Hq / Hkv : 1;
     const int HR = Hkv * umma_row_tiles(k, G);
-    const size_t slots = (size_t)B * HR + umma::pick_blocks(B, HR, max_seq_len);   // slot = unit index + block index
+    const size_t slots = (size_t)B * HR + umma::pick_blocks(B, HR, Hkv, max_seq_len);   // slot = unit index + block index
     return slots * 128 * (umma::HD + 1) * sizeof(float) + (size_t)B * HR * sizeof(int2) + sizeof(long long);
 }
 
@@ -731,7 +745,7 @@ int launch_umma(AttnParams p, cudaStream_t st) {
     p.ipt = 128 / p.G;
     p.row_tiles = umma_row_tiles(p.k, p.G);
     const int HR = Hkv * p.row_tiles;
-    p.nc = pick_blocks(p.B, HR, p.max_seq_len);
+    p.nc = pick_blocks(p.B, HR, Hkv, p.max_seq_len);
     const size_t slots = (size_t)p.B * HR + p.nc;
     p.part_lse = p.part_o + slots * 128 * HD;
     p.total_tiles = reinterpret_cast<long long*>(p.part_lse + slots * 128);      // 8-byte aligned: slots * 128 * 129 floats
