@@ -31,9 +31,9 @@ METRIC = "verified draft tokens/s per verify step"
 UNIT = "tokens/s"
 
 # DRAM bytes (read + write) of one lmhead_umma_kernel launch from ncu, per workload name; absent = not captured for
-# the kernel as it stands.  The capture ran at V = 65536 (542.2 MB of traffic for 537.13 MB algorithmic, ratio 1.0094);
-# every weight row is fetched once by one block, so the traffic scales with V to the full-size launch.
-LMHEAD_TRAFFIC = {"C2-qwen3-8b-verify": int(1244922112 * 1.0094)}
+# the kernel as it stands.  Captured at full size (M = 32, hidden 4096, V = 151936: 1 246 011 392 read + 5 147 392
+# written, dram__bytes_{read,write}.sum alone, one launch), 1.005 x the algorithmic bytes.
+LMHEAD_TRAFFIC = {"C2-qwen3-8b-verify": 1246011392 + 5147392}
 
 
 def load_peaks():
