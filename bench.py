@@ -234,6 +234,7 @@ def run_ours(args, cfg):
 
     def phase_attn():
         if not bidir:
+            vs.fork_draft_stats()          # sampling: the drafter-logit pass starts on a second stream (joined by accept)
             vs.reserve()
         vs.attn(append=not bidir)
 

@@ -54,6 +54,7 @@ extern "C" {
 
 #define DEER_ACC_GREEDY 0
 #define DEER_ACC_SAMPLE 1
+#define DEER_ACC_SAMPLE_PRESTATS 2 /* SAMPLE, the drafter statistics already in the workspace (deer_draft_stats) */
 
 #define DEER_MAX_BLOCK 32
 #define DEER_PAGE_SIZE 16
@@ -219,6 +220,17 @@ int deer_lmhead_select_static(const void* h, const void* w, int M, int hid, int 
  *   accept_len i32 [B];  out_ids i32 [B][k] (-1 padded);  n_out i32 [B]
  * ---------------------------------------------------------------------- */
 size_t deer_accept_workspace_bytes(int mode, int B, int k, int V);
+
+/* The drafter's side of Eq. 5, q(y_i): log-sum-exp of draft_logits[b][i][:] and
+ * the draft token's logit for every block row, one streaming pass over
+ * draft_logits, left in `workspace` (deer_accept's SAMPLE workspace, same size).
+ * q is known before the verifier has run, so this call may be issued on another
+ * stream while deer_block_attn / deer_lmhead_select run; the caller orders it
+ * before deer_accept(DEER_ACC_SAMPLE_PRESTATS, ..., same workspace), which then
+ * skips that pass, and after the previous deer_accept on that workspace.
+ * Errors: as deer_accept. */
+int deer_draft_stats(int B, int k, int V, const int32_t* draft_ids, const float* draft_logits,
+                     void* workspace, size_t workspace_bytes, void* stream);
 
 int deer_accept(int mode, int B, int k, int V,
                 const int32_t* draft_ids, const int32_t* target_ids,

@@ -19,13 +19,13 @@ DEER_OK = 0
 DEER_ERR_INVALID_ARG, DEER_ERR_UNSUPPORTED, DEER_ERR_NO_PAGES, DEER_ERR_CUDA, DEER_ERR_WORKSPACE, DEER_ERR_BAD_PAGE = 1, 2, 3, 4, 5, 6
 DEER_MASK_CAUSAL, DEER_MASK_BIDIR = 0, 1
 DEER_SEL_ARGMAX, DEER_SEL_ARGMAX_LOGPROB, DEER_SEL_SOFTMAX = 0, 1, 2
-DEER_ACC_GREEDY, DEER_ACC_SAMPLE = 0, 1
+DEER_ACC_GREEDY, DEER_ACC_SAMPLE, DEER_ACC_SAMPLE_PRESTATS = 0, 1, 2
 
 EXPORTS = [
     "deer_last_error", "deer_kv_create", "deer_kv_destroy", "deer_kv_reserve", "deer_kv_commit", "deer_kv_status",
     "deer_block_attn_workspace_bytes", "deer_block_attn", "deer_lmhead_workspace_bytes", "deer_lmhead_select",
     "deer_accept_workspace_bytes", "deer_accept", "deer_verify_step_host",
-    "deer_lmhead_static_max_rows", "deer_lmhead_select_static", "deer_emit",
+    "deer_lmhead_static_max_rows", "deer_lmhead_select_static", "deer_emit", "deer_draft_stats",
 ]
 
 
@@ -85,6 +85,7 @@ def lib() -> ctypes.CDLL:
     L.deer_accept.argtypes = [c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_float,
                               c_void_p, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t,
                               c_void_p]
+    L.deer_draft_stats.argtypes = [c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
     L.deer_emit.argtypes = [c_int, c_int, c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p,
                             c_void_p]
     L.deer_verify_step_host.argtypes = [c_void_p, POINTER(deer_step_dev), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
@@ -226,6 +227,11 @@ def deer_accept(mode, B, k, V, draft_ids, target_ids, target_logits, target_lse,
                              _ptr(accept_len), _ptr(out_ids), _ptr(n_out), _ptr(workspace),
                              workspace.numel() * workspace.element_size() if workspace is not None else 0,
                              _stream(stream)))
+
+
+def deer_draft_stats(B, k, V, draft_ids, draft_logits, workspace, stream=None):
+    _check(lib().deer_draft_stats(B, k, V, _ptr(draft_ids), _ptr(draft_logits), _ptr(workspace),
+                                  workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
 def deer_emit(accept_len, out_ids, n_out, eos_id, tokens, n_tokens, finished, keep, stream=None):

@@ -43,59 +43,70 @@ __global__ void accept_greedy_kernel(int B, int k, const int32_t* __restrict__ d
 }
 
 // ---------------------------------------------------------------- sample (a)
-// One block per block row: log-sum-exp of the drafter logits and the draft
-// token's logit.
-__global__ void __launch_bounds__(256) draft_row_stats_kernel(int V, const float* __restrict__ q_logits,
-                                                              const int32_t* __restrict__ draft, float* __restrict__ lse_q,
-                                                              float* __restrict__ zq_draft) {
-    const int row = blockIdx.x;
-    const float* z = q_logits + (size_t)row * V;
-    float m = -INFINITY, s = 0.f;
-    auto push = [&](float x) {
-        if (x > m) {
-            s = s * __expf(m - x) + 1.f;
-            m = x;
-        } else {
-            s += __expf(x - m);
-        }
-    };
-    if ((V & 3) == 0) {
-        const float4* z4 = reinterpret_cast<const float4*>(z);
-        for (int i = threadIdx.x; i < V / 4; i += blockDim.x) {
-            const float4 x = __ldg(z4 + i);
+// A block per block row (the blocks stride over the rows when there are fewer
+// of them): log-sum-exp of the drafter logits and the draft token's logit.
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS) draft_row_stats_kernel(int rows, int V, const float* __restrict__ q_logits,
+                                                                  const int32_t* __restrict__ draft, float* __restrict__ lse_q,
+                                                                  float* __restrict__ zq_draft) {
+    constexpr int NW = THREADS / 32;
+    __shared__ float sm[NW], ss[NW];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int row = blockIdx.x; row < rows; row += gridDim.x) {
+        const float* z = q_logits + (size_t)row * V;
+        float m = -INFINITY, s = 0.f;
+        auto push4 = [&](const float4 x) {
             const float mx = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
             if (mx > m) {
                 s *= __expf(m - mx);
                 m = mx;
             }
             s += __expf(x.x - m) + __expf(x.y - m) + __expf(x.z - m) + __expf(x.w - m);
+        };
+        if ((V & 3) == 0) {
+            const float4* z4 = reinterpret_cast<const float4*>(z);
+            const int n4 = V / 4;
+            int i = threadIdx.x;
+            for (; i + THREADS < n4; i += 2 * THREADS) {       // two loads in flight per thread
+                const float4 x0 = __ldcs(z4 + i), x1 = __ldcs(z4 + i + THREADS);   // read once: evict first
+                push4(x0);
+                push4(x1);
+            }
+            if (i < n4) push4(__ldcs(z4 + i));
+        } else {
+            for (int i = threadIdx.x; i < V; i += THREADS) {
+                const float x = z[i];
+                if (x > m) {
+                    s = s * __expf(m - x) + 1.f;
+                    m = x;
+                } else {
+                    s += __expf(x - m);
+                }
+            }
         }
-    } else {
-        for (int i = threadIdx.x; i < V; i += blockDim.x) push(z[i]);
-    }
-    __shared__ float sm[8], ss[8];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        const float om = __shfl_xor_sync(0xffffffffu, m, o);
-        const float os = __shfl_xor_sync(0xffffffffu, s, o);
-        const float nm = fmaxf(m, om);
-        s = (m > -INFINITY ? s * __expf(m - nm) : 0.f) + (om > -INFINITY ? os * __expf(om - nm) : 0.f);
-        m = nm;
-    }
-    if (lane == 0) {
-        sm[warp] = m;
-        ss[warp] = s;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        float M = -INFINITY;
-        for (int w = 0; w < 8; ++w) M = fmaxf(M, sm[w]);
-        float S = 0.f;
-        for (int w = 0; w < 8; ++w) S += (sm[w] > -INFINITY) ? ss[w] * __expf(sm[w] - M) : 0.f;
-        lse_q[row] = M + logf(S);
-        const int y = draft[row];
-        zq_draft[row] = (y >= 0 && y < V) ? z[y] : -INFINITY;
+        for (int o = 16; o > 0; o >>= 1) {
+            const float om = __shfl_xor_sync(0xffffffffu, m, o);
+            const float os = __shfl_xor_sync(0xffffffffu, s, o);
+            const float nm = fmaxf(m, om);
+            s = (m > -INFINITY ? s * __expf(m - nm) : 0.f) + (om > -INFINITY ? os * __expf(om - nm) : 0.f);
+            m = nm;
+        }
+        if (lane == 0) {
+            sm[warp] = m;
+            ss[warp] = s;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            float M = -INFINITY;
+            for (int w = 0; w < NW; ++w) M = fmaxf(M, sm[w]);
+            float S = 0.f;
+            for (int w = 0; w < NW; ++w) S += (sm[w] > -INFINITY) ? ss[w] * __expf(sm[w] - M) : 0.f;
+            lse_q[row] = M + logf(S);
+            const int y = draft[row];
+            zq_draft[row] = (y >= 0 && y < V) ? z[y] : -INFINITY;
+        }
+        __syncthreads();                                        // sm / ss are reused by the next row
     }
 }
 
@@ -433,8 +444,26 @@ extern "C" int deer_emit(int B, int k, const int32_t* accept_len, const int32_t*
 }
 
 extern "C" size_t deer_accept_workspace_bytes(int mode, int B, int k, int V) {
-    if (mode != DEER_ACC_SAMPLE || B <= 0 || k <= 0 || V <= 0) return 0;
+    if ((mode != DEER_ACC_SAMPLE && mode != DEER_ACC_SAMPLE_PRESTATS) || B <= 0 || k <= 0 || V <= 0) return 0;
     return carve(nullptr, B, k, V).bytes;
+}
+
+extern "C" int deer_draft_stats(int B, int k, int V, const int32_t* draft_ids, const float* draft_logits, void* workspace,
+                                size_t workspace_bytes, void* stream) {
+    DEER_CHECK_ARG(draft_ids && draft_logits, DEER_ERR_INVALID_ARG, "deer_draft_stats: null argument");
+    DEER_CHECK_ARG(k >= 1 && k <= DEER_MAX_BLOCK, DEER_ERR_UNSUPPORTED, "deer_draft_stats: k must be in [1, 32]");
+    DEER_CHECK_ARG(B >= 0 && B <= 65535 && V > 0, DEER_ERR_INVALID_ARG, "deer_draft_stats: bad sizes");
+    if (B == 0) return DEER_OK;
+    DEER_CHECK_ARG(deer_aligned16(draft_logits) && deer_aligned16(workspace), DEER_ERR_INVALID_ARG,
+                   "deer_draft_stats: logits and workspace must be 16-byte aligned");
+    const size_t need = deer_accept_workspace_bytes(DEER_ACC_SAMPLE, B, k, V);
+    DEER_CHECK_ARG(workspace && workspace_bytes >= need, DEER_ERR_WORKSPACE,
+                   "deer_draft_stats: workspace of %zu bytes needed, %zu given", need, workspace_bytes);
+    const SampleWs w = carve(workspace, B, k, V);
+    draft_row_stats_kernel<256><<<B * k, 256, 0, static_cast<cudaStream_t>(stream)>>>(B * k, V, draft_logits, draft_ids, w.lse_q,
+                                                                                     w.zq_draft);
+    DEER_CUDA(cudaGetLastError());
+    return DEER_OK;
 }
 
 extern "C" int deer_accept(int mode, int B, int k, int V, const int32_t* draft_ids, const int32_t* target_ids,
@@ -442,7 +471,8 @@ extern "C" int deer_accept(int mode, int B, int k, int V, const int32_t* draft_i
                            float temperature, const float* draft_logits, const float* u, const float* r, int32_t eos_id,
                            int32_t* accept_len, int32_t* out_ids, int32_t* n_out, void* workspace, size_t workspace_bytes,
                            void* stream) {
-    DEER_CHECK_ARG(mode == DEER_ACC_GREEDY || mode == DEER_ACC_SAMPLE, DEER_ERR_INVALID_ARG, "deer_accept: bad mode");
+    DEER_CHECK_ARG(mode == DEER_ACC_GREEDY || mode == DEER_ACC_SAMPLE || mode == DEER_ACC_SAMPLE_PRESTATS, DEER_ERR_INVALID_ARG,
+                   "deer_accept: bad mode");
     DEER_CHECK_ARG(draft_ids && accept_len && out_ids && n_out, DEER_ERR_INVALID_ARG, "deer_accept: null argument");
     DEER_CHECK_ARG(k >= 1 && k <= DEER_MAX_BLOCK, DEER_ERR_UNSUPPORTED, "deer_accept: k must be in [1, 32]");
     DEER_CHECK_ARG(B >= 0 && B <= 65535, DEER_ERR_UNSUPPORTED, "deer_accept: B must be in [0, 65535]");
@@ -464,8 +494,10 @@ extern "C" int deer_accept(int mode, int B, int k, int V, const int32_t* draft_i
                    "deer_accept: workspace of %zu bytes needed, %zu given", need, workspace_bytes);
     const SampleWs w = carve(workspace, B, k, V);
 
-    draft_row_stats_kernel<<<B * k, 256, 0, st>>>(V, draft_logits, draft_ids, w.lse_q, w.zq_draft);
-    DEER_CUDA(cudaGetLastError());
+    if (mode == DEER_ACC_SAMPLE) {       // otherwise deer_draft_stats has left them in the workspace
+        draft_row_stats_kernel<256><<<B * k, 256, 0, st>>>(B * k, V, draft_logits, draft_ids, w.lse_q, w.zq_draft);
+        DEER_CUDA(cudaGetLastError());
+    }
     accept_scan_kernel<<<(B + 3) / 4, 128, 0, st>>>(B, k, draft_ids, target_lse, target_draft_logit, 1.f / temperature,
                                                      w.lse_q, w.zq_draft, u, accept_len, out_ids, n_out, w.rej_pos,
                                                      w.done);

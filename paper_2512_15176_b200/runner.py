@@ -24,7 +24,7 @@ class VerifyStep:
     the device-resident LM-head weight [V, hid] bf16."""
 
     def __init__(self, cfg: StepConfig, kv: L.KVCache, w: torch.Tensor, max_seq_len: int, device="cuda",
-                 store_logits: Optional[bool] = None):
+                 store_logits: Optional[bool] = None, overlap_draft_stats: bool = True):
         self.cfg, self.kv, self.w, self.max_seq_len = cfg, kv, w, int(max_seq_len)
         B, k, Hq, Hkv, D, M, V = cfg.B, cfg.k, cfg.Hq, cfg.Hkv, cfg.D, cfg.M, cfg.V
         bf, i32, f32 = torch.bfloat16, torch.int32, torch.float32
@@ -54,6 +54,10 @@ class VerifyStep:
         self.acc_ws = _ws(L.deer_accept_workspace_bytes(L.DEER_ACC_SAMPLE if sample else L.DEER_ACC_GREEDY, B, k, V), dev)
         self.scale = 1.0 / math.sqrt(D)
         self.eos_id = -1                # Algorithm 1's EOS break inside a block; < 0 disables
+        # Sampling: the pass over the drafter's logits (q of Eq. 5) needs nothing from the verifier, so run() puts it
+        # on a second stream at the start of the step and joins before the acceptance.
+        self.side = torch.cuda.Stream(device=dev) if (sample and overlap_draft_stats) else None
+        self._stats_forked = False
 
     # ---- inputs -------------------------------------------------------------
     def load(self, q=None, k_blk=None, v_blk=None, h=None, draft_ids=None, q_logits=None, u=None, r=None):
@@ -88,10 +92,25 @@ class VerifyStep:
             L.deer_lmhead_select(self.h, self.w, L.DEER_SEL_SOFTMAX, c.temperature, self.draft_ids, self.target_ids, None,
                                  self.lse, self.draft_logit, self.logits, self.lm_ws)
 
+    def fork_draft_stats(self):
+        """Start the pass over the drafter's logits on the side stream (no-op without one); accept() joins it."""
+        if self.side is None:
+            return
+        c = self.cfg
+        self.side.wait_stream(torch.cuda.current_stream())   # after the inputs and the previous step's acceptance
+        with torch.cuda.stream(self.side):
+            L.deer_draft_stats(c.B, c.k, c.V, self.draft_ids, self.q_logits, self.acc_ws)
+        self._stats_forked = True
+
     def accept(self):
         c = self.cfg
+        prestats = self._stats_forked
+        if prestats:
+            torch.cuda.current_stream().wait_stream(self.side)
+            self._stats_forked = False
         if c.mode == "sample":
-            L.deer_accept(L.DEER_ACC_SAMPLE, c.B, c.k, c.V, self.draft_ids, None, self.logits, self.lse, self.draft_logit,
+            L.deer_accept(L.DEER_ACC_SAMPLE_PRESTATS if prestats else L.DEER_ACC_SAMPLE, c.B, c.k, c.V, self.draft_ids, None,
+                          self.logits, self.lse, self.draft_logit,
                           c.temperature, self.q_logits, self.u, self.r, self.eos_id, self.accept_len, self.out_ids, self.n_out,
                           self.acc_ws)
         else:
@@ -108,6 +127,9 @@ class VerifyStep:
             self.attn(append=False)
             self.lmhead()
             return
+        # At the start of the step: beside the page reservation and the attention kernel's set-up.  (Beside the LM head
+        # it cost more than it hid: that kernel is tensor-bound and lost 70-80 us to the company, measured.)
+        self.fork_draft_stats()
         self.reserve()
         self.attn(append=True)
         self.lmhead()

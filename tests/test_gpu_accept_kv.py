@@ -41,7 +41,8 @@ def test_greedy_bit_exact(B, k):
             np.testing.assert_array_equal(got[0], Lp)      # the planted-prefix invariant
 
 
-def _sample(cfg, zt32, ql, drafts, u, r, eos=-1):
+def _sample(cfg, zt32, ql, drafts, u, r, eos=-1, split=False):
+    """split: the drafter statistics come from deer_draft_stats on a second stream, joined before the acceptance."""
     from paper_2512_15176_b200 import binding as L
     B, k, V = cfg.B, cfg.k, cfg.V
     dev = "cuda"
@@ -52,8 +53,17 @@ def _sample(cfg, zt32, ql, drafts, u, r, eos=-1):
     o = torch.full((B, k), -9, dtype=torch.int32, device=dev)
     n = torch.full((B,), -9, dtype=torch.int32, device=dev)
     ws = torch.empty(L.deer_accept_workspace_bytes(L.DEER_ACC_SAMPLE, B, k, V), dtype=torch.uint8, device=dev)
-    L.deer_accept(L.DEER_ACC_SAMPLE, B, k, V, torch.as_tensor(drafts, device=dev), None, torch.from_numpy(zt32).to(dev), lse, zd,
-                  cfg.temperature, ql.to(dev), u.to(dev), r.to(dev), eos, a, o, n, ws)
+    d_dev, ql_dev = torch.as_tensor(drafts, device=dev), ql.to(dev)
+    mode = L.DEER_ACC_SAMPLE
+    if split:
+        mode = L.DEER_ACC_SAMPLE_PRESTATS
+        side, main = torch.cuda.Stream(), torch.cuda.current_stream()
+        side.wait_stream(main)
+        with torch.cuda.stream(side):
+            L.deer_draft_stats(B, k, V, d_dev, ql_dev, ws)
+        main.wait_stream(side)
+    L.deer_accept(mode, B, k, V, d_dev, None, torch.from_numpy(zt32).to(dev), lse, zd,
+                  cfg.temperature, ql_dev, u.to(dev), r.to(dev), eos, a, o, n, ws)
     torch.cuda.synchronize()
     return a.cpu().numpy(), o.cpu().numpy(), n.cpu().numpy()
 
@@ -72,6 +82,10 @@ def test_sampling_bit_exact_on_identical_logits(B, k, V, T):
     for g, w_, name in zip(got, want, ("accept_len", "out_ids", "n_out")):
         np.testing.assert_array_equal(g, w_, err_msg=name)
     assert len(set(want[0].tolist())) > 1 or B < 4
+    # the drafter statistics computed ahead of time on another stream: same result
+    got = _sample(cfg, zt32, ql, drafts, u, r, split=True)
+    for g, w_, name in zip(got, want, ("accept_len", "out_ids", "n_out")):
+        np.testing.assert_array_equal(g, w_, err_msg=name + " (deer_draft_stats)")
     # EOS: cut at a token that the oracle emitted
     eos = int(want[1][0, 0])
     got = _sample(cfg, zt32, ql, drafts, u, r, eos)
