@@ -128,23 +128,29 @@ def _truncate_at_eos(out_row, n_out, accept_len, eos_id):
     return n_out, accept_len
 
 
-def accept_greedy(draft_ids, target_ids, eos_id=-1):
+def accept_greedy(draft_ids, target_ids, eos_id=-1, bonus=False):
     """Temperature 0: p_AR is one-hot on the target argmax, so alpha_i is 1 if
     draft == target and 0 otherwise, and the residual is that one-hot.
-    Returns (accept_len [B], out_ids [B,k] padded with -1, n_out [B])."""
+    Returns (accept_len [B], out_ids [B,k] padded with -1, n_out [B]).
+
+    bonus: the block's k rows hold k-1 drafts (draft_ids[:, k-1] is ignored); row i
+    judges draft i, and when all k-1 are accepted the last row, whose input was the
+    last draft, gives one more token -- the parallel pass has p_AR(. | all drafts)
+    anyway.  Every block then emits accept_len + 1 tokens."""
     draft_ids = np.asarray(draft_ids)
     target_ids = np.asarray(target_ids)
     B, k = draft_ids.shape
+    kd = k - 1 if bonus else k                  # drafts under test
     accept_len = np.zeros(B, dtype=np.int32)
     out_ids = np.full((B, k), -1, dtype=np.int32)
     n_out = np.zeros(B, dtype=np.int32)
     for b in range(B):
         a = 0
-        while a < k and draft_ids[b, a] == target_ids[b, a]:
+        while a < kd and draft_ids[b, a] == target_ids[b, a]:
             out_ids[b, a] = draft_ids[b, a]
             a += 1
         n = a
-        if a < k:
+        if a < k:                               # a correction, or (bonus, a == k-1) the extra token
             out_ids[b, a] = target_ids[b, a]
             n = a + 1
         n, a = _truncate_at_eos(out_ids[b], n, a, eos_id)
@@ -174,7 +180,7 @@ def inverse_cdf(weights, total, r):
     return v
 
 
-def accept_sample(draft_ids, target_logits, temperature, draft_logits, u, r, eos_id=-1):
+def accept_sample(draft_ids, target_logits, temperature, draft_logits, u, r, eos_id=-1, bonus=False):
     """Speculative rejection sampling over one block per sequence.
 
     For i = 0..k-1: p = softmax(target_logits[b,i] / T), q = softmax(draft_logits[b,i]);
@@ -182,16 +188,22 @@ def accept_sample(draft_ids, target_logits, temperature, draft_logits, u, r, eos
     first rejection draw one token from the normalised residual max(0, p - q)
     (Eq. 6) by inverse CDF with r[b] in vocabulary order and stop; if the residual
     mass is exactly zero, draw from p instead.  No extra token is emitted when all
-    k drafts are accepted."""
+    k drafts are accepted.
+
+    bonus: the k rows hold k-1 drafts (column k-1 of draft_ids, draft_logits and u is
+    ignored); when all are accepted one more token is drawn from the last row's p
+    itself by the same inverse CDF with r[b] (nothing was proposed there, so there
+    is nothing to reject: the residual of p against q = 0 is p)."""
     draft_ids = np.asarray(draft_ids)
     B, k = draft_ids.shape
+    kd = k - 1 if bonus else k
     accept_len = np.zeros(B, dtype=np.int32)
     out_ids = np.full((B, k), -1, dtype=np.int32)
     n_out = np.zeros(B, dtype=np.int32)
     for b in range(B):
         a = 0
         n = 0
-        for i in range(k):
+        for i in range(kd):
             y = int(draft_ids[b, i])
             zp = np.asarray(target_logits[b, i], dtype=np.float64) / float(temperature)
             zq = np.asarray(draft_logits[b, i], dtype=np.float64)
@@ -212,6 +224,10 @@ def accept_sample(draft_ids, target_logits, temperature, draft_logits, u, r, eos
                 out_ids[b, i] = inverse_cdf(p, p.sum(), float(r[b]))
             n += 1
             break
+        if bonus and a == kd:
+            p = softmax_f64(target_logits[b, kd], temperature)
+            out_ids[b, kd] = inverse_cdf(p, p.sum(), float(r[b]))
+            n += 1
         n, a = _truncate_at_eos(out_ids[b], n, a, eos_id)
         accept_len[b] = a
         n_out[b] = n
@@ -305,10 +321,14 @@ class DecodeState:
         self.n_tokens = np.zeros(B, dtype=np.int32)
         self.finished = np.zeros(B, dtype=np.int32)
 
-    def emit(self, accept_len, out_ids, n_out, eos_id=-1):
+    def emit(self, accept_len, out_ids, n_out, eos_id=-1, pending=False):
         """Append this block's chosen tokens (``out_ids[b][:n_out[b]]``, already cut
         after an EOS by the acceptance rule).  A sequence that has finished emits
-        nothing and keeps nothing.  Returns keep [B]: cache rows to commit."""
+        nothing and keeps nothing.  Returns keep [B]: cache rows to commit.
+
+        pending: row 0 of the block was the token emitted last (its keys and values
+        were not in the cache yet) and rows 1.. the drafts, so one more row stays:
+        that token's, followed by the accepted drafts'."""
         B = self.tokens.shape[0]
         keep = np.zeros(B, dtype=np.int32)
         for b in range(B):
@@ -319,7 +339,7 @@ class DecodeState:
             for i in range(m):
                 self.tokens[b, self.n_tokens[b] + i] = out_ids[b][i]
             self.n_tokens[b] += m
-            keep[b] = min(int(accept_len[b]), m)
+            keep[b] = min(int(accept_len[b]), m) + (1 if pending else 0)
             hit_eos = eos_id >= 0 and any(int(out_ids[b][i]) == eos_id for i in range(m))
             if hit_eos or self.n_tokens[b] >= self.max_new:
                 self.finished[b] = 1

@@ -63,3 +63,19 @@ def test_eos_ends_a_sequence_and_later_passes_are_ignored():
     assert keep.tolist() == [2] and st.finished.tolist() == [1] and st.tokens[0, :3].tolist() == [3, 7, -1]
     keep = st.emit(np.array([4]), np.array([[1, 2, 3, 4]]), np.array([4]), eos_id=7)
     assert keep.tolist() == [0] and st.n_tokens.tolist() == [2]
+
+
+def test_pending_token_alignment_hand_worked():
+    """Row 0 of a block is the token emitted last, rows 1.. the drafts (k = 4 rows,
+    3 drafts, every block emits accept_len + 1 tokens).  By hand:
+    pass 1: seq0 accepts 2 drafts + correction [4,5,6] -> keeps the pending token's
+            row and the 2 drafts' rows = 3; seq1 accepts all 3 + the extra token
+            [1,2,3,7] -> keeps 4 rows
+    pass 2: seq0 has room for 1 of [8,9] (max 4 new tokens) -> keeps 1 + min(1, 1) = 2,
+            finished; seq1 was full after pass 1 -> finished there, keeps nothing now."""
+    st = O.DecodeState(2, 4)
+    keep = st.emit(np.array([2, 3]), np.array([[4, 5, 6, -1], [1, 2, 3, 7]]), np.array([3, 4]), pending=True)
+    assert keep.tolist() == [3, 4] and st.n_tokens.tolist() == [3, 4] and st.finished.tolist() == [0, 1]
+    keep = st.emit(np.array([1, 0]), np.array([[8, 9, -1, -1], [5, -1, -1, -1]]), np.array([2, 1]), pending=True)
+    assert keep.tolist() == [2, 0]
+    assert st.tokens.tolist() == [[4, 5, 6, 8], [1, 2, 3, 7]] and st.finished.tolist() == [1, 1]

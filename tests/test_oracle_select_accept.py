@@ -254,3 +254,74 @@ def test_sampling_eos():
     d = np.array([[1, 2, 3, 4]], dtype=np.int32)
     a, out, n = O.accept_sample(d, z, 1.0, z, np.full((1, 4), 0.5), np.array([0.5]), eos_id=2)
     assert a[0] == 2 and n[0] == 2 and out[0].tolist() == [1, 2, -1, -1]
+
+
+# ---------------------------------------------------------------- the extra token after a fully accepted block
+
+def test_greedy_bonus_exhaustive_small():
+    """k rows = k-1 drafts + one more row.  By the definition: the emitted tokens are
+    the target tokens up to and including the first mismatch among the k-1 drafts,
+    or all k target tokens when every draft matches; always accept_len + 1 of them."""
+    for k in range(1, 5):
+        for target in itertools.product(range(3), repeat=k):
+            drafts = np.array(list(itertools.product(range(3), repeat=k)), dtype=np.int32)
+            tgt = np.broadcast_to(np.array(target, dtype=np.int32), drafts.shape)
+            a, out, n = O.accept_greedy(drafts, tgt, bonus=True)
+            for row in range(drafts.shape[0]):
+                mism = [i for i in range(k - 1) if drafts[row, i] != target[i]]
+                first = mism[0] if mism else k - 1
+                assert a[row] == first and n[row] == first + 1
+                assert out[row, :n[row]].tolist() == list(target[:n[row]])
+                assert (out[row, n[row]:] == -1).all()
+
+
+def test_sampling_bonus_monte_carlo():
+    """With the extra row every block emits accept_len + 1 tokens, each distributed as
+    the verifier's own distribution of its row: the first token as p_0 whatever
+    happens, and the token after k-1 accepted drafts as p_{k-1} itself.  The mean
+    number of emitted tokens is 1 + sum_i prod_{t<=i} gamma_t (a closed form)."""
+    rng = np.random.default_rng(321)
+    V, k, N = 10, 3, 150000
+    zp = rng.normal(size=(k, V)) * 1.2
+    zq = zp + rng.normal(size=(k, V)) * 0.6
+    T = 0.9
+    p = sp_softmax(zp / T, axis=1)
+    q = sp_softmax(zq, axis=1)
+    drafts = np.stack([rng.choice(V, size=N, p=q[i]) for i in range(k)], axis=1).astype(np.int32)
+    u = rng.random((N, k))
+    r = rng.random(N)
+    a, out, n = O.accept_sample(drafts, np.broadcast_to(zp, (N, k, V)), T, np.broadcast_to(zq, (N, k, V)), u, r, bonus=True)
+    assert (n == a + 1).all() and a.max() == k - 1
+    first = np.bincount(out[:, 0], minlength=V) / N
+    assert (np.abs(first - p[0]) < 4.5 * np.sqrt(p[0] * (1 - p[0]) / N)).all()
+    full = a == k - 1
+    emp = np.bincount(out[full, k - 1], minlength=V) / full.sum()
+    assert (np.abs(emp - p[k - 1]) < 4.5 * np.sqrt(p[k - 1] * (1 - p[k - 1]) / full.sum()) + 1e-9).all()
+    gam = np.minimum(p, q).sum(axis=1)
+    want = 1.0 + sum(float(np.prod(gam[:i])) for i in range(1, k))
+    assert abs(n.mean() - want) < 4.5 * n.std() / math.sqrt(N)
+    # the draft in the last column is never looked at
+    drafts2 = drafts.copy()
+    drafts2[:, k - 1] = (drafts2[:, k - 1] + 1) % V
+    a2, out2, n2 = O.accept_sample(drafts2, np.broadcast_to(zp, (N, k, V)), T, np.broadcast_to(zq, (N, k, V)), u, r, bonus=True)
+    assert (a2 == a).all() and (out2 == out).all()
+
+
+def test_sampling_bonus_with_one_row_is_plain_sampling():
+    """k = 1: no drafts at all, the block is one ordinary decoding step: the token is
+    the inverse CDF of p at r (brute force over the cumulative sums)."""
+    rng = np.random.default_rng(5)
+    V = 7
+    z = rng.normal(size=(4, 1, V))
+    r = np.array([0.05, 0.4, 0.77, 0.999])
+    a, out, n = O.accept_sample(np.zeros((4, 1), np.int32), z, 1.3, z, np.full((4, 1), 0.5), r, bonus=True)
+    assert a.tolist() == [0] * 4 and n.tolist() == [1] * 4
+    for b in range(4):
+        pb = sp_softmax(z[b, 0] / 1.3)
+        acc, want = 0.0, None
+        for v in range(V):
+            acc += pb[v]
+            if acc >= r[b]:
+                want = v
+                break
+        assert out[b, 0] == want
