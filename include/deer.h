@@ -55,6 +55,8 @@ extern "C" {
 #define DEER_ACC_GREEDY 0
 #define DEER_ACC_SAMPLE 1
 #define DEER_ACC_SAMPLE_PRESTATS 2 /* SAMPLE, the drafter statistics already in the workspace (deer_draft_stats) */
+#define DEER_ACC_BONUS 4           /* or-ed into the mode: the k rows are k-1 drafts and one more row (see deer_accept) */
+#define DEER_EMIT_PENDING 1        /* deer_emit flag: row 0 of the block was the token emitted last */
 
 #define DEER_MAX_BLOCK 32
 #define DEER_PAGE_SIZE 16
@@ -208,8 +210,14 @@ int deer_lmhead_select_static(const void* h, const void* w, int M, int hid, int 
  *   q = softmax(draft_logits); accept iff u[b][i] <= alpha_i; at the first
  *   rejection one token is drawn from max(0, p - q) normalised, by inverse CDF
  *   in vocabulary order with r[b] (fp64 sums); if that mass is zero, from p.
- * No extra token is emitted when all k are accepted.  If eos_id >= 0 nothing is
- * emitted after the first emitted eos_id.
+ * No extra token is emitted when all k are accepted (Algorithm 1 as printed).
+ * With DEER_ACC_BONUS or-ed into the mode the block's k rows are k-1 drafts
+ * followed by one more row whose input was the last draft: column k-1 of
+ * draft_ids, draft_logits and u is ignored, and when all k-1 drafts are accepted
+ * one more token is taken from that row's p itself (GREEDY: target_ids[b][k-1];
+ * SAMPLE: inverse CDF of p with r[b]), so every block emits accept_len + 1
+ * tokens -- the parallel pass has that distribution anyway.  If eos_id >= 0
+ * nothing is emitted after the first emitted eos_id.
  *   draft_ids           i32 [B][k]
  *   target_ids          i32 [B][k]        GREEDY
  *   target_logits       f32 [B][k][V]     SAMPLE (deer_lmhead_select's out_logits)
@@ -249,6 +257,9 @@ int deer_accept(int mode, int B, int k, int V,
  * tokens; keep[b] = min(accept_len[b], tokens appended) is what
  * deer_kv_commit should keep.  A finished sequence appends nothing and gets
  * keep[b] = 0, so it may stay in the batch of later passes.
+ * flags & DEER_EMIT_PENDING: row 0 of the block was the token emitted last (its
+ * keys and values were not in the cache yet) and rows 1.. the drafts; one more
+ * row is then kept, keep[b] = 1 + min(accept_len[b], tokens appended).
  *   accept_len, n_out  i32 [B];  out_ids  i32 [B][k]
  *   tokens    i32 [B][max_new]  output tokens so far (caller fills it with -1 before the first pass)
  *   n_tokens  i32 [B]           their number           (caller zeroes it before the first pass)
@@ -257,7 +268,7 @@ int deer_accept(int mode, int B, int k, int V,
  * ---------------------------------------------------------------------- */
 int deer_emit(int B, int k, const int32_t* accept_len, const int32_t* out_ids, const int32_t* n_out,
               int32_t eos_id, int32_t max_new, int32_t* tokens, int32_t* n_tokens, int32_t* finished,
-              int32_t* keep, void* stream);
+              int32_t* keep, int flags, void* stream);
 
 /* ------------------------------------------------------------------------
  * One whole greedy verify step with HOST inputs and outputs (Algorithm 1, one

@@ -19,7 +19,8 @@ DEER_OK = 0
 DEER_ERR_INVALID_ARG, DEER_ERR_UNSUPPORTED, DEER_ERR_NO_PAGES, DEER_ERR_CUDA, DEER_ERR_WORKSPACE, DEER_ERR_BAD_PAGE = 1, 2, 3, 4, 5, 6
 DEER_MASK_CAUSAL, DEER_MASK_BIDIR = 0, 1
 DEER_SEL_ARGMAX, DEER_SEL_ARGMAX_LOGPROB, DEER_SEL_SOFTMAX = 0, 1, 2
-DEER_ACC_GREEDY, DEER_ACC_SAMPLE, DEER_ACC_SAMPLE_PRESTATS = 0, 1, 2
+DEER_ACC_GREEDY, DEER_ACC_SAMPLE, DEER_ACC_SAMPLE_PRESTATS, DEER_ACC_BONUS = 0, 1, 2, 4
+DEER_EMIT_PENDING = 1
 
 EXPORTS = [
     "deer_last_error", "deer_kv_create", "deer_kv_destroy", "deer_kv_reserve", "deer_kv_commit", "deer_kv_status",
@@ -87,7 +88,7 @@ def lib() -> ctypes.CDLL:
                               c_void_p]
     L.deer_draft_stats.argtypes = [c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
     L.deer_emit.argtypes = [c_int, c_int, c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p,
-                            c_void_p]
+                            c_int, c_void_p]
     L.deer_verify_step_host.argtypes = [c_void_p, POINTER(deer_step_dev), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                         c_void_p, c_int, c_int, c_int, c_int, c_int, c_float, c_int, c_void_p, c_void_p,
                                         c_void_p, c_void_p]
@@ -234,10 +235,10 @@ def deer_draft_stats(B, k, V, draft_ids, draft_logits, workspace, stream=None):
                                   workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
-def deer_emit(accept_len, out_ids, n_out, eos_id, tokens, n_tokens, finished, keep, stream=None):
+def deer_emit(accept_len, out_ids, n_out, eos_id, tokens, n_tokens, finished, keep, flags=0, stream=None):
     B, k = out_ids.shape
     _check(lib().deer_emit(B, k, _ptr(accept_len), _ptr(out_ids), _ptr(n_out), int(eos_id), tokens.shape[1], _ptr(tokens),
-                           _ptr(n_tokens), _ptr(finished), _ptr(keep), _stream(stream)))
+                           _ptr(n_tokens), _ptr(finished), _ptr(keep), int(flags), _stream(stream)))
 
 
 def deer_verify_step_host(kv: KVCache, dev: deer_step_dev, w, q_host, k_blk_host, v_blk_host, h_host, draft_ids_host,

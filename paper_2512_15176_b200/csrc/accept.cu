@@ -17,7 +17,7 @@ constexpr int NS = 32;             // vocabulary slices per rejected row
 constexpr int RES_THREADS = 256;
 
 // ---------------------------------------------------------------- greedy
-__global__ void accept_greedy_kernel(int B, int k, const int32_t* __restrict__ draft, const int32_t* __restrict__ target,
+__global__ void accept_greedy_kernel(int B, int k, int kd, const int32_t* __restrict__ draft, const int32_t* __restrict__ target,
                                      int32_t eos_id, int32_t* __restrict__ accept_len, int32_t* __restrict__ out_ids,
                                      int32_t* __restrict__ n_out) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
@@ -26,7 +26,7 @@ __global__ void accept_greedy_kernel(int B, int k, const int32_t* __restrict__ d
     const int32_t* t = target + (size_t)b * k;
     int32_t* o = out_ids + (size_t)b * k;
     int a = 0;
-    while (a < k && d[a] == t[a]) ++a;
+    while (a < kd && d[a] == t[a]) ++a;          // kd = k - 1 with the extra row: then a < k and t[a] is always emitted
     int n = a < k ? a + 1 : a;
     for (int i = 0; i < k; ++i) o[i] = i < a ? d[i] : (i == a ? t[i] : -1);
     if (eos_id >= 0) {
@@ -112,31 +112,32 @@ __global__ void __launch_bounds__(THREADS) draft_row_stats_kernel(int rows, int 
 
 // ---------------------------------------------------------------- sample (b)
 // One warp per sequence, lane i = block row i.
-__global__ void __launch_bounds__(128) accept_scan_kernel(int B, int k, const int32_t* __restrict__ draft,
+__global__ void __launch_bounds__(128) accept_scan_kernel(int B, int k, int kd, const int32_t* __restrict__ draft,
                                                           const float* __restrict__ lse_p, const float* __restrict__ zp_draft,
                                                           float inv_t, const float* __restrict__ lse_q,
                                                           const float* __restrict__ zq_draft, const float* __restrict__ u,
                                                           int32_t* __restrict__ accept_len, int32_t* __restrict__ out_ids,
                                                           int32_t* __restrict__ n_out, int32_t* __restrict__ rej_pos,
-                                                          int32_t* __restrict__ done) {
+                                                          int32_t* __restrict__ from_p, int32_t* __restrict__ done) {
     const int b = blockIdx.x * 4 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (b >= B) return;
     bool acc = true;
     int y = -1;
-    if (lane < k) {
+    if (lane < kd) {
         const size_t r = (size_t)b * k + lane;
         y = draft[r];
         const float log_alpha = fminf(0.f, (zp_draft[r] * inv_t - lse_p[r]) - (zq_draft[r] - lse_q[r]));
         acc = logf(u[r]) <= log_alpha;
     }
     const unsigned rejected = ~__ballot_sync(0xffffffffu, acc);
-    const int a = rejected ? __ffs(rejected) - 1 : k;     // lanes >= k always vote "accepted"
+    const int a = rejected ? __ffs(rejected) - 1 : kd;    // lanes >= kd always vote "accepted"
     if (lane < k) out_ids[(size_t)b * k + lane] = lane < a ? y : -1;
     if (lane == 0) {
         accept_len[b] = a;
         n_out[b] = a < k ? a + 1 : k;
-        rej_pos[b] = a < k ? a : -1;
+        rej_pos[b] = a < k ? a : -1;    // the row a token is drawn from: the first rejection, or the extra row
+        from_p[b] = (a == kd) ? 1 : 0;  // nothing was proposed for that row: the token comes from p itself
         done[b] = 0;                    // slices of the residual pass finished so far
     }
 }
@@ -148,6 +149,7 @@ __global__ void __launch_bounds__(128) accept_scan_kernel(int B, int k, const in
 struct ResidualArgs {
     int B, k, V, slice;
     const int32_t* rej_pos;
+    const int32_t* from_p;        // [B] 1: draw from p (the extra row after k-1 accepted drafts), q counts as 0
     const float* target_logits;   // [B][k][V]
     const float* draft_logits;    // [B][k][V]
     const float* lse_p;
@@ -205,7 +207,15 @@ __global__ void __launch_bounds__(RES_THREADS) residual_norm_kernel(ResidualArgs
     double* ep = a.e_p + (size_t)b * a.V;
     double* eq = a.e_q + (size_t)b * a.V;
     int v = v0 + threadIdx.x;
-    if ((a.V & 3) == 0) {
+    if (a.from_p[b]) {
+        // the extra row: only p is needed
+        for (; v < v1; v += RES_THREADS) {
+            const double x = exp((double)zp[v] * it - lp);
+            ep[v] = x;
+            eq[v] = 0.0;
+            sp += x;
+        }
+    } else if ((a.V & 3) == 0) {
         // v0 and V are multiples of 4, so v1 - v0 is as well
         for (int q = v0 + 4 * threadIdx.x; q < v1; q += 4 * RES_THREADS) {
             const float4 p4 = __ldg(reinterpret_cast<const float4*>(zp + q));
@@ -262,7 +272,7 @@ __global__ void __launch_bounds__(RES_THREADS) residual_pick_kernel(ResidualArgs
         Sp += a.sums[((size_t)b * NS + j) * 4 + 0];
         Sq += a.sums[((size_t)b * NS + j) * 4 + 1];
     }
-    const double ip = 1.0 / Sp, iq = 1.0 / Sq;
+    const double ip = 1.0 / Sp, iq = a.from_p[b] ? 0.0 : 1.0 / Sq;
     auto resid2 = [&](double x, double y) {
         const double res = x * ip - y * iq;
         return res > 0.0 ? res : 0.0;
@@ -372,7 +382,8 @@ __global__ void __launch_bounds__(RES_THREADS) residual_pick_kernel(ResidualArgs
 // sequence has finished (EOS or length limit), and how many cache rows survive (Algorithm 1's outer loop).
 __global__ void emit_kernel(int B, int k, const int32_t* __restrict__ accept_len, const int32_t* __restrict__ out_ids,
                             const int32_t* __restrict__ n_out, int32_t eos_id, int32_t max_new, int32_t* __restrict__ tokens,
-                            int32_t* __restrict__ n_tokens, int32_t* __restrict__ finished, int32_t* __restrict__ keep) {
+                            int32_t* __restrict__ n_tokens, int32_t* __restrict__ finished, int32_t* __restrict__ keep,
+                            int pending) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
     if (finished[b]) {
@@ -392,7 +403,7 @@ __global__ void emit_kernel(int B, int k, const int32_t* __restrict__ accept_len
     }
     n_tokens[b] = have + m;
     const int a = accept_len[b];
-    keep[b] = a < m ? (a < 0 ? 0 : a) : m;
+    keep[b] = (a < m ? (a < 0 ? 0 : a) : m) + pending;    // pending: row 0 was the token emitted last; it stays too
     if (eos || have + m >= max_new) finished[b] = 1;
 }
 
@@ -400,6 +411,7 @@ struct SampleWs {
     float* lse_q;
     float* zq_draft;
     int32_t* rej_pos;
+    int32_t* from_p;
     double* e_p;
     double* e_q;
     double* sums;
@@ -420,6 +432,7 @@ SampleWs carve(void* base, int B, int k, int V) {
     w.lse_q = static_cast<float*>(take((size_t)B * k * sizeof(float)));
     w.zq_draft = static_cast<float*>(take((size_t)B * k * sizeof(float)));
     w.rej_pos = static_cast<int32_t*>(take((size_t)B * sizeof(int32_t)));
+    w.from_p = static_cast<int32_t*>(take((size_t)B * sizeof(int32_t)));
     w.e_p = static_cast<double*>(take((size_t)B * V * sizeof(double)));
     w.e_q = static_cast<double*>(take((size_t)B * V * sizeof(double)));
     w.sums = static_cast<double*>(take((size_t)B * NS * 4 * sizeof(double)));
@@ -431,19 +444,23 @@ SampleWs carve(void* base, int B, int k, int V) {
 }  // namespace
 
 extern "C" int deer_emit(int B, int k, const int32_t* accept_len, const int32_t* out_ids, const int32_t* n_out, int32_t eos_id,
-                         int32_t max_new, int32_t* tokens, int32_t* n_tokens, int32_t* finished, int32_t* keep, void* stream) {
+                         int32_t max_new, int32_t* tokens, int32_t* n_tokens, int32_t* finished, int32_t* keep, int flags,
+                         void* stream) {
+    DEER_CHECK_ARG((flags & ~DEER_EMIT_PENDING) == 0, DEER_ERR_INVALID_ARG, "deer_emit: unknown flags");
     DEER_CHECK_ARG(accept_len && out_ids && n_out && (tokens || max_new == 0) && n_tokens && finished && keep, DEER_ERR_INVALID_ARG,
                    "deer_emit: null argument");
     DEER_CHECK_ARG(k >= 1 && k <= DEER_MAX_BLOCK, DEER_ERR_UNSUPPORTED, "deer_emit: k must be in [1, 32]");
     DEER_CHECK_ARG(B >= 0 && max_new >= 0, DEER_ERR_INVALID_ARG, "deer_emit: B and max_new must not be negative");
     if (B == 0) return DEER_OK;
     emit_kernel<<<(B + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(B, k, accept_len, out_ids, n_out, eos_id, max_new,
-                                                                               tokens, n_tokens, finished, keep);
+                                                                               tokens, n_tokens, finished, keep,
+                                                                               (flags & DEER_EMIT_PENDING) ? 1 : 0);
     DEER_CUDA(cudaGetLastError());
     return DEER_OK;
 }
 
 extern "C" size_t deer_accept_workspace_bytes(int mode, int B, int k, int V) {
+    mode &= ~DEER_ACC_BONUS;
     if ((mode != DEER_ACC_SAMPLE && mode != DEER_ACC_SAMPLE_PRESTATS) || B <= 0 || k <= 0 || V <= 0) return 0;
     return carve(nullptr, B, k, V).bytes;
 }
@@ -471,6 +488,8 @@ extern "C" int deer_accept(int mode, int B, int k, int V, const int32_t* draft_i
                            float temperature, const float* draft_logits, const float* u, const float* r, int32_t eos_id,
                            int32_t* accept_len, int32_t* out_ids, int32_t* n_out, void* workspace, size_t workspace_bytes,
                            void* stream) {
+    const int kd = (mode & DEER_ACC_BONUS) ? k - 1 : k;     // drafts under test
+    mode &= ~DEER_ACC_BONUS;
     DEER_CHECK_ARG(mode == DEER_ACC_GREEDY || mode == DEER_ACC_SAMPLE || mode == DEER_ACC_SAMPLE_PRESTATS, DEER_ERR_INVALID_ARG,
                    "deer_accept: bad mode");
     DEER_CHECK_ARG(draft_ids && accept_len && out_ids && n_out, DEER_ERR_INVALID_ARG, "deer_accept: null argument");
@@ -480,7 +499,7 @@ extern "C" int deer_accept(int mode, int B, int k, int V, const int32_t* draft_i
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (mode == DEER_ACC_GREEDY) {
         DEER_CHECK_ARG(target_ids, DEER_ERR_INVALID_ARG, "deer_accept: target_ids is required in GREEDY mode");
-        accept_greedy_kernel<<<(B + 127) / 128, 128, 0, st>>>(B, k, draft_ids, target_ids, eos_id, accept_len, out_ids, n_out);
+        accept_greedy_kernel<<<(B + 127) / 128, 128, 0, st>>>(B, k, kd, draft_ids, target_ids, eos_id, accept_len, out_ids, n_out);
         DEER_CUDA(cudaGetLastError());
         return DEER_OK;
     }
@@ -498,9 +517,9 @@ extern "C" int deer_accept(int mode, int B, int k, int V, const int32_t* draft_i
         draft_row_stats_kernel<256><<<B * k, 256, 0, st>>>(B * k, V, draft_logits, draft_ids, w.lse_q, w.zq_draft);
         DEER_CUDA(cudaGetLastError());
     }
-    accept_scan_kernel<<<(B + 3) / 4, 128, 0, st>>>(B, k, draft_ids, target_lse, target_draft_logit, 1.f / temperature,
+    accept_scan_kernel<<<(B + 3) / 4, 128, 0, st>>>(B, k, kd, draft_ids, target_lse, target_draft_logit, 1.f / temperature,
                                                      w.lse_q, w.zq_draft, u, accept_len, out_ids, n_out, w.rej_pos,
-                                                     w.done);
+                                                     w.from_p, w.done);
     DEER_CUDA(cudaGetLastError());
 
     ResidualArgs a;
@@ -509,6 +528,7 @@ extern "C" int deer_accept(int mode, int B, int k, int V, const int32_t* draft_i
     a.V = V;
     a.slice = ((V + NS - 1) / NS + 3) / 4 * 4;
     a.rej_pos = w.rej_pos;
+    a.from_p = w.from_p;
     a.target_logits = target_logits;
     a.draft_logits = draft_logits;
     a.lse_p = target_lse;

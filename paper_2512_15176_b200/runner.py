@@ -58,6 +58,7 @@ class VerifyStep:
         # on a second stream at the start of the step and joins before the acceptance.
         self.side = torch.cuda.Stream(device=dev) if (sample and overlap_draft_stats) else None
         self._stats_forked = False
+        self.bonus = False              # the k rows are k-1 drafts + one more row (deer_accept's DEER_ACC_BONUS)
 
     # ---- inputs -------------------------------------------------------------
     def load(self, q=None, k_blk=None, v_blk=None, h=None, draft_ids=None, q_logits=None, u=None, r=None):
@@ -108,13 +109,14 @@ class VerifyStep:
         if prestats:
             torch.cuda.current_stream().wait_stream(self.side)
             self._stats_forked = False
+        extra = L.DEER_ACC_BONUS if self.bonus else 0
         if c.mode == "sample":
-            L.deer_accept(L.DEER_ACC_SAMPLE_PRESTATS if prestats else L.DEER_ACC_SAMPLE, c.B, c.k, c.V, self.draft_ids, None,
+            L.deer_accept((L.DEER_ACC_SAMPLE_PRESTATS if prestats else L.DEER_ACC_SAMPLE) | extra, c.B, c.k, c.V, self.draft_ids, None,
                           self.logits, self.lse, self.draft_logit,
                           c.temperature, self.q_logits, self.u, self.r, self.eos_id, self.accept_len, self.out_ids, self.n_out,
                           self.acc_ws)
         else:
-            L.deer_accept(L.DEER_ACC_GREEDY, c.B, c.k, c.V, self.draft_ids, self.target_ids, None, None, None, 1.0, None,
+            L.deer_accept(L.DEER_ACC_GREEDY | extra, c.B, c.k, c.V, self.draft_ids, self.target_ids, None, None, None, 1.0, None,
                           None, None, self.eos_id, self.accept_len, self.out_ids, self.n_out, None)
 
     def commit(self):
@@ -148,11 +150,16 @@ class DecodeLoop:
     and then ``deer_emit`` -- the chosen tokens join each sequence's output,
     a sequence ends at an EOS or at ``max_new`` tokens, and the cache keeps only
     the accepted drafts that were emitted.  Nothing synchronises with the host
-    between passes; finished sequences stay in the batch and are ignored."""
+    between passes; finished sequences stay in the batch and are ignored.
 
-    def __init__(self, step: VerifyStep, eos_id: int, max_new: int):
-        self.vs, self.eos_id = step, int(eos_id)
+    ``pending``: row 0 of every block is the token emitted last (not in the cache
+    yet) and rows 1.. are the drafts; a fully accepted block then yields one more
+    token from its last row, and the cache keeps the pending token's row as well."""
+
+    def __init__(self, step: VerifyStep, eos_id: int, max_new: int, pending: bool = False):
+        self.vs, self.eos_id, self.pending = step, int(eos_id), bool(pending)
         step.eos_id = int(eos_id)
+        step.bonus = self.pending
         B, dev = step.cfg.B, step.q.device
         self.tokens = torch.full((B, max_new), -1, dtype=torch.int32, device=dev)
         self.n_tokens = torch.zeros(B, dtype=torch.int32, device=dev)
@@ -165,5 +172,6 @@ class DecodeLoop:
         vs.attn(append=True)
         vs.lmhead()
         vs.accept()
-        L.deer_emit(vs.accept_len, vs.out_ids, vs.n_out, self.eos_id, self.tokens, self.n_tokens, self.finished, self.keep)
+        L.deer_emit(vs.accept_len, vs.out_ids, vs.n_out, self.eos_id, self.tokens, self.n_tokens, self.finished, self.keep,
+                    L.DEER_EMIT_PENDING if self.pending else 0)
         L.deer_kv_commit(vs.kv, vs.seq_ids, self.keep, vs.cfg.k)

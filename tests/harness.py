@@ -98,9 +98,11 @@ def check_logits(got_f32, z64, label=""):
     assert err.max() <= 1e-3, f"{label}: logits err max {err.max():.3e} (expected ~1e-5)"
 
 
-def sampling_inputs(cfg, zt32, step=0, r_margin=1e-9):
+def sampling_inputs(cfg, zt32, step=0, r_margin=1e-9, bonus=False):
     """Drafter logits, sampled drafts, uniforms with cleared margins.
-    ``zt32`` are the target logits (fp32 values, [B,k,V]) the oracle will use."""
+    ``zt32`` are the target logits (fp32 values, [B,k,V]) the oracle will use.
+    bonus: the last row holds no draft; when the k-1 drafts before it are all
+    accepted, r is cleared against the edges of that row's own CDF."""
     T = float(np.float32(cfg.temperature))
     ql = W.draft_logits(cfg, step)
     drafts = W.sample_drafts(ql, cfg.seed, step)
@@ -109,8 +111,22 @@ def sampling_inputs(cfg, zt32, step=0, r_margin=1e-9):
     gen = W.rng(cfg.seed, f"redraw{step}")
     redraws = 0
     qn = ql.numpy()
+    def clear_r(b, wts, tot):
+        nonlocal redraws
+        cdf = np.cumsum(wts)
+        while True:
+            t = float(r[b]) * tot
+            v = min(int(np.searchsorted(cdf, t, side="left")), cfg.V - 1)
+            lo = cdf[v - 1] if v > 0 else 0.0
+            if t - lo > r_margin * tot and cdf[v] - t > r_margin * tot:
+                return
+            r[b] = np.float32((int(gen.integers(0, 1 << 24)) + 0.5) / (1 << 24))
+            redraws += 1
+
+    kd = cfg.k - 1 if bonus else cfg.k
     for b in range(cfg.B):
-        for i in range(cfg.k):
+        rejected = False
+        for i in range(kd):
             y = int(drafts[b, i])
             zp = zt32[b, i].astype(np.float64) / T
             zq = qn[b, i].astype(np.float64)
@@ -123,16 +139,12 @@ def sampling_inputs(cfg, zt32, step=0, r_margin=1e-9):
                 qd = O.softmax_f64(qn[b, i], 1.0)
                 res, S = O.residual_distribution(p, qd)
                 wts, tot = (res, S) if S > 0 else (p, p.sum())
-                cdf = np.cumsum(wts)
-                while True:
-                    t = float(r[b]) * tot
-                    v = min(int(np.searchsorted(cdf, t, side="left")), cfg.V - 1)
-                    lo = cdf[v - 1] if v > 0 else 0.0
-                    if t - lo > r_margin * tot and cdf[v] - t > r_margin * tot:
-                        break
-                    r[b] = np.float32((int(gen.integers(0, 1 << 24)) + 0.5) / (1 << 24))
-                    redraws += 1
+                clear_r(b, wts, tot)
+                rejected = True
                 break
+        if bonus and not rejected:
+            p = O.softmax_f64(zt32[b, kd], T)
+            clear_r(b, p, p.sum())
     return ql, drafts, torch.from_numpy(u), torch.from_numpy(r), redraws
 
 

@@ -13,14 +13,15 @@ from tests import harness as Hn
 pytestmark = pytest.mark.gpu
 
 
-def _greedy(draft, target, eos=-1):
+def _greedy(draft, target, eos=-1, bonus=False):
     from paper_2512_15176_b200 import binding as L
     B, k = draft.shape
     dev = "cuda"
     a = torch.full((B,), -9, dtype=torch.int32, device=dev)
     o = torch.full((B, k), -9, dtype=torch.int32, device=dev)
     n = torch.full((B,), -9, dtype=torch.int32, device=dev)
-    L.deer_accept(L.DEER_ACC_GREEDY, B, k, 100, torch.as_tensor(draft, device=dev), torch.as_tensor(target, device=dev),
+    L.deer_accept(L.DEER_ACC_GREEDY | (L.DEER_ACC_BONUS if bonus else 0), B, k, 100, torch.as_tensor(draft, device=dev),
+                  torch.as_tensor(target, device=dev),
                   None, None, None, 1.0, None, None, None, eos, a, o, n, None)
     torch.cuda.synchronize()
     return a.cpu().numpy(), o.cpu().numpy(), n.cpu().numpy()
@@ -39,9 +40,14 @@ def test_greedy_bit_exact(B, k):
             np.testing.assert_array_equal(g, w_)
         if eos < 0:
             np.testing.assert_array_equal(got[0], Lp)      # the planted-prefix invariant
+        # k-1 drafts and one more row: always accept_len + 1 tokens
+        got = _greedy(draft, target, eos, bonus=True)
+        want = O.accept_greedy(draft, target, eos, bonus=True)
+        for g, w_ in zip(got, want):
+            np.testing.assert_array_equal(g, w_)
 
 
-def _sample(cfg, zt32, ql, drafts, u, r, eos=-1, split=False):
+def _sample(cfg, zt32, ql, drafts, u, r, eos=-1, split=False, bonus=False):
     """split: the drafter statistics come from deer_draft_stats on a second stream, joined before the acceptance."""
     from paper_2512_15176_b200 import binding as L
     B, k, V = cfg.B, cfg.k, cfg.V
@@ -62,7 +68,7 @@ def _sample(cfg, zt32, ql, drafts, u, r, eos=-1, split=False):
         with torch.cuda.stream(side):
             L.deer_draft_stats(B, k, V, d_dev, ql_dev, ws)
         main.wait_stream(side)
-    L.deer_accept(mode, B, k, V, d_dev, None, torch.from_numpy(zt32).to(dev), lse, zd,
+    L.deer_accept(mode | (L.DEER_ACC_BONUS if bonus else 0), B, k, V, d_dev, None, torch.from_numpy(zt32).to(dev), lse, zd,
                   cfg.temperature, ql_dev, u.to(dev), r.to(dev), eos, a, o, n, ws)
     torch.cuda.synchronize()
     return a.cpu().numpy(), o.cpu().numpy(), n.cpu().numpy()
@@ -92,6 +98,24 @@ def test_sampling_bit_exact_on_identical_logits(B, k, V, T):
     want = O.accept_sample(drafts, zt32, float(np.float32(T)), ql.numpy(), u.numpy(), r.numpy(), eos)
     for g, w_ in zip(got, want):
         np.testing.assert_array_equal(g, w_)
+
+
+@pytest.mark.parametrize("B,k,V,T", [(6, 4, 1000, 1.0), (16, 8, 4099, 0.8), (5, 1, 300, 1.0)])
+def test_sampling_with_the_extra_row(B, k, V, T):
+    """k-1 drafts and one more row.  Target logits close to the drafter's, so that many
+    blocks are accepted in full and draw their last token from p of the extra row; r is
+    cleared against that row's CDF edges too."""
+    cfg = W.StepConfig("sb", B, 4, 2, 64, k, 64, V, (0, 0), mode="sample", temperature=T, seed=760 + V)
+    ql0 = W.draft_logits(cfg)
+    zt32 = (ql0 + W.normal(cfg.seed, "zt", (B, k, V), 0.15, dtype=torch.float32)).numpy() * np.float32(T)
+    ql, drafts, u, r, _ = Hn.sampling_inputs(cfg, zt32, bonus=True)
+    want = O.accept_sample(drafts, zt32, float(np.float32(T)), ql.numpy(), u.numpy(), r.numpy(), bonus=True)
+    assert (want[2] == want[0] + 1).all()
+    assert (want[0] == k - 1).any()                      # the extra row is exercised
+    for split in (False, True):
+        got = _sample(cfg, zt32, ql, drafts, u, r, split=split, bonus=True)
+        for g, w_, name in zip(got, want, ("accept_len", "out_ids", "n_out")):
+            np.testing.assert_array_equal(g, w_, err_msg=name)
 
 
 def test_sampling_identical_distributions_accept_everything():

@@ -13,7 +13,7 @@ from tests import harness as Hn
 pytestmark = pytest.mark.gpu
 
 
-def _emit_only(B, k, max_new, eos_id, passes, seed):
+def _emit_only(B, k, max_new, eos_id, passes, seed, pending=False):
     """deer_emit alone on random accept results."""
     from paper_2512_15176_b200 import binding as L
     rng = W.rng(seed, "emit")
@@ -26,10 +26,10 @@ def _emit_only(B, k, max_new, eos_id, passes, seed):
     for _ in range(passes):
         target = rng.integers(0, 12, size=(B, k)).astype(np.int32)
         draft = np.where(rng.random((B, k)) < 0.7, target, (target + 1) % 12).astype(np.int32)
-        a, out, n = O.accept_greedy(draft, target, eos_id)
-        want_keep = st.emit(a, out, n, eos_id)
+        a, out, n = O.accept_greedy(draft, target, eos_id, bonus=pending)
+        want_keep = st.emit(a, out, n, eos_id, pending=pending)
         L.deer_emit(torch.from_numpy(a).to(dev), torch.from_numpy(out).to(dev), torch.from_numpy(n).to(dev), eos_id, tokens,
-                    n_tokens, finished, keep)
+                    n_tokens, finished, keep, L.DEER_EMIT_PENDING if pending else 0)
         torch.cuda.synchronize()
         np.testing.assert_array_equal(keep.cpu().numpy(), want_keep)
         np.testing.assert_array_equal(tokens.cpu().numpy(), st.tokens)
@@ -45,9 +45,17 @@ def test_emit_bit_exact(B, k, max_new, eos_id):
         assert st.finished.all()                 # 8 passes of >= 1 token fill 3 new tokens
 
 
-def test_greedy_decode_loop_matches_oracle():
+@pytest.mark.parametrize("B,k,max_new,eos_id", [(1, 1, 3, -1), (9, 8, 20, 3), (200, 32, 64, 5)])
+def test_emit_pending_bit_exact(B, k, max_new, eos_id):
+    _emit_only(B, k, max_new, eos_id, passes=8, seed=950 + B, pending=True)
+
+
+@pytest.mark.parametrize("pending", [False, True])
+def test_greedy_decode_loop_matches_oracle(pending):
     """Six passes of the tiny verifier shape, four ragged sequences: one runs into
-    the length limit, the planted EOS ends others early, the rest keep going."""
+    the length limit, the planted EOS ends others early, the rest keep going.
+    pending: k-1 drafts behind the pending token, one more token from the last row,
+    the pending token's row kept in the cache."""
     from paper_2512_15176_b200 import binding as L
     from paper_2512_15176_b200.runner import DecodeLoop, VerifyStep
     passes, max_new = 6, 28                 # sequences 0 and 3 fill up, 2 meets the EOS, 1 keeps going
@@ -69,12 +77,12 @@ def test_greedy_decode_loop_matches_oracle():
         inputs.append((q, kb, vb, h, target, drafts))
     eos_id = int(inputs[1][4][2, 0])             # sequence 2 emits it in the second pass at the latest
     ost = O.DecodeState(cfg.B, max_new)
-    loop = DecodeLoop(vs, eos_id, max_new)
+    loop = DecodeLoop(vs, eos_id, max_new, pending=pending)
     for step, (q, kb, vb, h, target, drafts) in enumerate(inputs):
         assert okv.reserve(ids, cfg.k)
         okv.append(ids, Hn.f64(kb).astype(np.float32), Hn.f64(vb).astype(np.float32))
-        a, out, n = O.accept_greedy(drafts, target, eos_id)
-        okv.commit(ids, ost.emit(a, out, n, eos_id))
+        a, out, n = O.accept_greedy(drafts, target, eos_id, bonus=pending)
+        okv.commit(ids, ost.emit(a, out, n, eos_id, pending=pending))
         vs.load(q, kb, vb, h, drafts)
         loop.one_pass()                          # no synchronisation between the passes
     torch.cuda.synchronize()
