@@ -45,7 +45,7 @@ __global__ void accept_greedy_kernel(int B, int k, int kd, const int32_t* __rest
 // ---------------------------------------------------------------- sample (a)
 // A block per block row (the blocks stride over the rows when there are fewer
 // of them): log-sum-exp of the drafter logits and the draft token's logit.
-template <int THREADS>
+template <int THREADS, int DEPTH>
 __global__ void __launch_bounds__(THREADS) draft_row_stats_kernel(int rows, int V, const float* __restrict__ q_logits,
                                                                   const int32_t* __restrict__ draft, float* __restrict__ lse_q,
                                                                   float* __restrict__ zq_draft) {
@@ -67,12 +67,14 @@ __global__ void __launch_bounds__(THREADS) draft_row_stats_kernel(int rows, int 
             const float4* z4 = reinterpret_cast<const float4*>(z);
             const int n4 = V / 4;
             int i = threadIdx.x;
-            for (; i + THREADS < n4; i += 2 * THREADS) {       // two loads in flight per thread
-                const float4 x0 = __ldcs(z4 + i), x1 = __ldcs(z4 + i + THREADS);   // read once: evict first
-                push4(x0);
-                push4(x1);
+            for (; i + (DEPTH - 1) * THREADS < n4; i += DEPTH * THREADS) {       // DEPTH loads in flight per thread
+                float4 x[DEPTH];
+#pragma unroll
+                for (int d = 0; d < DEPTH; ++d) x[d] = __ldcs(z4 + i + d * THREADS);   // read once: evict first
+#pragma unroll
+                for (int d = 0; d < DEPTH; ++d) push4(x[d]);
             }
-            if (i < n4) push4(__ldcs(z4 + i));
+            for (; i < n4; i += THREADS) push4(__ldcs(z4 + i));
         } else {
             for (int i = threadIdx.x; i < V; i += THREADS) {
                 const float x = z[i];
@@ -477,8 +479,8 @@ extern "C" int deer_draft_stats(int B, int k, int V, const int32_t* draft_ids, c
     DEER_CHECK_ARG(workspace && workspace_bytes >= need, DEER_ERR_WORKSPACE,
                    "deer_draft_stats: workspace of %zu bytes needed, %zu given", need, workspace_bytes);
     const SampleWs w = carve(workspace, B, k, V);
-    draft_row_stats_kernel<256><<<B * k, 256, 0, static_cast<cudaStream_t>(stream)>>>(B * k, V, draft_logits, draft_ids, w.lse_q,
-                                                                                     w.zq_draft);
+    draft_row_stats_kernel<256, 2><<<B * k, 256, 0, static_cast<cudaStream_t>(stream)>>>(B * k, V, draft_logits, draft_ids,
+                                                                                        w.lse_q, w.zq_draft);
     DEER_CUDA(cudaGetLastError());
     return DEER_OK;
 }
@@ -514,7 +516,7 @@ extern "C" int deer_accept(int mode, int B, int k, int V, const int32_t* draft_i
     const SampleWs w = carve(workspace, B, k, V);
 
     if (mode == DEER_ACC_SAMPLE) {       // otherwise deer_draft_stats has left them in the workspace
-        draft_row_stats_kernel<256><<<B * k, 256, 0, st>>>(B * k, V, draft_logits, draft_ids, w.lse_q, w.zq_draft);
+        draft_row_stats_kernel<256, 2><<<B * k, 256, 0, st>>>(B * k, V, draft_logits, draft_ids, w.lse_q, w.zq_draft);
         DEER_CUDA(cudaGetLastError());
     }
     accept_scan_kernel<<<(B + 3) / 4, 128, 0, st>>>(B, k, kd, draft_ids, target_lse, target_draft_logit, 1.f / temperature,
