@@ -479,8 +479,16 @@ extern "C" int deer_draft_stats(int B, int k, int V, const int32_t* draft_ids, c
     DEER_CHECK_ARG(workspace && workspace_bytes >= need, DEER_ERR_WORKSPACE,
                    "deer_draft_stats: workspace of %zu bytes needed, %zu given", need, workspace_bytes);
     const SampleWs w = carve(workspace, B, k, V);
-    draft_row_stats_kernel<256, 2><<<B * k, 256, 0, static_cast<cudaStream_t>(stream)>>>(B * k, V, draft_logits, draft_ids,
-                                                                                        w.lse_q, w.zq_draft);
+    // Meant to run beside the attention kernel, whose blocks take 56 K of an SM's 64 K registers and most of its
+    // shared memory.  Two things let a block of this kernel share an SM with one of those: at most one block per SM
+    // (148 blocks of 256 threads and 32 registers, striding over the rows; a block per row filled the SMs first and
+    // the two kernels took turns), and the same shared-memory carve-out as that kernel asks for -- blocks of kernels
+    // with different carve-outs do not share an SM at all (measured: without it the LM head beside this kernel took
+    // 496 us instead of 283).
+    const int rows = B * k;
+    DEER_CUDA(cudaFuncSetAttribute(draft_row_stats_kernel<256, 4>, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
+    draft_row_stats_kernel<256, 4><<<rows < 148 ? rows : 148, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        rows, V, draft_logits, draft_ids, w.lse_q, w.zq_draft);
     DEER_CUDA(cudaGetLastError());
     return DEER_OK;
 }

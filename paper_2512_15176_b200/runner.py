@@ -129,8 +129,7 @@ class VerifyStep:
             self.attn(append=False)
             self.lmhead()
             return
-        # At the start of the step: beside the page reservation and the attention kernel's set-up.  (Beside the LM head
-        # it cost more than it hid: that kernel is tensor-bound and lost 70-80 us to the company, measured.)
+        # At the start of the step: it runs beside the attention kernel, which leaves bandwidth and issue slots free.
         self.fork_draft_stats()
         self.reserve()
         self.attn(append=True)
