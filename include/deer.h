@@ -278,6 +278,13 @@ int deer_emit(int B, int k, const int32_t* accept_len, const int32_t* out_ids, c
  * lmhead_select(argmax) -> accept(greedy) -> commit(keep = accept_len), and
  * copies accept_len / out_ids / n_out back.  Model state (w, the KV cache)
  * stays on the device.  Returns after the stream has been synchronised.
+ * On a stream other than the legacy default one, with page-locked host
+ * buffers, the first call with a given set of arguments records the copies and
+ * kernels into a CUDA graph and later calls with the same arguments replay it
+ * (one launch instead of sixteen enqueues); the graph belongs to the library
+ * and is replaced when the arguments change.  The environment variable
+ * DEER_STEP_GRAPH=0 turns this off.  Not to be called on a stream that is being
+ * captured.
  * ---------------------------------------------------------------------- */
 typedef struct deer_step_dev {
     void* q; void* k_blk; void* v_blk; void* attn_out;     /* bf16 staging, shapes as in deer_block_attn */

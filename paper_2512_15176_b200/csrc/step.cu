@@ -1,31 +1,81 @@
 // One greedy verify step driven from host buffers: the end-to-end form of
 // Algorithm 1's loop body on the verifier side (copy the block in, score it,
 // accept, commit, copy the verdict out).
+//
+// The five copies in, eight kernels and three copies out are sixteen
+// enqueue calls; issued one by one they cost more host time than the copies
+// take on the bus.  So the sequence is captured once into a CUDA graph, keyed
+// by every argument, and replayed with one launch while the arguments stay
+// the same (a decoding loop calls with the same buffers every step).
+// DEER_STEP_GRAPH=0 turns this off; pageable host buffers and a stream that
+// is already being captured take the plain path too.
+
+#include <stdlib.h>
+#include <string.h>
+
+#include <mutex>
 
 #include "common.cuh"
 
-extern "C" int deer_verify_step_host(deer_kv* kv, const deer_step_dev* dev, const void* w, const void* q_host,
-                                     const void* k_blk_host, const void* v_blk_host, const void* h_host,
-                                     const int32_t* draft_ids_host, int B, int k, int Hq, int hid, int V, float scale,
-                                     int max_seq_len, int32_t* accept_len_host, int32_t* out_ids_host, int32_t* n_out_host,
-                                     void* stream) {
-    DEER_CHECK_ARG(kv && dev && w && q_host && k_blk_host && v_blk_host && h_host && draft_ids_host && accept_len_host &&
-                       out_ids_host && n_out_host,
-                   DEER_ERR_INVALID_ARG, "deer_verify_step_host: null argument");
-    DEER_CHECK_ARG(B > 0 && k >= 1 && k <= DEER_MAX_BLOCK, DEER_ERR_UNSUPPORTED, "deer_verify_step_host: bad B or k");
+namespace {
+
+struct StepKey {
+    const void* p[16];
+    int i[8];
+    float scale;
+    int device;
+};
+
+struct StepCache {
+    StepKey key;
+    cudaGraphExec_t exec = nullptr;
+};
+
+std::mutex g_mu;
+StepCache g_cache;
+
+// A second stream for the copies that the attention does not need (hidden states, draft ids): they cross the bus
+// while the attention kernel runs.  Created on first use, one per process.
+cudaStream_t g_side = nullptr;
+cudaEvent_t g_fork = nullptr, g_join = nullptr;
+
+int side_stream() {
+    if (g_side) return DEER_OK;
+    DEER_CUDA(cudaStreamCreateWithFlags(&g_side, cudaStreamNonBlocking));
+    DEER_CUDA(cudaEventCreateWithFlags(&g_fork, cudaEventDisableTiming));
+    DEER_CUDA(cudaEventCreateWithFlags(&g_join, cudaEventDisableTiming));
+    return DEER_OK;
+}
+
+int enqueue(deer_kv* kv, const deer_step_dev* dev, const void* w, const void* q_host, const void* k_blk_host,
+            const void* v_blk_host, const void* h_host, const int32_t* draft_ids_host, int B, int k, int Hq, int hid, int V,
+            float scale, int max_seq_len, int32_t* accept_len_host, int32_t* out_ids_host, int32_t* n_out_host, void* stream,
+            bool fork) {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int Hkv = kv->d.n_kv_heads, D = kv->d.head_dim;
     const size_t M = (size_t)B * k;
+    // fork (worth its extra calls only where they are recorded once): hidden states and draft ids on the second stream
+    int rc = DEER_OK;
+    cudaStream_t sh = st;
+    if (fork) {
+        rc = side_stream();
+        if (rc != DEER_OK) return rc;
+        sh = g_side;
+        DEER_CUDA(cudaEventRecord(g_fork, st));
+        DEER_CUDA(cudaStreamWaitEvent(g_side, g_fork, 0));
+    }
+    DEER_CUDA(cudaMemcpyAsync(dev->h, h_host, M * hid * 2, cudaMemcpyHostToDevice, sh));
+    DEER_CUDA(cudaMemcpyAsync(dev->draft_ids, draft_ids_host, M * sizeof(int32_t), cudaMemcpyHostToDevice, sh));
+    if (fork) DEER_CUDA(cudaEventRecord(g_join, g_side));
     DEER_CUDA(cudaMemcpyAsync(dev->q, q_host, M * Hq * D * 2, cudaMemcpyHostToDevice, st));
     DEER_CUDA(cudaMemcpyAsync(dev->k_blk, k_blk_host, M * Hkv * D * 2, cudaMemcpyHostToDevice, st));
     DEER_CUDA(cudaMemcpyAsync(dev->v_blk, v_blk_host, M * Hkv * D * 2, cudaMemcpyHostToDevice, st));
-    DEER_CUDA(cudaMemcpyAsync(dev->h, h_host, M * hid * 2, cudaMemcpyHostToDevice, st));
-    DEER_CUDA(cudaMemcpyAsync(dev->draft_ids, draft_ids_host, M * sizeof(int32_t), cudaMemcpyHostToDevice, st));
-    int rc = deer_kv_reserve(kv, dev->seq_ids, B, k, stream);
+    rc = deer_kv_reserve(kv, dev->seq_ids, B, k, stream);
     if (rc != DEER_OK) return rc;
     rc = deer_block_attn(kv, dev->seq_ids, dev->q, dev->k_blk, dev->v_blk, dev->attn_out, B, k, Hq, DEER_MASK_CAUSAL, 1, scale,
                          max_seq_len, dev->attn_ws, dev->attn_ws_bytes, stream);
     if (rc != DEER_OK) return rc;
+    if (fork) DEER_CUDA(cudaStreamWaitEvent(st, g_join, 0));
     rc = deer_lmhead_select(dev->h, w, (int)M, hid, V, DEER_SEL_ARGMAX, 1.f, nullptr, dev->target_ids, nullptr, nullptr, nullptr,
                             nullptr, dev->lm_ws, dev->lm_ws_bytes, stream);
     if (rc != DEER_OK) return rc;
@@ -37,6 +87,81 @@ extern "C" int deer_verify_step_host(deer_kv* kv, const deer_step_dev* dev, cons
     DEER_CUDA(cudaMemcpyAsync(accept_len_host, dev->accept_len, (size_t)B * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     DEER_CUDA(cudaMemcpyAsync(out_ids_host, dev->out_ids, M * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     DEER_CUDA(cudaMemcpyAsync(n_out_host, dev->n_out, (size_t)B * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    return DEER_OK;
+}
+
+bool pinned(const void* p) {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, p) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return at.type == cudaMemoryTypeHost;
+}
+
+}  // namespace
+
+extern "C" int deer_verify_step_host(deer_kv* kv, const deer_step_dev* dev, const void* w, const void* q_host,
+                                     const void* k_blk_host, const void* v_blk_host, const void* h_host,
+                                     const int32_t* draft_ids_host, int B, int k, int Hq, int hid, int V, float scale,
+                                     int max_seq_len, int32_t* accept_len_host, int32_t* out_ids_host, int32_t* n_out_host,
+                                     void* stream) {
+    DEER_CHECK_ARG(kv && dev && w && q_host && k_blk_host && v_blk_host && h_host && draft_ids_host && accept_len_host &&
+                       out_ids_host && n_out_host,
+                   DEER_ERR_INVALID_ARG, "deer_verify_step_host: null argument");
+    DEER_CHECK_ARG(B > 0 && k >= 1 && k <= DEER_MAX_BLOCK, DEER_ERR_UNSUPPORTED, "deer_verify_step_host: bad B or k");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    const char* env = getenv("DEER_STEP_GRAPH");
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    DEER_CUDA(cudaStreamIsCapturing(st, &cap));
+    // the legacy default stream cannot be captured
+    const bool use_graph = !(env && atoi(env) == 0) && st != nullptr && cap == cudaStreamCaptureStatusNone && pinned(q_host) &&
+                           pinned(k_blk_host) && pinned(v_blk_host) && pinned(h_host) && pinned(draft_ids_host) &&
+                           pinned(accept_len_host) && pinned(out_ids_host) && pinned(n_out_host);
+    if (!use_graph) {
+        const int rc = enqueue(kv, dev, w, q_host, k_blk_host, v_blk_host, h_host, draft_ids_host, B, k, Hq, hid, V, scale,
+                               max_seq_len, accept_len_host, out_ids_host, n_out_host, stream, false);
+        if (rc != DEER_OK) return rc;
+        DEER_CUDA(cudaStreamSynchronize(st));
+        return DEER_OK;
+    }
+
+    StepKey key;
+    memset(&key, 0, sizeof(key));
+    const void* ptrs[] = {kv,          w,           q_host,       k_blk_host,   v_blk_host,    h_host,       draft_ids_host,
+                          accept_len_host, out_ids_host, n_out_host, dev->q,       dev->attn_ws,  dev->lm_ws,   kv->d.k_pool,
+                          kv->d.page_table, dev->seq_ids};
+    for (int j = 0; j < 16; ++j) key.p[j] = ptrs[j];
+    const int ints[] = {B, k, Hq, hid, V, max_seq_len, (int)dev->attn_ws_bytes, (int)dev->lm_ws_bytes};
+    for (int j = 0; j < 8; ++j) key.i[j] = ints[j];
+    key.scale = scale;
+    DEER_CUDA(cudaGetDevice(&key.device));
+
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!g_cache.exec || memcmp(&g_cache.key, &key, sizeof(key)) != 0) {
+        if (g_cache.exec) {
+            cudaGraphExecDestroy(g_cache.exec);
+            g_cache.exec = nullptr;
+        }
+        DEER_CUDA(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+        const int rc = enqueue(kv, dev, w, q_host, k_blk_host, v_blk_host, h_host, draft_ids_host, B, k, Hq, hid, V, scale,
+                               max_seq_len, accept_len_host, out_ids_host, n_out_host, stream, true);
+        cudaGraph_t graph = nullptr;
+        const cudaError_t ce = cudaStreamEndCapture(st, &graph);      // always, so that the stream leaves capture mode
+        if (rc != DEER_OK) {
+            if (graph) cudaGraphDestroy(graph);
+            cudaGetLastError();
+            return rc;
+        }
+        DEER_CUDA(ce);
+        const cudaError_t ci = cudaGraphInstantiate(&g_cache.exec, graph, 0);
+        cudaGraphDestroy(graph);
+        if (ci != cudaSuccess) g_cache.exec = nullptr;
+        DEER_CUDA(ci);
+        g_cache.key = key;
+    }
+    DEER_CUDA(cudaGraphLaunch(g_cache.exec, st));
     DEER_CUDA(cudaStreamSynchronize(st));
     return DEER_OK;
 }

@@ -172,3 +172,54 @@ def test_c5_sweep_points(B, ctx, k, mask):
         Hn.check_ids(vs.target_ids.cpu().numpy(), O.select_argmax(z), z, cfg.name)
     else:
         _greedy_step(cfg, stress=True, steps=3)
+
+
+@pytest.mark.parametrize("own_stream", [False, True])
+def test_host_buffer_step_matches_oracle(own_stream):
+    """deer_verify_step_host, four consecutive steps from pinned host buffers that are refilled in place: on the legacy
+    default stream every call enqueues its copies and kernels one by one; on a stream of its own the first call
+    captures them into a graph and the later ones replay it.  Verdicts and cache state against the oracle."""
+    from paper_2512_15176_b200 import binding as L
+    from paper_2512_15176_b200.runner import VerifyStep
+    steps = 4
+    cfg = W.config(0).with_(growth=steps * W.config(0).k)
+    st = Hn.draw_state(cfg, None, True)
+    okv, kv = Hn.oracle_kv(st), Hn.gpu_kv(st)
+    w = W.lm_head(cfg)
+    w64 = Hn.f64(w)
+    w_dev = w.cuda()
+    vs = VerifyStep(cfg, kv, w_dev, int(st.lengths.max()) + steps * cfg.k, store_logits=False)
+    ids = np.arange(cfg.B)
+    pin = lambda t: t.contiguous().pin_memory()
+    q0, kb0, vb0 = Hn.draw_block(cfg, 0, True)
+    hq, hkb, hvb = pin(q0), pin(kb0), pin(vb0)
+    hh = pin(torch.empty(cfg.M, cfg.hid, dtype=torch.bfloat16))
+    hd = pin(torch.empty(cfg.B, cfg.k, dtype=torch.int32))
+    ha = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
+    ho = torch.empty(cfg.B, cfg.k, dtype=torch.int32).pin_memory()
+    hn = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
+    sd = L.deer_step_dev(vs.q.data_ptr(), vs.k_blk.data_ptr(), vs.v_blk.data_ptr(), vs.attn_out.data_ptr(), vs.h.data_ptr(),
+                         vs.seq_ids.data_ptr(), vs.draft_ids.data_ptr(), vs.target_ids.data_ptr(), vs.accept_len.data_ptr(),
+                         vs.out_ids.data_ptr(), vs.n_out.data_ptr(), vs.attn_ws.data_ptr(), vs.attn_ws.numel(),
+                         vs.lm_ws.data_ptr(), vs.lm_ws.numel())
+    stream = torch.cuda.Stream() if own_stream else None
+    torch.cuda.synchronize()
+    for step in range(steps):
+        q, kb, vb = Hn.draw_block(cfg, step, True)
+        h, z, _ = Hn.draw_hidden_with_margin(cfg, w64, step)
+        target = O.select_argmax(z).reshape(cfg.B, cfg.k)
+        drafts = W.plant_drafts(cfg, target, W.planted_prefix_lengths(cfg, step), step)
+        for dst, src in ((hq, q), (hkb, kb), (hvb, vb), (hh, h), (hd, torch.from_numpy(drafts))):
+            dst.copy_(src.reshape(dst.shape))
+        assert okv.reserve(ids, cfg.k)
+        okv.append(ids, Hn.f64(kb).astype(np.float32), Hn.f64(vb).astype(np.float32))
+        a, out, n = O.accept_greedy(drafts, target)
+        okv.commit(ids, a)
+        L.deer_verify_step_host(kv, sd, w_dev, hq, hkb, hvb, hh, hd, cfg.B, cfg.k, cfg.Hq, cfg.hid, cfg.V, vs.scale,
+                                int(st.lengths.max()) + steps * cfg.k, ha, ho, hn, stream=stream)
+        np.testing.assert_array_equal(ha.numpy(), a)
+        np.testing.assert_array_equal(ho.numpy(), out)
+        np.testing.assert_array_equal(hn.numpy(), n)
+        assert L.deer_kv_status(kv) == 0
+        Hn.kv_state_equal(kv, okv, f"host step {step}")
+    Hn.kv_contents_equal(kv, okv, label="host steps")
