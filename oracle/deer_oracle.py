@@ -344,3 +344,45 @@ class DecodeState:
             if hit_eos or self.n_tokens[b] >= self.max_new:
                 self.finished[b] = 1
         return keep
+
+
+# --------------------------------------------------------------------------
+# (6) The rest of a verifier layer around the block attention.  The paper takes
+#     its verifiers (Qwen3) as given; this is the public pre-norm decoder layer of
+#     that family written out: RMSNorm, Q/K/V projections, a per-head RMSNorm of
+#     q and k, rotary position embedding (half-split pairing), attention, output
+#     projection, residual; RMSNorm, gate/up projections, SiLU(gate) * up, down
+#     projection, residual.  All in float64; the caller rounds where the device
+#     stores bf16.
+# --------------------------------------------------------------------------
+
+def linear(x, w):
+    """y[m][n] = sum_c x[m][c] * w[n][c]  (weights stored [out][in])."""
+    return np.asarray(x, dtype=np.float64) @ np.asarray(w, dtype=np.float64).T
+
+
+def rmsnorm(x, gamma, eps):
+    """y = x / sqrt(mean(x^2) + eps) * gamma over the last axis."""
+    x = np.asarray(x, dtype=np.float64)
+    ms = (x * x).mean(axis=-1, keepdims=True)
+    return x / np.sqrt(ms + eps) * np.asarray(gamma, dtype=np.float64)
+
+
+def rope(x, positions, theta):
+    """Rotary embedding of x [..., T, H, D] at integer positions [..., T]: dimension
+    d < D/2 is paired with d + D/2 and the pair is rotated by the angle
+    pos * theta^(-2d / D)."""
+    x = np.asarray(x, dtype=np.float64)
+    D = x.shape[-1]
+    half = D // 2
+    inv_freq = float(theta) ** (-np.arange(half, dtype=np.float64) * 2.0 / D)
+    ang = np.asarray(positions, dtype=np.float64)[..., None, None] * inv_freq          # [..., T, 1, half]
+    c, s = np.cos(ang), np.sin(ang)
+    a, b = x[..., :half], x[..., half:]
+    return np.concatenate([a * c - b * s, b * c + a * s], axis=-1)
+
+
+def swiglu(gate, up):
+    """SiLU(gate) * up with SiLU(g) = g / (1 + exp(-g))."""
+    g = np.asarray(gate, dtype=np.float64)
+    return g / (1.0 + np.exp(-g)) * np.asarray(up, dtype=np.float64)
