@@ -271,6 +271,32 @@ int deer_emit(int B, int k, const int32_t* accept_len, const int32_t* out_ids, c
               int32_t* keep, int flags, void* stream);
 
 /* ------------------------------------------------------------------------
+ * (6) The rest of a verifier layer around the block attention.  The paper takes
+ * its verifiers (the Qwen3 family) as given; these are that family's public
+ * pre-norm decoder layer, at the M = B k rows of a draft block.  bf16 in and
+ * out, fp32 arithmetic, all stream-ordered.
+ *
+ * deer_linear: y[m][n] = sum_c x[m][c] w[n][c] (+ residual[m][n]), the Q/K/V,
+ *   output, gate/up and down projections.  x bf16 [M][K], w bf16 [N][K],
+ *   residual bf16 [M][N] or NULL, y bf16 [M][N]; K a multiple of 64, N >= 16.
+ *   The LM-head kernels without their selection: weight-streaming for small M.
+ * deer_rmsnorm: y = x / sqrt(mean(x^2) + eps) * gamma over each row of
+ *   x bf16 [M][hid]; gamma bf16 [hid].
+ * deer_qk_norm_rope: in place on q bf16 [B][k][Hq][D] and k_blk bf16
+ *   [B][k][Hkv][D]: if q_gamma / k_gamma (bf16 [D]) are given, RMSNorm over each
+ *   head's D values first; then the rotary embedding at position
+ *   seq_len[seq_ids[b]] + i: dimension d < D/2 pairs with d + D/2, the pair
+ *   turns by position * theta^(-2d/D).
+ * deer_swiglu: y[m][c] = silu(gate_up[m][c]) * gate_up[m][I + c];
+ *   gate_up bf16 [M][2 I], y bf16 [M][I].
+ * ---------------------------------------------------------------------- */
+int deer_linear(const void* x, const void* w, const void* residual, void* y, int M, int K, int N, void* stream);
+int deer_rmsnorm(const void* x, const void* gamma, void* y, int M, int hid, float eps, void* stream);
+int deer_qk_norm_rope(deer_kv* kv, const int32_t* seq_ids, void* q, void* k_blk, const void* q_gamma,
+                      const void* k_gamma, int B, int k, int Hq, float eps, float theta, void* stream);
+int deer_swiglu(const void* gate_up, void* y, int M, int I, void* stream);
+
+/* ------------------------------------------------------------------------
  * One whole greedy verify step with HOST inputs and outputs (Algorithm 1, one
  * iteration of the while loop on the verifier side): copies the block's
  * q/k_blk/v_blk, hidden states and draft ids from host memory to the device

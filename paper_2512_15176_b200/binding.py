@@ -27,6 +27,7 @@ EXPORTS = [
     "deer_block_attn_workspace_bytes", "deer_block_attn", "deer_lmhead_workspace_bytes", "deer_lmhead_select",
     "deer_accept_workspace_bytes", "deer_accept", "deer_verify_step_host",
     "deer_lmhead_static_max_rows", "deer_lmhead_select_static", "deer_emit", "deer_draft_stats",
+    "deer_linear", "deer_rmsnorm", "deer_qk_norm_rope", "deer_swiglu",
 ]
 
 
@@ -86,6 +87,11 @@ def lib() -> ctypes.CDLL:
     L.deer_accept.argtypes = [c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_float,
                               c_void_p, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t,
                               c_void_p]
+    L.deer_linear.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p]
+    L.deer_rmsnorm.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int, c_float, c_void_p]
+    L.deer_qk_norm_rope.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_float,
+                                    c_float, c_void_p]
+    L.deer_swiglu.argtypes = [c_void_p, c_void_p, c_int, c_int, c_void_p]
     L.deer_draft_stats.argtypes = [c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
     L.deer_emit.argtypes = [c_int, c_int, c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p,
                             c_int, c_void_p]
@@ -228,6 +234,28 @@ def deer_accept(mode, B, k, V, draft_ids, target_ids, target_logits, target_lse,
                              _ptr(accept_len), _ptr(out_ids), _ptr(n_out), _ptr(workspace),
                              workspace.numel() * workspace.element_size() if workspace is not None else 0,
                              _stream(stream)))
+
+
+def deer_linear(x, w, y, residual=None, stream=None):
+    M, K = x.shape
+    N = w.shape[0]
+    _check(lib().deer_linear(_ptr(x), _ptr(w), _ptr(residual), _ptr(y), M, K, N, _stream(stream)))
+
+
+def deer_rmsnorm(x, gamma, y, eps, stream=None):
+    M, hid = x.shape
+    _check(lib().deer_rmsnorm(_ptr(x), _ptr(gamma), _ptr(y), M, hid, float(eps), _stream(stream)))
+
+
+def deer_qk_norm_rope(kv: "KVCache", seq_ids, q, k_blk, q_gamma, k_gamma, eps, theta, stream=None):
+    B, k, Hq, _ = q.shape
+    _check(lib().deer_qk_norm_rope(kv.handle, _ptr(seq_ids), _ptr(q), _ptr(k_blk), _ptr(q_gamma), _ptr(k_gamma), B, k, Hq,
+                                   float(eps), float(theta), _stream(stream)))
+
+
+def deer_swiglu(gate_up, y, stream=None):
+    M, I = y.shape
+    _check(lib().deer_swiglu(_ptr(gate_up), _ptr(y), M, I, _stream(stream)))
 
 
 def deer_draft_stats(B, k, V, draft_ids, draft_logits, workspace, stream=None):

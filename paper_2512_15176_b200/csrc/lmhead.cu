@@ -123,6 +123,8 @@ extern "C" int deer_lmhead_select(const void* h, const void* w, int M, int hid, 
     p.draft_ids = (mode == DEER_SEL_SOFTMAX) ? draft_ids : nullptr;
     p.out_draft_logit = (mode == DEER_SEL_SOFTMAX) ? out_draft_logit : nullptr;
     p.out_logits = out_logits;
+    p.out_bf16 = nullptr;
+    p.residual = nullptr;
     p.part = static_cast<Partial*>(workspace);
     p.nparts = pl.nparts;
     // DEER_LMHEAD_IMPL=mma forces the warp-level kernel, =single the one-block tcgen05 kernel at every M
@@ -150,4 +152,36 @@ extern "C" int deer_lmhead_select(const void* h, const void* w, int M, int hid, 
     lmhead_finalize_kernel<<<(M + 7) / 8, 256, 0, st>>>(fa);
     DEER_CUDA(cudaGetLastError());
     return DEER_OK;
+}
+
+// ------------------------------------------------------------------------------
+// A plain linear layer on the same kernels: y = x w^T (+ residual) in bf16.  The
+// projections around the block attention in a verifier layer (Q/K/V, output,
+// gate/up, down) are this at M = B k rows: weight-streaming at small M,
+// tensor-bound above ~200 rows, exactly like the LM head without its selection.
+extern "C" int deer_linear(const void* x, const void* w, const void* residual, void* y, int M, int K, int N, void* stream) {
+    using namespace lmhead;
+    DEER_CHECK_ARG(x && w && y, DEER_ERR_INVALID_ARG, "deer_linear: null argument");
+    DEER_CHECK_ARG(deer_aligned16(x) && deer_aligned16(w) && deer_aligned16(y) && deer_aligned16(residual), DEER_ERR_INVALID_ARG,
+                   "deer_linear: pointers must be 16-byte aligned");
+    DEER_CHECK_ARG(M >= 0 && N > 0 && K > 0, DEER_ERR_INVALID_ARG, "deer_linear: bad sizes");
+    DEER_CHECK_ARG(umma_supported(M > 0 ? M : 1, K, N), DEER_ERR_UNSUPPORTED,
+                   "deer_linear: K must be a multiple of 64 and N at least 16");
+    if (M == 0) return DEER_OK;
+    Params p;
+    p.h = static_cast<const __nv_bfloat16*>(x);
+    p.w = static_cast<const __nv_bfloat16*>(w);
+    p.M = M;
+    p.hid = K;
+    p.V = N;
+    p.inv_t_log2 = LOG2E;
+    p.draft_ids = nullptr;
+    p.out_draft_logit = nullptr;
+    p.out_logits = nullptr;
+    p.out_bf16 = static_cast<__nv_bfloat16*>(y);
+    p.residual = static_cast<const __nv_bfloat16*>(residual);
+    p.part = nullptr;
+    p.nparts = 0;
+    int nparts = 0;
+    return launch_umma(p, 0, true, &nparts, static_cast<cudaStream_t>(stream));
 }

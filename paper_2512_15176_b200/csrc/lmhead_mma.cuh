@@ -32,6 +32,8 @@ struct Params {
     const int32_t* draft_ids;    // [M] or null
     float* out_draft_logit;      // [M] or null
     float* out_logits;           // [M][V] or null
+    __nv_bfloat16* out_bf16;     // [M][V] or null: plain linear layer, y = h w^T (+ residual), nothing selected
+    const __nv_bfloat16* residual;   // [M][V] or null, added before the bf16 rounding
     Partial* part;               // [nparts][M]
     int nparts;
 };

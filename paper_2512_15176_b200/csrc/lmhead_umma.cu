@@ -54,6 +54,8 @@ struct Args {
     const int32_t* draft_ids;
     float* out_draft_logit;
     float* out_logits;
+    __nv_bfloat16* out_bf16; // linear-layer mode: the product (+ residual) in bf16 is all that is written
+    const __nv_bfloat16* residual;
     Partial* part;           // [nparts][M]
 };
 
@@ -63,6 +65,34 @@ __device__ __forceinline__ void consume16(const uint32_t (&r)[16], int vbase, in
     if (!row_ok || vbase >= V) return;
     const int nv = min(16, V - vbase);
     float v[16];
+    if (a.out_bf16) {
+        // linear layer: y = acc (+ residual), rounded to bf16; 16 columns = 32 contiguous bytes of the row
+        __nv_bfloat16* dst = a.out_bf16 + zrow + vbase;
+        const __nv_bfloat16* res = a.residual ? a.residual + zrow + vbase : nullptr;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
+        if (nv == 16 && ((zrow + vbase) & 7) == 0) {
+            if (res) {
+                const uint4 r0 = *reinterpret_cast<const uint4*>(res), r1 = *reinterpret_cast<const uint4*>(res + 8);
+                const uint32_t rw[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    v[2 * j] += __uint_as_float(rw[j] << 16);
+                    v[2 * j + 1] += __uint_as_float(rw[j] & 0xffff0000u);
+                }
+            }
+            uint4 o0, o1;
+            o0.x = pack_bf16(v[0], v[1]);  o0.y = pack_bf16(v[2], v[3]);   o0.z = pack_bf16(v[4], v[5]);   o0.w = pack_bf16(v[6], v[7]);
+            o1.x = pack_bf16(v[8], v[9]);  o1.y = pack_bf16(v[10], v[11]); o1.z = pack_bf16(v[12], v[13]); o1.w = pack_bf16(v[14], v[15]);
+            *reinterpret_cast<uint4*>(dst) = o0;
+            *reinterpret_cast<uint4*>(dst + 8) = o1;
+        } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if (j < nv) dst[j] = __float2bfloat16(v[j] + (res ? __bfloat162float(res[j]) : 0.f));
+        }
+        return;
+    }
 #pragma unroll
     for (int j = 0; j < 16; ++j) v[j] = (j < nv) ? __uint_as_float(r[j]) : -INFINITY;
     if (store) {
@@ -197,7 +227,7 @@ __device__ __forceinline__ void epilogue(const Args& a, const CUtensorMap* tm_z,
         }
     }
     if (lane == 0) bulk_wait<0>();               // the staging area outlives every store that reads it
-    if (row_ok) {
+    if (row_ok && !a.out_bf16) {
         Partial pr;
         pr.m = run_m;
         pr.idx = run_i;
@@ -506,6 +536,8 @@ int launch_umma(const Params& p, int need_sum, bool allow_pair, int* nparts_out,
     a.draft_ids = p.draft_ids;
     a.out_draft_logit = p.out_draft_logit;
     a.out_logits = p.out_logits;
+    a.out_bf16 = p.out_bf16;
+    a.residual = p.residual;
     a.part = p.part;
     CUtensorMap tm_h, tm_w_hi, tm_w_lo;
     int rc = make_operand_map(&tm_h, p.h, (uint64_t)p.M, (uint64_t)p.hid, (uint32_t)a.h_box_rows);

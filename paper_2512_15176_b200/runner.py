@@ -174,3 +174,45 @@ class DecodeLoop:
         L.deer_emit(vs.accept_len, vs.out_ids, vs.n_out, self.eos_id, self.tokens, self.n_tokens, self.finished, self.keep,
                     L.DEER_EMIT_PENDING if self.pending else 0)
         L.deer_kv_commit(vs.kv, vs.seq_ids, self.keep, vs.cfg.k)
+
+
+class VerifierLayer:
+    """One pre-norm decoder layer of a Qwen3-style verifier at the M = B k rows of a
+    draft block, on the library's calls: RMSNorm -> Q/K/V projections -> per-head
+    RMSNorm of q, k + rotary embedding -> block attention against the paged cache
+    (the block's K/V rows are appended) -> output projection + residual -> RMSNorm
+    -> gate/up projection -> SiLU(gate) * up -> down projection + residual.
+    Weights are [out][in] bf16 tensors on the device; every intermediate stays
+    there (attributes, so that a test can look at each stage)."""
+
+    def __init__(self, cfg: StepConfig, kv: L.KVCache, weights: dict, max_seq_len: int, inter: int, eps=1e-6,
+                 theta=1.0e6, device="cuda"):
+        self.cfg, self.kv, self.w, self.max_seq_len = cfg, kv, weights, int(max_seq_len)
+        self.inter, self.eps, self.theta = int(inter), float(eps), float(theta)
+        B, k, Hq, Hkv, D, M, hid = cfg.B, cfg.k, cfg.Hq, cfg.Hkv, cfg.D, cfg.M, cfg.hid
+        bf = torch.bfloat16
+        e = lambda *shape: torch.empty(*shape, dtype=bf, device=device)
+        self.seq_ids = torch.arange(B, dtype=torch.int32, device=device)
+        self.xn, self.q, self.k_blk, self.v_blk = e(M, hid), e(B, k, Hq, D), e(B, k, Hkv, D), e(B, k, Hkv, D)
+        self.attn_out, self.x1, self.xn2 = e(B, k, Hq, D), e(M, hid), e(M, hid)
+        self.gu, self.act, self.x2 = e(M, 2 * self.inter), e(M, self.inter), e(M, hid)
+        self.attn_ws = _ws(L.deer_block_attn_workspace_bytes(B, k, Hq, Hkv, D, self.max_seq_len), device)
+        self.scale = 1.0 / math.sqrt(D)
+
+    def forward(self, x: torch.Tensor) -> torch.Tensor:
+        c, w = self.cfg, self.w
+        M = c.M
+        L.deer_rmsnorm(x, w["ln1"], self.xn, self.eps)
+        L.deer_linear(self.xn, w["wq"], self.q.view(M, -1))
+        L.deer_linear(self.xn, w["wk"], self.k_blk.view(M, -1))
+        L.deer_linear(self.xn, w["wv"], self.v_blk.view(M, -1))
+        L.deer_qk_norm_rope(self.kv, self.seq_ids, self.q, self.k_blk, w.get("q_norm"), w.get("k_norm"), self.eps, self.theta)
+        L.deer_kv_reserve(self.kv, self.seq_ids, c.k)
+        L.deer_block_attn(self.kv, self.seq_ids, self.q, self.k_blk, self.v_blk, self.attn_out, L.DEER_MASK_CAUSAL, True,
+                          self.scale, self.max_seq_len, self.attn_ws)
+        L.deer_linear(self.attn_out.view(M, -1), w["wo"], self.x1, residual=x)
+        L.deer_rmsnorm(self.x1, w["ln2"], self.xn2, self.eps)
+        L.deer_linear(self.xn2, w["wgu"], self.gu)
+        L.deer_swiglu(self.gu, self.act)
+        L.deer_linear(self.act, w["wd"], self.x2, residual=self.x1)
+        return self.x2
