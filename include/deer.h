@@ -280,6 +280,10 @@ int deer_emit(int B, int k, const int32_t* accept_len, const int32_t* out_ids, c
  *   output, gate/up and down projections.  x bf16 [M][K], w bf16 [N][K],
  *   residual bf16 [M][N] or NULL, y bf16 [M][N]; K a multiple of 64, N >= 16.
  *   The LM-head kernels without their selection: weight-streaming for small M.
+ *   With a workspace of deer_linear_workspace_bytes (may be NULL / 0: slower for
+ *   few output columns) the contraction is cut into ranges whose fp32 partial
+ *   products are summed by a second kernel, so that every SM streams weights
+ *   even when N is only a few thousand.
  * deer_rmsnorm: y = x / sqrt(mean(x^2) + eps) * gamma over each row of
  *   x bf16 [M][hid]; gamma bf16 [hid].
  * deer_qk_norm_rope: in place on q bf16 [B][k][Hq][D] and k_blk bf16
@@ -290,7 +294,9 @@ int deer_emit(int B, int k, const int32_t* accept_len, const int32_t* out_ids, c
  * deer_swiglu: y[m][c] = silu(gate_up[m][c]) * gate_up[m][I + c];
  *   gate_up bf16 [M][2 I], y bf16 [M][I].
  * ---------------------------------------------------------------------- */
-int deer_linear(const void* x, const void* w, const void* residual, void* y, int M, int K, int N, void* stream);
+size_t deer_linear_workspace_bytes(int M, int K, int N);
+int deer_linear(const void* x, const void* w, const void* residual, void* y, int M, int K, int N,
+                void* workspace, size_t workspace_bytes, void* stream);
 int deer_rmsnorm(const void* x, const void* gamma, void* y, int M, int hid, float eps, void* stream);
 int deer_qk_norm_rope(deer_kv* kv, const int32_t* seq_ids, void* q, void* k_blk, const void* q_gamma,
                       const void* k_gamma, int B, int k, int Hq, float eps, float theta, void* stream);

@@ -27,7 +27,7 @@ EXPORTS = [
     "deer_block_attn_workspace_bytes", "deer_block_attn", "deer_lmhead_workspace_bytes", "deer_lmhead_select",
     "deer_accept_workspace_bytes", "deer_accept", "deer_verify_step_host",
     "deer_lmhead_static_max_rows", "deer_lmhead_select_static", "deer_emit", "deer_draft_stats",
-    "deer_linear", "deer_rmsnorm", "deer_qk_norm_rope", "deer_swiglu",
+    "deer_linear_workspace_bytes", "deer_linear", "deer_rmsnorm", "deer_qk_norm_rope", "deer_swiglu",
 ]
 
 
@@ -87,7 +87,9 @@ def lib() -> ctypes.CDLL:
     L.deer_accept.argtypes = [c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_float,
                               c_void_p, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t,
                               c_void_p]
-    L.deer_linear.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p]
+    L.deer_linear_workspace_bytes.restype = c_size_t
+    L.deer_linear_workspace_bytes.argtypes = [c_int] * 3
+    L.deer_linear.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_size_t, c_void_p]
     L.deer_rmsnorm.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int, c_float, c_void_p]
     L.deer_qk_norm_rope.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_float,
                                     c_float, c_void_p]
@@ -236,10 +238,15 @@ def deer_accept(mode, B, k, V, draft_ids, target_ids, target_logits, target_lse,
                              _stream(stream)))
 
 
-def deer_linear(x, w, y, residual=None, stream=None):
+def deer_linear_workspace_bytes(M, K, N) -> int:
+    return lib().deer_linear_workspace_bytes(M, K, N)
+
+
+def deer_linear(x, w, y, residual=None, workspace=None, stream=None):
     M, K = x.shape
     N = w.shape[0]
-    _check(lib().deer_linear(_ptr(x), _ptr(w), _ptr(residual), _ptr(y), M, K, N, _stream(stream)))
+    _check(lib().deer_linear(_ptr(x), _ptr(w), _ptr(residual), _ptr(y), M, K, N, _ptr(workspace),
+                             workspace.numel() * workspace.element_size() if workspace is not None else 0, _stream(stream)))
 
 
 def deer_rmsnorm(x, gamma, y, eps, stream=None):

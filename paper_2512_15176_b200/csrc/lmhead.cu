@@ -11,7 +11,7 @@
 namespace lmhead {
 
 bool umma_supported(int M, int hid, int V);
-int launch_umma(const Params& p, int need_sum, bool allow_pair, int* nparts_out, cudaStream_t st);
+int launch_umma(const Params& p, int need_sum, bool allow_pair, int* nparts_out, cudaStream_t st, int* ksplit_out = nullptr);
 
 struct FinalizeArgs {
     const Partial* part;
@@ -125,6 +125,8 @@ extern "C" int deer_lmhead_select(const void* h, const void* w, int M, int hid, 
     p.out_logits = out_logits;
     p.out_bf16 = nullptr;
     p.residual = nullptr;
+    p.lin_part = nullptr;
+    p.max_ksplit = 1;
     p.part = static_cast<Partial*>(workspace);
     p.nparts = pl.nparts;
     // DEER_LMHEAD_IMPL=mma forces the warp-level kernel, =single the one-block tcgen05 kernel at every M
@@ -159,15 +161,60 @@ extern "C" int deer_lmhead_select(const void* h, const void* w, int M, int hid, 
 // projections around the block attention in a verifier layer (Q/K/V, output,
 // gate/up, down) are this at M = B k rows: weight-streaming at small M,
 // tensor-bound above ~200 rows, exactly like the LM head without its selection.
-extern "C" int deer_linear(const void* x, const void* w, const void* residual, void* y, int M, int K, int N, void* stream) {
+// With few output columns (N up to ~19 000 at M <= 128) the blocks take full
+// 256-column tiles and a range of the contraction each; their fp32 partial
+// products land in the workspace and a second kernel adds them up.
+namespace {
+
+constexpr int LIN_MAX_KSPLIT = 16;
+
+__global__ void __launch_bounds__(256) linear_reduce_kernel(const float* __restrict__ part, int ksplit, long long total,
+                                                            const __nv_bfloat16* __restrict__ residual,
+                                                            __nv_bfloat16* __restrict__ y) {
+    const long long i = ((long long)blockIdx.x * 256 + threadIdx.x) * 2;
+    if (i >= total) return;
+    float s0 = 0.f, s1 = 0.f;
+    if (i + 1 < total && (total & 1) == 0) {
+        for (int s = 0; s < ksplit; ++s) {
+            const float2 v = *reinterpret_cast<const float2*>(part + (size_t)s * total + i);
+            s0 += v.x;
+            s1 += v.y;
+        }
+        if (residual) {
+            s0 += __bfloat162float(residual[i]);
+            s1 += __bfloat162float(residual[i + 1]);
+        }
+        *reinterpret_cast<uint32_t*>(y + i) = pack_bf16(s0, s1);
+    } else {
+        for (long long j = i; j < total && j < i + 2; ++j) {
+            float t = 0.f;
+            for (int s = 0; s < ksplit; ++s) t += part[(size_t)s * total + j];
+            if (residual) t += __bfloat162float(residual[j]);
+            y[j] = __float2bfloat16(t);
+        }
+    }
+}
+
+}  // namespace
+
+extern "C" size_t deer_linear_workspace_bytes(int M, int K, int N) {
+    (void)K;
+    if (M <= 0 || N <= 0 || M > 128) return 0;            // larger M never cuts the contraction
+    return (size_t)LIN_MAX_KSPLIT * M * N * sizeof(float);
+}
+
+extern "C" int deer_linear(const void* x, const void* w, const void* residual, void* y, int M, int K, int N, void* workspace,
+                           size_t workspace_bytes, void* stream) {
     using namespace lmhead;
     DEER_CHECK_ARG(x && w && y, DEER_ERR_INVALID_ARG, "deer_linear: null argument");
-    DEER_CHECK_ARG(deer_aligned16(x) && deer_aligned16(w) && deer_aligned16(y) && deer_aligned16(residual), DEER_ERR_INVALID_ARG,
-                   "deer_linear: pointers must be 16-byte aligned");
+    DEER_CHECK_ARG(deer_aligned16(x) && deer_aligned16(w) && deer_aligned16(y) && deer_aligned16(residual) &&
+                       deer_aligned16(workspace),
+                   DEER_ERR_INVALID_ARG, "deer_linear: pointers must be 16-byte aligned");
     DEER_CHECK_ARG(M >= 0 && N > 0 && K > 0, DEER_ERR_INVALID_ARG, "deer_linear: bad sizes");
     DEER_CHECK_ARG(umma_supported(M > 0 ? M : 1, K, N), DEER_ERR_UNSUPPORTED,
                    "deer_linear: K must be a multiple of 64 and N at least 16");
     if (M == 0) return DEER_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
     Params p;
     p.h = static_cast<const __nv_bfloat16*>(x);
     p.w = static_cast<const __nv_bfloat16*>(w);
@@ -180,8 +227,23 @@ extern "C" int deer_linear(const void* x, const void* w, const void* residual, v
     p.out_logits = nullptr;
     p.out_bf16 = static_cast<__nv_bfloat16*>(y);
     p.residual = static_cast<const __nv_bfloat16*>(residual);
+    // the contraction is cut only as far as the caller's workspace holds the partial products (none: never)
+    p.lin_part = static_cast<float*>(workspace);
+    p.max_ksplit = workspace ? (int)(workspace_bytes / ((size_t)M * N * sizeof(float))) : 1;
+    if (p.max_ksplit > LIN_MAX_KSPLIT) p.max_ksplit = LIN_MAX_KSPLIT;
+    if (p.max_ksplit < 2) {
+        p.lin_part = nullptr;
+        p.max_ksplit = 1;
+    }
     p.part = nullptr;
     p.nparts = 0;
-    int nparts = 0;
-    return launch_umma(p, 0, true, &nparts, static_cast<cudaStream_t>(stream));
+    int nparts = 0, ksplit = 1;
+    const int rc = launch_umma(p, 0, true, &nparts, st, &ksplit);
+    if (rc != DEER_OK) return rc;
+    if (ksplit > 1) {
+        const long long total = (long long)M * N;
+        linear_reduce_kernel<<<(unsigned)((total / 2 + 256) / 256), 256, 0, st>>>(p.lin_part, ksplit, total, p.residual, p.out_bf16);
+        DEER_CUDA(cudaGetLastError());
+    }
+    return DEER_OK;
 }

@@ -56,6 +56,8 @@ struct Args {
     float* out_logits;
     __nv_bfloat16* out_bf16; // linear-layer mode: the product (+ residual) in bf16 is all that is written
     const __nv_bfloat16* residual;
+    int ksplit;              // linear-layer mode, few output columns: the contraction is cut into ksplit ranges, one per
+    float* lin_part;         // blockIdx.y / nparts; the partial sums go to lin_part[ksplit][M][V] (fp32) and are added up after
     Partial* part;           // [nparts][M]
 };
 
@@ -65,6 +67,21 @@ __device__ __forceinline__ void consume16(const uint32_t (&r)[16], int vbase, in
     if (!row_ok || vbase >= V) return;
     const int nv = min(16, V - vbase);
     float v[16];
+    if (a.out_bf16 && a.ksplit > 1) {
+        // partial sum over this block's range of the contraction: plain fp32 stores of the rows that exist
+        float* dst = a.lin_part + ((size_t)(blockIdx.y / a.nparts) * a.M * a.V) + zrow + vbase;
+        if (nv == 16 && ((zrow + vbase) & 3) == 0) {
+#pragma unroll
+            for (int j = 0; j < 16; j += 4)
+                *reinterpret_cast<float4*>(dst + j) = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
+                                                                  __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+        } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if (j < nv) dst[j] = __uint_as_float(r[j]);
+        }
+        return;
+    }
     if (a.out_bf16) {
         // linear layer: y = acc (+ residual), rounded to bf16; 16 columns = 32 contiguous bytes of the row
         __nv_bfloat16* dst = a.out_bf16 + zrow + vbase;
@@ -252,10 +269,12 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int m0 = blockIdx.x * BM;
-    const int part = blockIdx.y;
+    const int part = blockIdx.y % a.nparts;        // vocabulary (output-column) part
+    const int ks = blockIdx.y / a.nparts;          // range of the contraction (linear layers with few columns only)
     const Tiles tl = block_tiles(a, part);
     const int n_tiles = tl.n;
-    const int KB = a.hid / BK;
+    const int KBall = a.hid / BK;
+    const int kb0 = (int)((long)ks * KBall / a.ksplit), KB = (int)((long)(ks + 1) * KBall / a.ksplit) - kb0;
 
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t bar_base = smem_u32(bars);
@@ -304,8 +323,8 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
                     mbar_expect_tx(full_bar(s), stage_tx);
                     const uint32_t sa = smem_base + s * stage_bytes;
-                    tma_load_2d(sa + a.a_bytes, tm_w, kb * BK, row0, full_bar(s));     // the whole N-row tile in one box
-                    tma_load_2d(sa, &tm_h, kb * BK, m0, full_bar(s));
+                    tma_load_2d(sa + a.a_bytes, tm_w, (kb0 + kb) * BK, row0, full_bar(s));     // the whole N-row tile in one box
+                    tma_load_2d(sa, &tm_h, (kb0 + kb) * BK, m0, full_bar(s));
                 }
             }
         }
@@ -381,10 +400,12 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
     const uint32_t rank = cluster_ctarank();
     const bool leader = (rank == 0);
     const int m0 = (int)(blockIdx.x >> 1) * (2 * BM) + (int)rank * BM;
-    const int part = blockIdx.y;
+    const int part = blockIdx.y % a.nparts;        // vocabulary (output-column) part
+    const int ks = blockIdx.y / a.nparts;          // range of the contraction (linear layers with few columns only)
     const Tiles tl = block_tiles(a, part);
     const int n_tiles = tl.n;
-    const int KB = a.hid / BK;
+    const int KBall = a.hid / BK;
+    const int kb0 = (int)((long)ks * KBall / a.ksplit), KB = (int)((long)(ks + 1) * KBall / a.ksplit) - kb0;
 
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t bar_base = smem_u32(bars);
@@ -431,8 +452,8 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
                     if (leader) mbar_expect_tx(full_bar(s), stage_tx);
                     const uint32_t lead_full = map_to_cta(full_bar(s), 0);
                     const uint32_t sa = smem_base + s * stage_bytes;
-                    tma_load_2d_pair(sa + A_SPAN, tm_w, kb * BK, row0, lead_full);
-                    tma_load_2d_pair(sa, &tm_h, kb * BK, m0, lead_full);
+                    tma_load_2d_pair(sa + A_SPAN, tm_w, (kb0 + kb) * BK, row0, lead_full);
+                    tma_load_2d_pair(sa, &tm_h, (kb0 + kb) * BK, m0, lead_full);
                 }
             }
         }
@@ -501,7 +522,7 @@ bool umma_supported(int M, int hid, int V) { return M > 0 && hid % umma::BK == 0
 
 // Launches the tcgen05 kernel; the partials it writes are merged by lmhead_finalize_kernel.
 // *nparts_out receives the number of vocabulary parts written.
-int launch_umma(const Params& p, int need_sum, bool allow_pair, int* nparts_out, cudaStream_t st) {
+int launch_umma(const Params& p, int need_sum, bool allow_pair, int* nparts_out, cudaStream_t st, int* ksplit_out) {
     using namespace umma;
     // more than 128 block rows: pairs of blocks share the weight tiles (256 rows per pair)
     const bool pair = allow_pair && p.M > BM;
@@ -510,6 +531,18 @@ int launch_umma(const Params& p, int need_sum, bool allow_pair, int* nparts_out,
     if (nparts < 1) nparts = 1;
     const int gran = (p.V + 15) / 16;                    // 16-row granules of the vocabulary
     if (nparts > gran) nparts = gran;
+    // A linear layer with few output columns would leave each block a sliver of a tile (or leave SMs idle): give the
+    // blocks full 16-granule column tiles instead and cut the contraction into ranges, summed up afterwards.
+    int ksplit = 1;
+    if (p.out_bf16 && p.lin_part && m_tiles == 1 && gran < 148 * 8) {
+        const int col_parts = (gran + 15) / 16;
+        const int kb_all = p.hid / BK;
+        ksplit = 148 / col_parts;
+        if (ksplit > kb_all / 4) ksplit = kb_all / 4;    // at least four 64-wide steps per range
+        if (ksplit > p.max_ksplit) ksplit = p.max_ksplit;
+        if (ksplit < 1) ksplit = 1;
+        if (ksplit > 1) nparts = col_parts;
+    }
     const int cmax = (gran + nparts - 1) / nparts;       // granules of the largest block
     const int T = (cmax + 15) / 16;                      // tiles per block so that a tile has <= 16 granules
     Args a;
@@ -538,6 +571,8 @@ int launch_umma(const Params& p, int need_sum, bool allow_pair, int* nparts_out,
     a.out_logits = p.out_logits;
     a.out_bf16 = p.out_bf16;
     a.residual = p.residual;
+    a.ksplit = ksplit;
+    a.lin_part = p.lin_part;
     a.part = p.part;
     CUtensorMap tm_h, tm_w_hi, tm_w_lo;
     int rc = make_operand_map(&tm_h, p.h, (uint64_t)p.M, (uint64_t)p.hid, (uint32_t)a.h_box_rows);
@@ -555,7 +590,8 @@ int launch_umma(const Params& p, int need_sum, bool allow_pair, int* nparts_out,
         if (rc != DEER_OK) return rc;
     }
     const int smem_bytes = a.stages * a.stage_bytes + (a.z_tma ? STAGING_BYTES : 0) + 1024 /*alignment slack*/ + 256 /*barriers*/;
-    dim3 grid(m_tiles, nparts);
+    dim3 grid(m_tiles, nparts * ksplit);
+    if (ksplit_out) *ksplit_out = ksplit;
     if (pair) {
         DEER_CUDA(cudaFuncSetAttribute(lmhead_umma_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
         lmhead_umma_pair_kernel<<<grid, umma::THREADS, smem_bytes, st>>>(tm_h, tm_w_hi, tm_w_lo, tm_z, a);

@@ -4,6 +4,7 @@ program that profiler captures are taken from.
     python -m paper_2512_15176_b200.profile_case lmhead --M 32 --hid 4096 --V 32768 --iters 3
     python -m paper_2512_15176_b200.profile_case attn --B 8 --Hq 32 --Hkv 8 --k 32 --ctx 8192 --iters 3
     python -m paper_2512_15176_b200.profile_case qstats --B 4 --k 32 --V 151936 --iters 3
+    python -m paper_2512_15176_b200.profile_case layer --B 1 --k 32 --ctx 4096 --hid 4096 --inter 12288 --iters 20
 
 Prints the average CUDA-event time per call and the achieved GB/s over the
 call's algorithmic bytes.
@@ -22,7 +23,8 @@ from . import workload as W
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["lmhead", "attn", "qstats"])
+    ap.add_argument("what", choices=["lmhead", "attn", "qstats", "layer"])
+    ap.add_argument("--inter", type=int, default=12288)
     ap.add_argument("--M", type=int, default=32)
     ap.add_argument("--hid", type=int, default=4096)
     ap.add_argument("--V", type=int, default=32768)
@@ -71,6 +73,34 @@ def main():
         call = lambda: L.deer_block_attn(kv, seq_ids, q, kb, vb, out, cfg.mask, 0, 1.0 / math.sqrt(a.D), a.ctx, ws)
         nbytes = W.algorithmic_bytes(cfg, lengths)["attn"]
         flops = float(W.algorithmic_flops(cfg, lengths)["attn"])
+    elif a.what == "layer":
+        # one verifier layer (Qwen3-8B shape by default) at M = B k rows, replayed from a CUDA graph
+        from .runner import VerifierLayer
+        cfg = W.StepConfig("prof", a.B, a.Hq, a.Hkv, a.D, a.k, a.hid, 64, (a.ctx, a.ctx), seed=34, growth=a.k)
+        lengths = W.seq_lengths(cfg)
+        lay = W.kv_layout(cfg, lengths)
+        kp, vp = W.kv_pools(cfg, lay.num_pages, device=dev, sigma=1.0)
+        kv = L.KVCache.from_layout(lay, kp, vp, dev)
+        hid, QD, KD = a.hid, a.Hq * a.D, a.Hkv * a.D
+        mk = lambda n, shape, sig: W.normal(34, n, shape, sig, device=dev)
+        w = {"ln1": mk("ln1", (hid,), 1.0), "ln2": mk("ln2", (hid,), 1.0), "q_norm": mk("qn", (a.D,), 1.0),
+             "k_norm": mk("kn", (a.D,), 1.0), "wq": mk("wq", (QD, hid), hid ** -0.5), "wk": mk("wk", (KD, hid), hid ** -0.5),
+             "wv": mk("wv", (KD, hid), hid ** -0.5), "wo": mk("wo", (hid, QD), QD ** -0.5),
+             "wgu": mk("wgu", (2 * a.inter, hid), hid ** -0.5), "wd": mk("wd", (hid, a.inter), a.inter ** -0.5)}
+        x = mk("x", (cfg.M, hid), 1.0)
+        layer = VerifierLayer(cfg, kv, w, a.ctx + a.k, a.inter)
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            for _ in range(3):
+                layer.forward(x)
+            side.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                layer.forward(x)
+        torch.cuda.synchronize()
+        call = g.replay
+        nbytes = sum(t.numel() * 2 for n, t in w.items()) + W.algorithmic_bytes(cfg, lengths)["attn"]
+        flops = 2.0 * cfg.M * sum(t.numel() for n, t in w.items() if n.startswith("w"))
     else:
         M = a.B * a.k
         ql = W.normal(33, "ql", (a.B, a.k, a.V), 1.0, dtype=torch.float32, device=dev)

@@ -197,22 +197,23 @@ class VerifierLayer:
         self.attn_out, self.x1, self.xn2 = e(B, k, Hq, D), e(M, hid), e(M, hid)
         self.gu, self.act, self.x2 = e(M, 2 * self.inter), e(M, self.inter), e(M, hid)
         self.attn_ws = _ws(L.deer_block_attn_workspace_bytes(B, k, Hq, Hkv, D, self.max_seq_len), device)
+        self.lin_ws = _ws(max(L.deer_linear_workspace_bytes(M, hid, n) for n in (Hq * D, 2 * self.inter, hid)) or 16, device)
         self.scale = 1.0 / math.sqrt(D)
 
     def forward(self, x: torch.Tensor) -> torch.Tensor:
         c, w = self.cfg, self.w
         M = c.M
         L.deer_rmsnorm(x, w["ln1"], self.xn, self.eps)
-        L.deer_linear(self.xn, w["wq"], self.q.view(M, -1))
-        L.deer_linear(self.xn, w["wk"], self.k_blk.view(M, -1))
-        L.deer_linear(self.xn, w["wv"], self.v_blk.view(M, -1))
+        L.deer_linear(self.xn, w["wq"], self.q.view(M, -1), workspace=self.lin_ws)
+        L.deer_linear(self.xn, w["wk"], self.k_blk.view(M, -1), workspace=self.lin_ws)
+        L.deer_linear(self.xn, w["wv"], self.v_blk.view(M, -1), workspace=self.lin_ws)
         L.deer_qk_norm_rope(self.kv, self.seq_ids, self.q, self.k_blk, w.get("q_norm"), w.get("k_norm"), self.eps, self.theta)
         L.deer_kv_reserve(self.kv, self.seq_ids, c.k)
         L.deer_block_attn(self.kv, self.seq_ids, self.q, self.k_blk, self.v_blk, self.attn_out, L.DEER_MASK_CAUSAL, True,
                           self.scale, self.max_seq_len, self.attn_ws)
-        L.deer_linear(self.attn_out.view(M, -1), w["wo"], self.x1, residual=x)
+        L.deer_linear(self.attn_out.view(M, -1), w["wo"], self.x1, residual=x, workspace=self.lin_ws)
         L.deer_rmsnorm(self.x1, w["ln2"], self.xn2, self.eps)
-        L.deer_linear(self.xn2, w["wgu"], self.gu)
+        L.deer_linear(self.xn2, w["wgu"], self.gu, workspace=self.lin_ws)
         L.deer_swiglu(self.gu, self.act)
-        L.deer_linear(self.act, w["wd"], self.x2, residual=self.x1)
+        L.deer_linear(self.act, w["wd"], self.x2, residual=self.x1, workspace=self.lin_ws)
         return self.x2

@@ -27,15 +27,18 @@ def _close(got_bf16, want64, label, extra=0.0):
     assert (err <= tol).all(), f"{label}: max err {err.max():.3e} at tolerance {tol.flat[err.argmax()]:.3e}"
 
 
-@pytest.mark.parametrize("M,K,N,res", [(8, 512, 1536, False), (32, 4096, 1024, True), (33, 128, 1000, True),
-                                       (200, 256, 520, False), (300, 192, 4096, True)])
-def test_linear(M, K, N, res):
+@pytest.mark.parametrize("M,K,N,res,ws", [(8, 512, 1536, False, True), (32, 4096, 1024, True, True), (32, 4096, 1024, True, False),
+                                          (33, 128, 1000, True, True), (32, 12288, 4096, True, True), (100, 1024, 24576, False, True),
+                                          (200, 256, 520, False, True), (300, 192, 4096, True, False)])
+def test_linear(M, K, N, res, ws):
+    """ws: with the workspace that lets the call cut the contraction into ranges (few output columns, M <= 128)."""
     from paper_2512_15176_b200 import binding as L
     x = W.normal(11, "x", (M, K), 1.0)
     w = W.normal(11, "w", (N, K), 1.0 / math.sqrt(K))
     r = W.normal(11, "r", (M, N), 1.0) if res else None
     y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
-    L.deer_linear(x.cuda(), w.cuda(), y, residual=r.cuda() if res else None)
+    work = torch.empty(max(L.deer_linear_workspace_bytes(M, K, N), 16), dtype=torch.uint8, device="cuda") if ws else None
+    L.deer_linear(x.cuda(), w.cuda(), y, residual=r.cuda() if res else None, workspace=work)
     torch.cuda.synchronize()
     want = O.linear(Hn.f64(x), Hn.f64(w)) + (Hn.f64(r) if res else 0.0)
     _close(y, want, f"linear {M}x{K}x{N}")
