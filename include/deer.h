@@ -300,6 +300,11 @@ int deer_linear(const void* x, const void* w, const void* residual, void* y, int
 int deer_rmsnorm(const void* x, const void* gamma, void* y, int M, int hid, float eps, void* stream);
 int deer_qk_norm_rope(deer_kv* kv, const int32_t* seq_ids, void* q, void* k_blk, const void* q_gamma,
                       const void* k_gamma, int B, int k, int Hq, float eps, float theta, void* stream);
+/* As deer_qk_norm_rope, fed by ONE fused projection: qkv bf16 [B k][(Hq + 2 Hkv) D] holds each row's query heads,
+ * then its key heads, then its value heads; q and k_blk receive the transformed heads, v_blk a copy of the rest. */
+int deer_qkv_split_norm_rope(deer_kv* kv, const int32_t* seq_ids, const void* qkv, void* q, void* k_blk, void* v_blk,
+                             const void* q_gamma, const void* k_gamma, int B, int k, int Hq, float eps, float theta,
+                             void* stream);
 int deer_swiglu(const void* gate_up, void* y, int M, int I, void* stream);
 
 /* ------------------------------------------------------------------------

@@ -27,7 +27,7 @@ EXPORTS = [
     "deer_block_attn_workspace_bytes", "deer_block_attn", "deer_lmhead_workspace_bytes", "deer_lmhead_select",
     "deer_accept_workspace_bytes", "deer_accept", "deer_verify_step_host",
     "deer_lmhead_static_max_rows", "deer_lmhead_select_static", "deer_emit", "deer_draft_stats",
-    "deer_linear_workspace_bytes", "deer_linear", "deer_rmsnorm", "deer_qk_norm_rope", "deer_swiglu",
+    "deer_linear_workspace_bytes", "deer_linear", "deer_rmsnorm", "deer_qk_norm_rope", "deer_qkv_split_norm_rope", "deer_swiglu",
 ]
 
 
@@ -93,6 +93,8 @@ def lib() -> ctypes.CDLL:
     L.deer_rmsnorm.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int, c_float, c_void_p]
     L.deer_qk_norm_rope.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_float,
                                     c_float, c_void_p]
+    L.deer_qkv_split_norm_rope.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int,
+                                           c_int, c_int, c_float, c_float, c_void_p]
     L.deer_swiglu.argtypes = [c_void_p, c_void_p, c_int, c_int, c_void_p]
     L.deer_draft_stats.argtypes = [c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
     L.deer_emit.argtypes = [c_int, c_int, c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p,
@@ -258,6 +260,12 @@ def deer_qk_norm_rope(kv: "KVCache", seq_ids, q, k_blk, q_gamma, k_gamma, eps, t
     B, k, Hq, _ = q.shape
     _check(lib().deer_qk_norm_rope(kv.handle, _ptr(seq_ids), _ptr(q), _ptr(k_blk), _ptr(q_gamma), _ptr(k_gamma), B, k, Hq,
                                    float(eps), float(theta), _stream(stream)))
+
+
+def deer_qkv_split_norm_rope(kv: "KVCache", seq_ids, qkv, q, k_blk, v_blk, q_gamma, k_gamma, eps, theta, stream=None):
+    B, k, Hq, _ = q.shape
+    _check(lib().deer_qkv_split_norm_rope(kv.handle, _ptr(seq_ids), _ptr(qkv), _ptr(q), _ptr(k_blk), _ptr(v_blk), _ptr(q_gamma),
+                                          _ptr(k_gamma), B, k, Hq, float(eps), float(theta), _stream(stream)))
 
 
 def deer_swiglu(gate_up, y, stream=None):

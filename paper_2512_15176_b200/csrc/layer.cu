@@ -38,21 +38,34 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const __nv_bfloat16* __res
 
 // One warp per (block row, head) of q or k: optional RMSNorm over the head's D values, then the rotation of the
 // pairs (d, d + D/2) by pos * theta^(-2d/D).  In place.
+// With `qkv` (the packed output [B k][(Hq + 2 Hkv) D] of one fused projection) the values are read from there and
+// q, k_blk, v_blk are written (v copied as it is); without it q and k_blk are transformed in place.
 __global__ void __launch_bounds__(128) qk_norm_rope_kernel(deer_kv_desc kv, const int32_t* __restrict__ seq_ids,
+                                                           const __nv_bfloat16* __restrict__ qkv,
                                                            __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ kb,
+                                                           __nv_bfloat16* __restrict__ vb,
                                                            const __nv_bfloat16* __restrict__ q_gamma,
                                                            const __nv_bfloat16* __restrict__ k_gamma, int B, int k, int Hq, int Hkv,
                                                            int D, float eps, double log2_theta) {
     const int lane = threadIdx.x & 31;
     const long long item = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
     const long long nq = (long long)B * k * Hq, nk = (long long)B * k * Hkv;
-    if (item >= nq + nk) return;
+    if (item >= nq + nk + (qkv ? nk : 0)) return;
+    if (item >= nq + nk) {                                        // a V head: copy out of the packed rows
+        const long long r = item - nq - nk;
+        const long long bi = r / Hkv;
+        const int hh = (int)(r % Hkv);
+        const __nv_bfloat16* src = qkv + (bi * (Hq + 2 * Hkv) + Hq + Hkv + hh) * D;
+        for (int d = lane; d < D; d += 32) vb[r * D + d] = src[d];
+        return;
+    }
     const bool is_q = item < nq;
     const long long r = is_q ? item : item - nq;
     const int H = is_q ? Hq : Hkv;
     const long long bi = r / H;                                   // b * k + i
     const int b = (int)(bi / k), i = (int)(bi % k);
     __nv_bfloat16* v = (is_q ? q : kb) + r * D;
+    const __nv_bfloat16* in = qkv ? qkv + (bi * (Hq + 2 * Hkv) + (is_q ? 0 : Hq) + (r % H)) * D : v;
     const __nv_bfloat16* gamma = is_q ? q_gamma : k_gamma;
     const int s = seq_ids[b];
     const int n = (s >= 0 && s < kv.max_seqs) ? kv.seq_len[s] : 0;
@@ -66,8 +79,8 @@ __global__ void __launch_bounds__(128) qk_norm_rope_kernel(deer_kv_desc kv, cons
         const int d = lane + 32 * t;
         a[t] = c[t] = 0.f;
         if (d < half) {
-            a[t] = __bfloat162float(v[d]);
-            c[t] = __bfloat162float(v[d + half]);
+            a[t] = __bfloat162float(in[d]);
+            c[t] = __bfloat162float(in[d + half]);
             ss += a[t] * a[t] + c[t] * c[t];
         }
     }
@@ -117,8 +130,8 @@ extern "C" int deer_rmsnorm(const void* x, const void* gamma, void* y, int M, in
     return DEER_OK;
 }
 
-extern "C" int deer_qk_norm_rope(deer_kv* kv, const int32_t* seq_ids, void* q, void* k_blk, const void* q_gamma,
-                                 const void* k_gamma, int B, int k, int Hq, float eps, float theta, void* stream) {
+static int qk_norm_rope(deer_kv* kv, const int32_t* seq_ids, const void* qkv, void* q, void* k_blk, void* v_blk, const void* q_gamma,
+                        const void* k_gamma, int B, int k, int Hq, float eps, float theta, void* stream) {
     DEER_CHECK_ARG(kv && seq_ids && q && k_blk, DEER_ERR_INVALID_ARG, "deer_qk_norm_rope: null argument");
     DEER_CHECK_ARG((q_gamma == nullptr) == (k_gamma == nullptr), DEER_ERR_INVALID_ARG,
                    "deer_qk_norm_rope: q_gamma and k_gamma come together");
@@ -126,13 +139,26 @@ extern "C" int deer_qk_norm_rope(deer_kv* kv, const int32_t* seq_ids, void* q, v
                    "deer_qk_norm_rope: bad sizes");
     if (B == 0) return DEER_OK;
     const int Hkv = kv->d.n_kv_heads, D = kv->d.head_dim;
-    const long long items = (long long)B * k * (Hq + Hkv);
+    const long long items = (long long)B * k * (Hq + Hkv + (qkv ? Hkv : 0));
     qk_norm_rope_kernel<<<(unsigned)((items + 3) / 4), 128, 0, static_cast<cudaStream_t>(stream)>>>(
-        kv->d, seq_ids, static_cast<__nv_bfloat16*>(q), static_cast<__nv_bfloat16*>(k_blk),
+        kv->d, seq_ids, static_cast<const __nv_bfloat16*>(qkv), static_cast<__nv_bfloat16*>(q), static_cast<__nv_bfloat16*>(k_blk),
+        static_cast<__nv_bfloat16*>(v_blk),
         static_cast<const __nv_bfloat16*>(q_gamma), static_cast<const __nv_bfloat16*>(k_gamma), B, k, Hq, Hkv, D, eps,
         log2((double)theta));
     DEER_CUDA(cudaGetLastError());
     return DEER_OK;
+}
+
+extern "C" int deer_qk_norm_rope(deer_kv* kv, const int32_t* seq_ids, void* q, void* k_blk, const void* q_gamma,
+                                 const void* k_gamma, int B, int k, int Hq, float eps, float theta, void* stream) {
+    return qk_norm_rope(kv, seq_ids, nullptr, q, k_blk, nullptr, q_gamma, k_gamma, B, k, Hq, eps, theta, stream);
+}
+
+extern "C" int deer_qkv_split_norm_rope(deer_kv* kv, const int32_t* seq_ids, const void* qkv, void* q, void* k_blk, void* v_blk,
+                                        const void* q_gamma, const void* k_gamma, int B, int k, int Hq, float eps, float theta,
+                                        void* stream) {
+    DEER_CHECK_ARG(qkv && v_blk, DEER_ERR_INVALID_ARG, "deer_qkv_split_norm_rope: null argument");
+    return qk_norm_rope(kv, seq_ids, qkv, q, k_blk, v_blk, q_gamma, k_gamma, B, k, Hq, eps, theta, stream);
 }
 
 extern "C" int deer_swiglu(const void* gate_up, void* y, int M, int I, void* stream) {

@@ -84,8 +84,8 @@ def main():
         hid, QD, KD = a.hid, a.Hq * a.D, a.Hkv * a.D
         mk = lambda n, shape, sig: W.normal(34, n, shape, sig, device=dev)
         w = {"ln1": mk("ln1", (hid,), 1.0), "ln2": mk("ln2", (hid,), 1.0), "q_norm": mk("qn", (a.D,), 1.0),
-             "k_norm": mk("kn", (a.D,), 1.0), "wq": mk("wq", (QD, hid), hid ** -0.5), "wk": mk("wk", (KD, hid), hid ** -0.5),
-             "wv": mk("wv", (KD, hid), hid ** -0.5), "wo": mk("wo", (hid, QD), QD ** -0.5),
+             "k_norm": mk("kn", (a.D,), 1.0), "wqkv": mk("wqkv", (QD + 2 * KD, hid), hid ** -0.5),
+             "wo": mk("wo", (hid, QD), QD ** -0.5),
              "wgu": mk("wgu", (2 * a.inter, hid), hid ** -0.5), "wd": mk("wd", (hid, a.inter), a.inter ** -0.5)}
         x = mk("x", (cfg.M, hid), 1.0)
         layer = VerifierLayer(cfg, kv, w, a.ctx + a.k, a.inter)

@@ -182,8 +182,9 @@ class VerifierLayer:
     RMSNorm of q, k + rotary embedding -> block attention against the paged cache
     (the block's K/V rows are appended) -> output projection + residual -> RMSNorm
     -> gate/up projection -> SiLU(gate) * up -> down projection + residual.
-    Weights are [out][in] bf16 tensors on the device; every intermediate stays
-    there (attributes, so that a test can look at each stage)."""
+    Weights are [out][in] bf16 tensors on the device ("wqkv" = the query, key and
+    value projections stacked in that order); every intermediate stays there
+    (attributes, so that a test can look at each stage)."""
 
     def __init__(self, cfg: StepConfig, kv: L.KVCache, weights: dict, max_seq_len: int, inter: int, eps=1e-6,
                  theta=1.0e6, device="cuda"):
@@ -194,20 +195,20 @@ class VerifierLayer:
         e = lambda *shape: torch.empty(*shape, dtype=bf, device=device)
         self.seq_ids = torch.arange(B, dtype=torch.int32, device=device)
         self.xn, self.q, self.k_blk, self.v_blk = e(M, hid), e(B, k, Hq, D), e(B, k, Hkv, D), e(B, k, Hkv, D)
+        self.qkv = e(M, (Hq + 2 * Hkv) * D)
         self.attn_out, self.x1, self.xn2 = e(B, k, Hq, D), e(M, hid), e(M, hid)
         self.gu, self.act, self.x2 = e(M, 2 * self.inter), e(M, self.inter), e(M, hid)
         self.attn_ws = _ws(L.deer_block_attn_workspace_bytes(B, k, Hq, Hkv, D, self.max_seq_len), device)
-        self.lin_ws = _ws(max(L.deer_linear_workspace_bytes(M, hid, n) for n in (Hq * D, 2 * self.inter, hid)) or 16, device)
+        self.lin_ws = _ws(max(L.deer_linear_workspace_bytes(M, hid, n) for n in ((Hq + 2 * Hkv) * D, 2 * self.inter, hid)) or 16, device)
         self.scale = 1.0 / math.sqrt(D)
 
     def forward(self, x: torch.Tensor) -> torch.Tensor:
         c, w = self.cfg, self.w
         M = c.M
         L.deer_rmsnorm(x, w["ln1"], self.xn, self.eps)
-        L.deer_linear(self.xn, w["wq"], self.q.view(M, -1), workspace=self.lin_ws)
-        L.deer_linear(self.xn, w["wk"], self.k_blk.view(M, -1), workspace=self.lin_ws)
-        L.deer_linear(self.xn, w["wv"], self.v_blk.view(M, -1), workspace=self.lin_ws)
-        L.deer_qk_norm_rope(self.kv, self.seq_ids, self.q, self.k_blk, w.get("q_norm"), w.get("k_norm"), self.eps, self.theta)
+        L.deer_linear(self.xn, w["wqkv"], self.qkv, workspace=self.lin_ws)
+        L.deer_qkv_split_norm_rope(self.kv, self.seq_ids, self.qkv, self.q, self.k_blk, self.v_blk, w.get("q_norm"),
+                                   w.get("k_norm"), self.eps, self.theta)
         L.deer_kv_reserve(self.kv, self.seq_ids, c.k)
         L.deer_block_attn(self.kv, self.seq_ids, self.q, self.k_blk, self.v_blk, self.attn_out, L.DEER_MASK_CAUSAL, True,
                           self.scale, self.max_seq_len, self.attn_ws)

@@ -98,6 +98,7 @@ def test_verifier_layer_matches_oracle():
          "wv": mk("wv", (Hkv * D, hid), hid ** -0.5), "wo": mk("wo", (hid, Hq * D), (Hq * D) ** -0.5),
          "wgu": mk("wgu", (2 * inter, hid), hid ** -0.5), "wd": mk("wd", (hid, inter), inter ** -0.5)}
     wd = {n: t.cuda() for n, t in w.items()}
+    wd["wqkv"] = torch.cat([w["wq"], w["wk"], w["wv"]], dim=0).contiguous().cuda()
     w64 = {n: Hn.f64(t) for n, t in w.items()}
     x = mk("x", (M, hid), 1.0)
     layer = VerifierLayer(cfg, kv, wd, int(st.lengths.max()) + cfg.k, inter, eps, theta)
