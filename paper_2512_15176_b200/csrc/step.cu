@@ -35,15 +35,21 @@ std::mutex g_mu;
 StepCache g_cache;
 
 // A second stream for the copies that the attention does not need (hidden states, draft ids): they cross the bus
-// while the attention kernel runs.  Created on first use, one per process.
+// while the attention kernel runs.  Created on first use; they belong to the device that was current then and are
+// made anew when the call comes on another device (the cached graph is keyed by the device as well).
 cudaStream_t g_side = nullptr;
 cudaEvent_t g_fork = nullptr, g_join = nullptr;
+int g_side_device = -1;
 
 int side_stream() {
-    if (g_side) return DEER_OK;
+    int device = 0;
+    DEER_CUDA(cudaGetDevice(&device));
+    if (g_side && g_side_device == device) return DEER_OK;
+    g_side = nullptr;                 // the old ones stay with their device for the life of the process
     DEER_CUDA(cudaStreamCreateWithFlags(&g_side, cudaStreamNonBlocking));
     DEER_CUDA(cudaEventCreateWithFlags(&g_fork, cudaEventDisableTiming));
     DEER_CUDA(cudaEventCreateWithFlags(&g_join, cudaEventDisableTiming));
+    g_side_device = device;
     return DEER_OK;
 }
 
