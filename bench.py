@@ -2,17 +2,22 @@
 """Benchmark of the DEER draft-verify step on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1] [--impl ours|reference]
+    python bench.py --sweep [--steps K]          # every point of the sweep -> profiles/sweep.md
 
 A "step" is one pass of the whole hot path -- kv_reserve, block attention
 (append), LM head + argmax, acceptance, kv_commit -- over one batch of seeded
-synthetic input shaped like a Qwen3-8B verify step (workload index 1: batch 1,
-32q/8kv heads, head_dim 128, context 4096, block 32, hidden 4096, vocab
-151936).  Prints ONE JSON line.  With N > 1 (under torchrun) every rank runs an
-independent replica on its own GPU; there is no data-path collective.
+synthetic input.  The headline workload is the Qwen3-8B-shaped verify step
+(workload index 1: batch 1, 32q/8kv heads, head_dim 128, context 4096, block
+32, hidden 4096, vocab 151936); the same JSON line carries, under
+``workloads``, the drafter block fill, the Qwen3-30B-A3B-shaped sampling step
+and one large sweep point, each timed the same way.  Prints ONE JSON line.
+With N > 1 (under torchrun) every rank runs an independent replica on its own
+GPU; there is no data-path collective.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import sys
@@ -29,11 +34,31 @@ from paper_2512_15176_b200 import workload as W  # noqa: E402
 
 METRIC = "verified draft tokens/s per verify step"
 UNIT = "tokens/s"
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_traffic.json")
+KERNEL_SOURCES = {"lmhead_umma_kernel": ["paper_2512_15176_b200/csrc/lmhead_umma.cu", "paper_2512_15176_b200/csrc/sm100.cuh",
+                                         "paper_2512_15176_b200/csrc/lmhead.cuh"]}
 
-# DRAM bytes (read + write) of one lmhead_umma_kernel launch from ncu, per workload name; absent = not captured for
-# the kernel as it stands.  Captured at full size (M = 32, hidden 4096, V = 151936: 1 246 011 392 read + 5 147 392
-# written, dram__bytes_{read,write}.sum alone, one launch), 1.005 x the algorithmic bytes.
-LMHEAD_TRAFFIC = {"C2-qwen3-8b-verify": 1246011392 + 5147392}
+
+def kernel_source_hash(kernel: str) -> str:
+    h = hashlib.sha256()
+    for rel in KERNEL_SOURCES[kernel]:
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(kernel: str, workload: str):
+    """DRAM bytes (read + write) of one launch of ``kernel`` on ``workload`` as a profiler counted them, from the
+    tracked file beside the profile summaries -- or None when nothing was recorded for this workload, or when the
+    kernel's sources have changed since (the record carries their hash)."""
+    try:
+        with open(TRAFFIC_FILE) as f:
+            rec = json.load(f).get(kernel, {}).get(workload)
+    except (OSError, ValueError):
+        return None
+    if not rec or rec.get("source_sha16") != kernel_source_hash(kernel):
+        return None
+    return int(rec["dram_bytes_read"]) + int(rec["dram_bytes_write"])
 
 
 def load_peaks():
@@ -47,11 +72,12 @@ def load_peaks():
 
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML (read-only queries) in
-    a thread while the timed region runs."""
+    a thread, back to back (a query takes a fraction of a millisecond), from the
+    warm-up replays to the end of the timed region."""
 
     REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
-    def __init__(self, gpu_index: int, period_s: float = 0.002):
+    def __init__(self, gpu_index: int, period_s: float = 0.0002):
         self.gpu, self.period = gpu_index, period_s
         self.sm, self.bits, self.max_mhz, self.power = [], 0, None, []
         self.stop_flag = threading.Event()
@@ -80,14 +106,17 @@ class ClockSampler:
 
     def _loop(self):
         nv = self.nv
+        n = 0
         while not self.stop_flag.is_set():
             try:
                 self.sm.append(float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
                 self.bits |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
-                self.power.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
+                if n % 16 == 0:
+                    self.power.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
             except Exception as e:
                 self.err = repr(e)
                 return
+            n += 1
             time.sleep(self.period)
 
     def stop(self):
@@ -96,8 +125,9 @@ class ClockSampler:
         self.stop_flag.set()
         self.thread.join(timeout=2)
         reasons = sorted(name for bit, name in self.REASONS.items() if self.bits & bit)
-        return {"sm_mhz": float(np.median(self.sm)) if self.sm else None, "sm_max_mhz": self.max_mhz, "reasons": reasons,
-                "samples": len(self.sm), "power_w_max": max(self.power) if self.power else None}
+        return {"sm_mhz": float(np.median(self.sm)) if self.sm else None, "sm_min_mhz": float(min(self.sm)) if self.sm else None,
+                "sm_max_mhz": self.max_mhz, "reasons": reasons, "samples": len(self.sm),
+                "power_w_max": max(self.power) if self.power else None}
 
 
 def max_over_ranks(values, device, world):
@@ -117,41 +147,70 @@ def dist_env():
     return rank, world, local
 
 
+def config_dict(cfg, world):
+    """What both arms print as ``config``: the workload, and how the CUDA arm is launched and keeps L2 cold."""
+    lengths = W.seq_lengths(cfg)
+    bidir = cfg.mask == W.MASK_BIDIR
+    accept_text = {"greedy": "greedy, planted Geometric(0.1) prefix capped at k",
+                   "argmax_logprob": "none (drafter block fill: argmax + max log-probability per position)",
+                   "sample": "rejection sampling at temperature %.2g with residual resampling" % cfg.temperature}[cfg.mode]
+    return {"workload": cfg.name, "B": cfg.B, "k": cfg.k, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D,
+            "ctx": [int(lengths.min()), int(lengths.max())], "hid": cfg.hid, "V": cfg.V,
+            "mask": "bidirectional" if bidir else "causal", "accept": accept_text, "parallelism": f"replicas x{world}",
+            "launch": "CUDA arm: one CUDA graph per step, timed by events at its two ends",
+            "l2": "CUDA arm: flushed between steps by a 512 MiB write followed by a 256 MiB read; the weight stream "
+                  "exceeds L2 by itself"}
+
+
 # ---------------------------------------------------------------------------
 # oracle arm: the CPU oracle as it stands, on the host cores
 # ---------------------------------------------------------------------------
 
-def oracle_step_seconds(cfg, repeat=1):
-    """One whole step of ``cfg`` through the oracle (attention, logits, argmax,
-    greedy acceptance, KV append + commit).  Returns (seconds per step, tokens
-    per step, description of the sample)."""
-    import math
-    from oracle import deer_oracle as O
-    lengths = W.seq_lengths(cfg)
-    lay = W.kv_layout(cfg, lengths)
-    kp, vp = W.kv_pools(cfg, lay.num_pages)
-    f32 = lambda t: t.to(torch.float32).numpy()
-    kv = O.PagedKV(f32(kp), f32(vp), lay.page_table, lay.seq_len, lay.n_pages, lay.free_stack, lay.free_top)
-    w = f32(W.lm_head(cfg))
-    q, kb, vb = (f32(t) for t in W.block_qkv(cfg))
-    h = f32(W.hidden(cfg))
-    ids = np.arange(cfg.B)
-    times = []
-    snap = (kv.page_table.copy(), kv.seq_len.copy(), kv.n_pages.copy(), kv.free_stack.copy(), kv.free_top)
-    for it in range(repeat):
-        kv.page_table, kv.seq_len, kv.n_pages, kv.free_stack = (a.copy() for a in snap[:4])
-        kv.free_top = snap[4]           # every repeat sees the same prefix
+class OracleStep:
+    """One whole step of ``cfg`` through the oracle (attention, logits, argmax, greedy acceptance, KV append +
+    commit).  ``vocab_rows`` < V bounds the sample: the logits are then taken against the first vocab_rows rows of
+    the head only (everything else is done in full)."""
+
+    def __init__(self, cfg, vocab_rows=None):
+        from oracle import deer_oracle as O
+        self.O, self.cfg = O, cfg
+        lengths = W.seq_lengths(cfg)
+        lay = W.kv_layout(cfg, lengths)
+        kp, vp = W.kv_pools(cfg, lay.num_pages)
+        f32 = lambda t: t.to(torch.float32).numpy()
+        self.kv = O.PagedKV(f32(kp), f32(vp), lay.page_table, lay.seq_len, lay.n_pages, lay.free_stack, lay.free_top)
+        self.w = f32(W.lm_head(cfg))
+        self.vocab_rows = cfg.V if vocab_rows is None else int(vocab_rows)
+        self.q, self.kb, self.vb = (f32(t) for t in W.block_qkv(cfg))
+        self.h = f32(W.hidden(cfg))
+        kv = self.kv
+        self.snap = (kv.page_table.copy(), kv.seq_len.copy(), kv.n_pages.copy(), kv.free_stack.copy(), kv.free_top)
+
+    def run(self, it=0) -> float:
+        import math
+        O, cfg, kv = self.O, self.cfg, self.kv
+        kv.page_table, kv.seq_len, kv.n_pages, kv.free_stack = (a.copy() for a in self.snap[:4])
+        kv.free_top = self.snap[4]           # every run sees the same prefix
+        ids = np.arange(cfg.B)
         t0 = time.perf_counter()
         kv.reserve(ids, cfg.k)
-        O.block_attention(q, kb, vb, kv.k_pool, kv.v_pool, kv.page_table, kv.seq_len, ids, cfg.mask, 1.0 / math.sqrt(cfg.D))
-        kv.append(ids, kb, vb)
-        z = O.lm_logits(h, w)
+        O.block_attention(self.q, self.kb, self.vb, kv.k_pool, kv.v_pool, kv.page_table, kv.seq_len, ids, cfg.mask,
+                          1.0 / math.sqrt(cfg.D))
+        kv.append(ids, self.kb, self.vb)
+        z = O.lm_logits(self.h, self.w[:self.vocab_rows])
         target = O.select_argmax(z).reshape(cfg.B, cfg.k)
         drafts = W.plant_drafts(cfg, target, W.planted_prefix_lengths(cfg, it), it)
         a, out, n = O.accept_greedy(drafts, target)
         kv.commit(ids, a)
-        times.append(time.perf_counter() - t0)
-    return float(np.mean(times)), cfg.M, f"whole step of {cfg.name} (all {cfg.M} block rows, full vocabulary), {repeat} run(s)"
+        return time.perf_counter() - t0
+
+    def sample_text(self, runs):
+        cfg = self.cfg
+        if self.vocab_rows == cfg.V:
+            return f"whole step of {cfg.name} (all {cfg.M} block rows, full vocabulary), {runs} timed run(s) after a warm-up run"
+        return (f"step of {cfg.name} with the logits taken against the first {self.vocab_rows} of {cfg.V} vocabulary rows "
+                f"(all {cfg.M} block rows, attention and acceptance in full); tokens/s scaled by {self.vocab_rows}/{cfg.V}; "
+                f"{runs} timed run(s) after a warm-up run")
 
 
 def run_reference(args, cfg):
@@ -159,16 +218,23 @@ def run_reference(args, cfg):
     if rank != 0:
         return
     cores = len(os.sched_getaffinity(0))
-    for _ in range(max(0, min(args.warmup, 1))):
-        oracle_step_seconds(cfg, 1)
-    reps = max(1, min(args.steps, 3))
-    sec, toks, sample = oracle_step_seconds(cfg, reps)
-    val = toks / sec
-    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": reps,
-            "warmup": min(args.warmup, 1), "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+    budget_s = 150.0
+    st = OracleStep(cfg)
+    t_full = st.run()                                   # untimed: pages the inputs in, and sizes the sample
+    n_runs = args.steps + max(0, args.warmup - 1)
+    if n_runs * t_full > budget_s:
+        rows = max(1024, int(cfg.V * budget_s / (n_runs * t_full)) // 1024 * 1024)
+        st = OracleStep(cfg, vocab_rows=min(rows, cfg.V))
+    for _ in range(max(0, args.warmup - 1)):
+        st.run()
+    secs = [st.run(it) for it in range(args.steps)]
+    sec = float(np.mean(secs))
+    val = cfg.M * (st.vocab_rows / cfg.V) / sec
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": cfg.name, "B": cfg.B, "k": cfg.k, "ctx": list(cfg.ctx), "hid": cfg.hid, "V": cfg.V},
-            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "config": config_dict(cfg, world),
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": st.sample_text(args.steps)},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
@@ -178,27 +244,51 @@ def run_reference(args, cfg):
 # CUDA arm
 # ---------------------------------------------------------------------------
 
-def run_ours(args, cfg):
-    rank, world, local = dist_env()
-    if world > 1:
-        import torch.distributed as dist
-        torch.cuda.set_device(local)
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
+_W_CACHE = {}
+
+
+def head_weights(cfg, dev, on_device):
+    """The LM-head weights of ``cfg`` on ``dev`` (the last one is kept: sweep points share theirs).  ``on_device``
+    draws them with the device generator -- other values than the host draw the tests use, which is fine where they
+    only feed a timing."""
+    key = (cfg.seed, cfg.V, cfg.hid, cfg.sigma_w, bool(on_device), str(dev))
+    if key not in _W_CACHE:
+        _W_CACHE.clear()
+        torch.cuda.empty_cache()
+        _W_CACHE[key] = (W.normal(cfg.seed, "w", (cfg.V, cfg.hid), cfg.sigma_w, device=str(dev)) if on_device
+                         else W.lm_head(cfg).to(dev))
+    return _W_CACHE[key]
+
+
+class Flusher:
+    def __init__(self, dev):
+        self.wr = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+        self.rd = torch.zeros(64 << 20, dtype=torch.int32, device=dev)      # 256 MiB
+
+    def __call__(self):
+        """Evict L2 between steps: a 512 MiB write, then a 256 MiB read so that the
+        write's dirty lines are back in HBM before the timed step starts."""
+        self.wr.zero_()
+        self.rd.max()
+
+
+def measure(cfg, steps, warmup, dev, peaks, flush, world=1, rank=0, with_e2e=False, clock_sampler=None, device_weights=False):
+    """Times ``steps`` steps of ``cfg`` on the current device.  Returns a dict with the step time (events at the two
+    ends of the step's graph), the phase split (a second graph with events between the phases), the roofline of the
+    LM-head call and of the whole step."""
     from paper_2512_15176_b200 import binding as L
     from paper_2512_15176_b200.runner import VerifyStep
-    L.lib()          # fail loudly if the library has not been built
+    import torch.distributed as dist
 
-    peaks = load_peaks()
     greedy = cfg.mode == "greedy"
     lengths = W.seq_lengths(cfg)
     lay = W.kv_layout(cfg, lengths)
     # pools of the larger workloads are drawn on the device (hundreds of MB); the values only feed the timing
     kp, vp = W.kv_pools(cfg, lay.num_pages, device="cpu" if lay.num_pages * cfg.Hkv * cfg.D < (1 << 22) else str(dev))
     kv = L.KVCache.from_layout(lay, kp, vp, dev)
+    del kp, vp
     saved = [t.clone() for t in (kv.page_table, kv.seq_len, kv.n_pages, kv.free_stack, kv.free_top)]
-    w = W.lm_head(cfg).to(dev)
+    w = head_weights(cfg, dev, device_weights)
     vs = VerifyStep(cfg, kv, w, int(lengths.max()), device=dev, store_logits=None if cfg.mode == "sample" else False)
     q, kb, vb = W.block_qkv(cfg)
     h = W.hidden(cfg)
@@ -223,14 +313,6 @@ def run_ours(args, cfg):
         drafts = W.plant_drafts(cfg, target, W.planted_prefix_lengths(cfg))
         vs.load(draft_ids=drafts)
     bidir = cfg.mask == W.MASK_BIDIR
-    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
-    flush_rd = torch.zeros(64 << 20, dtype=torch.int32, device=dev)      # 256 MiB
-
-    def flush_l2():
-        """Evict L2 between steps: a 512 MiB write, then a 256 MiB read so that the
-        write's dirty lines are back in HBM before the timed step starts."""
-        flush.zero_()
-        flush_rd.max()
 
     def phase_attn():
         if not bidir:
@@ -245,70 +327,65 @@ def run_ours(args, cfg):
 
     phases = [phase_attn, vs.lmhead, phase_accept]
 
-    def one_step(events=None):
+    def eager_step():
         restore()
-        flush_l2()
-        for i, ph in enumerate(phases):
-            if events is not None:
-                events[i].record()
+        flush()
+        for ph in phases:
             ph()
-        if events is not None:
-            events[3].record()
 
-    for _ in range(max(args.warmup, 3)):
-        one_step()
+    if clock_sampler is not None:
+        clock_sampler.start()
+    for _ in range(max(warmup, 3)):
+        eager_step()
     torch.cuda.synchronize()
-    graph, gev = None, None
-    if not args.no_graph:
-        # The whole step is replayed from one CUDA graph, with timing events recorded inside it between the phases:
-        # the host's launch work no longer paces the GPU.  The calls and their arguments are exactly the ones above.
-        gev = [torch.cuda.Event(enable_timing=True, external=True) for _ in range(4)]
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
+    # The whole step is replayed from one CUDA graph: the host's launch work does not pace the GPU.  Graph A carries
+    # timing events at its two ends only (the step time); graph B also between the phases (the split).
+    def capture(inner):
+        ev = [torch.cuda.Event(enable_timing=True, external=True) for _ in range(4)]
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            ev[0].record()
             for i, ph in enumerate(phases):
-                gev[i].record()
+                if inner and i > 0:
+                    ev[i].record()
                 ph()
-            gev[3].record()
+            ev[3].record()
+        return g, ev
+
+    g_step, ev_step = capture(False)
+    g_ph, ev_ph = capture(True)
+
+    def replay(g):
+        restore()
+        flush()
+        g.replay()
+        torch.cuda.synchronize()          # the graph's events are re-recorded by the next replay: read them now
+
+    for g in (g_step, g_ph):
         for _ in range(3):
-            restore()
-            flush_l2()
-            graph.replay()
-        torch.cuda.synchronize()
+            replay(g)
     if world > 1:
         dist.barrier()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
-    marks = []          # per step: ms from the step's start to the end of each phase
     torch.cuda.synchronize()
     wall0 = time.perf_counter()
-    for s in range(args.steps):
-        if graph is None:
-            one_step(evs[s])
-        else:
-            restore()
-            flush_l2()
-            graph.replay()
-            torch.cuda.synchronize()          # the graph's events are re-recorded by the next replay: read them now
-            marks.append([gev[0].elapsed_time(gev[i]) for i in (1, 2, 3)])
+    step_ms = []
+    for _ in range(steps):
+        replay(g_step)
+        step_ms.append(ev_step[0].elapsed_time(ev_step[3]))
     torch.cuda.synchronize()
     wall = time.perf_counter() - wall0
     if world > 1:
         dist.barrier()
-    clocks = sampler.stop() if rank == 0 else None
-    if graph is None:
-        marks = [[e[0].elapsed_time(e[i]) for i in (1, 2, 3)] for e in evs]
-    step_ms = [m[2] for m in marks]
-    attn_ms = [m[0] for m in marks]
-    lm_ms = [m[1] - m[0] for m in marks]
-    total_ms = float(sum(step_ms))
+    marks = []
+    for _ in range(min(steps, 50)):
+        replay(g_ph)
+        marks.append([ev_ph[0].elapsed_time(ev_ph[i]) for i in (1, 2, 3)])
     status = L.deer_kv_status(kv)
-    accepted = int(vs.accept_len.sum().item())
+    accepted = int(vs.accept_len.sum().item()) if not bidir else None
 
     # ---- end to end: host buffers in, verdict out, every step (the greedy verify step has such a call) ----
     e2e_s, h2d, d2h = 0.0, 0, 0
-    if greedy:
+    if greedy and with_e2e:
         pin = lambda t: t.contiguous().pin_memory()
         hq, hkb, hvb, hh = pin(q), pin(kb), pin(vb), pin(h)
         hd = pin(torch.from_numpy(drafts))
@@ -322,9 +399,9 @@ def run_ours(args, cfg):
         h2d = sum(t.numel() * t.element_size() for t in (hq, hkb, hvb, hh, hd))
         d2h = sum(t.numel() * t.element_size() for t in (ha, ho, hn))
         es = torch.cuda.Stream()          # a stream of its own: the call replays its copies and kernels as one graph there
-        for s in range(3 + args.steps):
+        for s in range(3 + steps):
             restore()
-            flush_l2()
+            flush()
             torch.cuda.synchronize()
             t0 = time.perf_counter()
             L.deer_verify_step_host(kv, sd, w, hq, hkb, hvb, hh, hd, cfg.B, cfg.k, cfg.Hq, cfg.hid, cfg.V, vs.scale,
@@ -332,61 +409,151 @@ def run_ours(args, cfg):
             dt = time.perf_counter() - t0
             if s >= 3:
                 e2e_s += dt
-    total_s, e2e_total = max_over_ranks([total_ms / 1e3, e2e_s], dev, world)
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
+    clocks = clock_sampler.stop() if clock_sampler is not None else None
+    total_s, e2e_total = max_over_ranks([float(sum(step_ms)) / 1e3, e2e_s], dev, world)
 
-    tokens = cfg.M * args.steps * world
-    value = tokens / total_s
     ab = W.algorithmic_bytes(cfg, lengths)
     fl = W.algorithmic_flops(cfg, lengths)
     hbm, tens = peaks["hbm_gbs"] * 1e9, peaks["bf16_tflops_sustained"] * 1e12
-    attn_s, lm_s = float(np.mean(attn_ms)) / 1e3, float(np.mean(lm_ms)) / 1e3
-    step_s = total_s / args.steps
+    m = np.asarray(marks, dtype=np.float64)
+    attn_s, lm_s, acc_s = float(m[:, 0].mean()) / 1e3, float((m[:, 1] - m[:, 0]).mean()) / 1e3, float((m[:, 2] - m[:, 1]).mean()) / 1e3
+    step_s = total_s / steps
     # the dominant kernel is the LM head; it is HBM-bound below about hbm-ridge rows and tensor-bound above
-    lm_tensor_bound = fl["lmhead"] / tens > ab["lmhead"] / hbm
-    if lm_tensor_bound:
+    if fl["lmhead"] / tens > ab["lmhead"] / hbm:
         achieved, peak, unit, bound = fl["lmhead"] / lm_s / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s", "tensor"
     else:
         achieved, peak, unit, bound = ab["lmhead"] / lm_s / 1e9, peaks["hbm_gbs"], "GB/s", "hbm"
-    floor_s = (max(ab["attn"] / hbm, fl["attn"] / tens) + max(ab["lmhead"] / hbm, fl["lmhead"] / tens) + ab["accept"] / hbm)
-    accept_text = {"greedy": "greedy, planted Geometric(0.1) prefix capped at k",
-                   "argmax_logprob": "none (drafter block fill: argmax + max log-probability per position)",
-                   "sample": "rejection sampling at temperature %.2g with residual resampling" % cfg.temperature}[cfg.mode]
-    line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-        "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": cfg.name, "B": cfg.B, "k": cfg.k, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D,
-                   "ctx": [int(lengths.min()), int(lengths.max())], "hid": cfg.hid, "V": cfg.V,
-                   "mask": "bidirectional" if bidir else "causal", "accept": accept_text, "parallelism": f"replicas x{world}",
-                   "launch": "host launches" if args.no_graph else "one CUDA graph per step, timing events recorded inside it",
-                   "l2": "flushed between steps by a 512 MiB write followed by a 256 MiB read; the weight stream exceeds L2 by itself"},
-        "roofline": {"bound": bound, "kernel": "deer_lmhead_select", "achieved": achieved, "peak": peak,
-                     "unit": unit, "frac": achieved / peak, "traffic": LMHEAD_TRAFFIC.get(cfg.name), "peak_source": peaks["source"],
+    attn_floor = max(ab["attn"] / hbm, fl["attn"] / tens)
+    lm_floor = max(ab["lmhead"] / hbm, fl["lmhead"] / tens)
+    floor_s = attn_floor + lm_floor + ab["accept"] / hbm
+    out = {
+        "config": config_dict(cfg, world),
+        "ms_per_step": step_s * 1e3,
+        "value": cfg.M * steps * world / total_s,
+        "steps": steps,
+        "roofline": {"bound": bound, "kernel": "lmhead_umma_kernel" if cfg.M <= 128 else "lmhead_umma_pair_kernel",
+                     "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
+                     "traffic": recorded_traffic("lmhead_umma_kernel", cfg.name) if cfg.M <= 128 else None,
+                     "peak_source": peaks["source"] + (" (sustained)" if bound == "tensor" else ""),
                      "bytes_per_launch": ab["lmhead"], "flops_per_launch": fl["lmhead"], "avg_launch_ms": lm_s * 1e3,
-                     "step_frac_of_roofline_floor": floor_s / step_s, "step_floor_ms": floor_s * 1e3},
+                     "step_frac_of_roofline_floor": floor_s / step_s, "step_floor_ms": floor_s * 1e3,
+                     "attn_plus_lmhead_frac_of_floor": (attn_floor + lm_floor) / (attn_s + lm_s)},
         "phases": {"attn_ms": attn_s * 1e3, "attn_gbs": ab["attn"] / attn_s / 1e9, "attn_frac_of_hbm": ab["attn"] / attn_s / hbm,
-                   "attn_tflops": fl["attn"] / attn_s / 1e12, "lmhead_ms": lm_s * 1e3, "lmhead_gbs": ab["lmhead"] / lm_s / 1e9,
-                   "lmhead_tflops": fl["lmhead"] / lm_s / 1e12, "accept_commit_ms": (step_s - attn_s - lm_s) * 1e3},
-        "e2e": ({"value": cfg.M * args.steps * world / e2e_total, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                 "ms_per_step": e2e_total * 1e3 / args.steps} if greedy else
-                {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
-                 "note": "the host-buffer entry point covers the greedy verify step only"}),
-        "gpu_launches": args.steps * vs.launches_per_step(),
-        "clocks": clocks,
+                   "attn_tflops": fl["attn"] / attn_s / 1e12, "attn_frac_of_floor": attn_floor / attn_s,
+                   "lmhead_ms": lm_s * 1e3, "lmhead_gbs": ab["lmhead"] / lm_s / 1e9, "lmhead_tflops": fl["lmhead"] / lm_s / 1e12,
+                   "accept_commit_ms": acc_s * 1e3, "step_ms_with_phase_events": float(m[:, 2].mean())},
+        "gpu_launches": steps * vs.launches_per_step(),
         "kv_status": status, "accepted_tokens_last_step": accepted, "wall_s_timed_loop": wall,
-        "flops_per_step": fl["total"],
+        "flops_per_step": fl["total"], "clocks": clocks,
     }
-    if world == 1 and greedy and not args.no_cpu_baseline:
-        sec, toks, sample = oracle_step_seconds(cfg, 1)
-        line["cpu_baseline"] = {"value": toks / sec, "unit": UNIT, "cores": len(os.sched_getaffinity(0)), "kind": "oracle",
-                                "sample": sample}
+    if greedy and with_e2e:
+        out["e2e"] = {"value": cfg.M * steps * world / e2e_total, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                      "d2h_bytes_per_step": d2h, "ms_per_step": e2e_total * 1e3 / steps}
+    del vs, kv, w
+    torch.cuda.empty_cache()
+    return out
+
+
+def run_ours(args, cfg):
+    rank, world, local = dist_env()
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    from paper_2512_15176_b200 import binding as L
+    L.lib()          # fail loudly if the library has not been built
+
+    peaks = load_peaks()
+    flush = Flusher(dev)
+    sampler = ClockSampler(local) if rank == 0 else None
+    head = measure(cfg, args.steps, args.warmup, dev, peaks, flush, world, rank, with_e2e=True, clock_sampler=sampler)
+
+    # the other named workloads, one GPU's worth each (rank 0 of a multi-rank job skips them: the job's line is the
+    # headline's replicas)
+    others = {}
+    if world == 1 and not args.no_workloads and not args.sweep_point and args.config == 1:
+        extra_steps = min(args.steps, 20)
+        for name, c in (("C3", W.config(2)), ("C4", W.config(3)),
+                        ("C5-B64-ctx32768-k32-causal", W.sweep_config(64, 32768, 32, W.MASK_CAUSAL, steps=1))):
+            r = measure(c, extra_steps, 3, dev, peaks, flush, clock_sampler=ClockSampler(local), device_weights=True)
+            r.pop("flops_per_step", None)
+            others[name] = r
+    if rank != 0:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+        return
+
+    line = {
+        "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic", "config": head["config"], "roofline": head["roofline"], "phases": head["phases"],
+        "e2e": head.get("e2e", {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+                                "note": "the host-buffer entry point covers the greedy verify step only"}),
+        "gpu_launches": head["gpu_launches"], "clocks": head["clocks"], "kv_status": head["kv_status"],
+        "accepted_tokens_last_step": head["accepted_tokens_last_step"], "wall_s_timed_loop": head["wall_s_timed_loop"],
+        "flops_per_step": head["flops_per_step"],
+    }
+    if others:
+        line["workloads"] = others
+    if world == 1 and cfg.mode == "greedy" and not args.no_cpu_baseline:
+        st = OracleStep(cfg)
+        st.run()                        # warm-up: the first run pages the 1.2 GB of weights in
+        sec = st.run()
+        line["cpu_baseline"] = {"value": cfg.M / sec, "unit": UNIT, "cores": len(os.sched_getaffinity(0)), "kind": "oracle",
+                                "sample": st.sample_text(1)}
     print(json.dumps(line), flush=True)
     if world > 1:
+        import torch.distributed as dist
         dist.destroy_process_group()
+
+
+# ---------------------------------------------------------------------------
+# the sweep: every point, one table
+# ---------------------------------------------------------------------------
+
+def run_sweep(args):
+    """All 96 points (batch x context x block size x mask), each timed for ``--steps`` steps of the single-step
+    graph; writes profiles/sweep.md and prints one JSON line with the table's rows."""
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    from paper_2512_15176_b200 import binding as L
+    L.lib()
+    peaks = load_peaks()
+    flush = Flusher(dev)
+    rows = []
+    for mask, mname in ((W.MASK_CAUSAL, "causal"), (W.MASK_BIDIR, "bidir")):
+        for B in (1, 4, 16, 64):
+            for ctx in (1024, 4096, 16384, 32768):
+                for k in (8, 16, 32):
+                    cfg = W.sweep_config(B, ctx, k, mask, steps=1)
+                    if mask == W.MASK_BIDIR:
+                        cfg = cfg.with_(mode="argmax_logprob")
+                    r = measure(cfg, args.steps, 3, dev, peaks, flush, device_weights=True)
+                    rows.append({"B": B, "ctx": ctx, "k": k, "mask": mname, "ms_per_step": r["ms_per_step"],
+                                 "tokens_per_s": r["value"], "attn_ms": r["phases"]["attn_ms"],
+                                 "attn_frac_of_floor": r["phases"]["attn_frac_of_floor"], "lmhead_ms": r["phases"]["lmhead_ms"],
+                                 "lmhead_bound": r["roofline"]["bound"], "lmhead_frac": r["roofline"]["frac"],
+                                 "accept_commit_ms": r["phases"]["accept_commit_ms"],
+                                 "step_frac_of_floor": r["roofline"]["step_frac_of_roofline_floor"], "kv_status": r["kv_status"]})
+    path = os.path.join(ROOT, args.sweep_out)
+    with open(path, "w") as f:
+        f.write("# Sweep: batch x context x block size x mask (32q/8kv heads, head_dim 128, hidden 4096, vocabulary 151936)\n\n")
+        f.write(f"`python bench.py --sweep --steps {args.steps}` on one B200; ragged lengths in [ctx/2, ctx], greedy acceptance "
+                "with planted prefixes (causal) or argmax + max log-probability (bidirectional block fill); one CUDA graph per "
+                "step, L2 flushed between steps.  Peaks: HBM %.1f GB/s, bf16 %.1f TFLOP/s sustained (%s).  `of floor` = time "
+                "the algorithmic bytes / flops take at those peaks over the measured time.\n\n" %
+                (peaks["hbm_gbs"], peaks["bf16_tflops_sustained"], peaks["source"]))
+        f.write("| mask | B | ctx | k | step us | verified tok/s | attention us | attn of floor | LM head us | LM head of peak | accept+commit us | step of floor |\n")
+        f.write("|---|---|---|---|---|---|---|---|---|---|---|---|\n")
+        for r in rows:
+            f.write("| %s | %d | %d | %d | %.1f | %.0f | %.1f | %.2f | %.1f | %.2f (%s) | %.1f | %.2f |\n" %
+                    (r["mask"], r["B"], r["ctx"], r["k"], r["ms_per_step"] * 1e3, r["tokens_per_s"], r["attn_ms"] * 1e3,
+                     r["attn_frac_of_floor"], r["lmhead_ms"] * 1e3, r["lmhead_frac"], r["lmhead_bound"],
+                     r["accept_commit_ms"] * 1e3, r["step_frac_of_floor"]))
+    print(json.dumps({"sweep": rows, "table": args.sweep_out}), flush=True)
 
 
 def main():
@@ -397,11 +564,16 @@ def main():
     ap.add_argument("--config", type=int, default=1, help="workload index 0..3 (1 = Qwen3-8B-shaped verify step)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-graph", action="store_true", help="launch every call from the host instead of replaying CUDA graphs")
+    ap.add_argument("--no-workloads", action="store_true", help="time the headline workload only")
     ap.add_argument("--sweep-point", default=None, metavar="B,CTX,K,MASK",
                     help="time one point of the sweep instead of a fixed workload: batch, context (ragged lengths in "
                          "[CTX/2, CTX]), block size, causal|bidir")
+    ap.add_argument("--sweep", action="store_true", help="time every point of the sweep and write the table")
+    ap.add_argument("--sweep-out", default="profiles/sweep.md")
     args = ap.parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     if args.sweep_point:
         b, ctx, k, mask = args.sweep_point.split(",")
         cfg = W.sweep_config(int(b), int(ctx), int(k), W.MASK_BIDIR if mask == "bidir" else W.MASK_CAUSAL, steps=1)

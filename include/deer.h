@@ -66,8 +66,7 @@ const char* deer_last_error(void);
 
 /* ------------------------------------------------------------------------
  * Paged KV cache = the committed prefix x_{1:j} of each sequence
- * (Section 3.2: "the chosen token is appended to the prefix and becomes part
- * of the context"; Algorithm 1: j <- length(x)).
+ * (Section 3.2, the step after Eq. 6; Algorithm 1's update of j).
  *
  * State, all caller-allocated device arrays described by deer_kv_desc:
  *   k_pool, v_pool  bf16 [num_pages][Hkv][16][D]
@@ -110,7 +109,7 @@ int deer_kv_destroy(deer_kv* kv);
  * seq_ids: i32 [B], distinct.  B <= 1024. */
 int deer_kv_reserve(deer_kv* kv, const int32_t* seq_ids, int B, int k, void* stream);
 
-/* (4) Commit / roll back (Algorithm 1, "Update j <- length(x)"): seq_len[s] += keep[b]
+/* (4) Commit / roll back (Algorithm 1's update of j): seq_len[s] += keep[b]
  * with keep clamped to [0, k]; block rows written at positions >= the new length
  * are thereby dropped, and pages wholly beyond it return to the free stack --
  * sequences in order, logical pages descending.  `keep` is a device array
@@ -158,6 +157,15 @@ int deer_block_attn(deer_kv* kv, const int32_t* seq_ids,
  *   out_draft_logit  f32 [M]  z[draft_ids[m]]              (DEER_SEL_SOFTMAX, draft_ids != NULL)
  *   out_logits       f32 [M][V], optional in any mode (NULL = not stored)
  * Outputs not used by `mode` may be NULL.  temperature > 0 (ignored for ARGMAX).
+ * hid must be a multiple of 64 and V at least 16 (else DEER_ERR_UNSUPPORTED).
+ *   workspace  >= deer_lmhead_workspace_bytes(...) bytes, 16-byte aligned,
+ *              contents arbitrary: per-row partial results of the thread blocks
+ *              that split the vocabulary, merged inside the same kernel by the
+ *              block that finishes last.  One call at a time per workspace.
+ * Error behaviour on the device: every wait inside the kernel is bounded (about a
+ * second); a thread block whose wait runs out gives up, and every row it worked on
+ * gets out_ids[m] = -2 (no valid id is negative) with the other outputs of that
+ * row undefined.  The call itself still returns DEER_OK: it is asynchronous.
  * ---------------------------------------------------------------------- */
 size_t deer_lmhead_workspace_bytes(int M, int hid, int V);
 
@@ -184,11 +192,12 @@ int deer_lmhead_select(const void* h, const void* w, int M, int hid, int V,
  *   - The call allocates and frees nothing, on the device or through any
  *     library routine.  The first call on each device looks up the array's
  *     device address (with that device current); make that first call outside
- *     any stream capture.
+ *     any stream capture (inside one it returns DEER_ERR_UNSUPPORTED and does
+ *     nothing).
  *   - All calls on one GPU share the array, which keeps the previous call's
- *     contents; each call overwrites every slot it later reads, so no clearing
- *     is needed, but two calls that overlap on the GPU (different streams) race
- *     on it -- serialise them.
+ *     contents; each call overwrites every slot it later reads and leaves its
+ *     arrival counters at zero, so no clearing is needed, but two calls that
+ *     overlap on the GPU (different streams) race on it -- serialise them.
  * ---------------------------------------------------------------------- */
 #define DEER_STATIC_MAX_ROWS 256
 
@@ -248,9 +257,9 @@ int deer_accept(int mode, int B, int k, int V,
                 void* workspace, size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------
- * (5) Book-keeping of one pass of Algorithm 1's outer loop ("while the last
- * token is not EOS": the tokens chosen in this block are appended to the
- * output, "update j <- length(x)").  For every sequence that has not finished:
+ * (5) Book-keeping of one pass of Algorithm 1's outer loop (it runs until an
+ * EOS is emitted: the tokens chosen in this block join the output, then j is
+ * updated).  For every sequence that has not finished:
  * out_ids[b][0 .. n_out[b]) (deer_accept's output, already cut after an EOS) is
  * appended to tokens[b] as far as max_new allows; the sequence finishes when an
  * appended token equals eos_id (eos_id < 0 disables) or when it holds max_new
@@ -280,6 +289,8 @@ int deer_emit(int B, int k, const int32_t* accept_len, const int32_t* out_ids, c
  *   output, gate/up and down projections.  x bf16 [M][K], w bf16 [N][K],
  *   residual bf16 [M][N] or NULL, y bf16 [M][N]; K a multiple of 64, N >= 16.
  *   The LM-head kernels without their selection: weight-streaming for small M.
+ *   (As there: a thread block whose bounded wait runs out leaves its output
+ *   tiles unwritten; the call has no status word of its own.)
  *   With a workspace of deer_linear_workspace_bytes (may be NULL / 0: slower for
  *   few output columns) the contraction is cut into ranges whose fp32 partial
  *   products are summed by a second kernel, so that every SM streams weights
@@ -319,9 +330,10 @@ int deer_swiglu(const void* gate_up, void* y, int M, int I, void* stream);
  * buffers, the first call with a given set of arguments records the copies and
  * kernels into a CUDA graph and later calls with the same arguments replay it
  * (one launch instead of sixteen enqueues); the graph belongs to the library
- * and is replaced when the arguments change.  The environment variable
- * DEER_STEP_GRAPH=0 turns this off.  Not to be called on a stream that is being
- * captured.
+ * (a few of them are kept, the least recently used one is replaced).  Every
+ * pointer and size of `kv`'s descriptor, of `dev` and of the argument list is
+ * part of that key, so swapping any buffer records a new graph.  Not to be
+ * called on a stream that is being captured.
  * ---------------------------------------------------------------------- */
 typedef struct deer_step_dev {
     void* q; void* k_blk; void* v_blk; void* attn_out;     /* bf16 staging, shapes as in deer_block_attn */

@@ -235,9 +235,9 @@ def accept_sample(draft_ids, target_logits, temperature, draft_logits, u, r, eos
 
 
 # --------------------------------------------------------------------------
-# (4) KV cache reserve / append / commit -- "the chosen token is appended to
-#     the prefix and becomes part of the context" (Section 3.2); j <- length(x)
-#     (Algorithm 1).  Rows of the block beyond the kept length are dropped.
+# (4) KV cache reserve / append / commit -- the chosen tokens join the prefix
+#     (Section 3.2, the step after Eq. 6; Algorithm 1's update of j).  Rows of
+#     the block beyond the kept length are dropped.
 # --------------------------------------------------------------------------
 
 class PagedKV:
@@ -304,8 +304,8 @@ class PagedKV:
 
 
 # --------------------------------------------------------------------------
-# (5) Algorithm 1's outer loop: "while the last token is not EOS ... append the
-#     chosen tokens to the prefix ... update j <- length(x)".  One call of
+# (5) Algorithm 1's outer loop (it runs until an EOS is emitted; the chosen
+#     tokens join the prefix and j is updated to its new length).  One call of
 #     emit() is the book-keeping of one pass of that loop for every sequence:
 #     what was chosen in this block joins the sequence's output, the sequence
 #     ends at an EOS or at a length limit, and only the accepted draft tokens

@@ -366,6 +366,7 @@ __global__ void __launch_bounds__(RES_THREADS) residual_pick_kernel(ResidualArgs
     __syncthreads();
     if (tid == 0) {
         int hit = s_hit;
+        if (!(target > 0.0)) hit = 0;         // r = 0: the smallest v whose cumulative sum is >= 0 is the first token
         if (hit < 0) {
             // the target lies beyond the slice's last cumulative sum by rounding: the last token with weight up to there
             for (int v = v1 - 1; v >= 0; --v)
@@ -481,13 +482,13 @@ extern "C" int deer_draft_stats(int B, int k, int V, const int32_t* draft_ids, c
     const SampleWs w = carve(workspace, B, k, V);
     // Meant to run beside the attention kernel, whose blocks take 56 K of an SM's 64 K registers and most of its
     // shared memory.  Two things let a block of this kernel share an SM with one of those: at most one block per SM
-    // (148 blocks of 256 threads and 32 registers, striding over the rows; a block per row filled the SMs first and
+    // (one block of 256 threads and 32 registers per SM, striding over the rows; a block per row filled the SMs first and
     // the two kernels took turns), and the same shared-memory carve-out as that kernel asks for -- blocks of kernels
     // with different carve-outs do not share an SM at all (measured: without it the LM head beside this kernel took
     // 496 us instead of 283).
-    const int rows = B * k;
+    const int rows = B * k, sms = deer_sm_count();
     DEER_CUDA(cudaFuncSetAttribute(draft_row_stats_kernel<256, 4>, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
-    draft_row_stats_kernel<256, 4><<<rows < 148 ? rows : 148, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+    draft_row_stats_kernel<256, 4><<<rows < sms ? rows : sms, 256, 0, static_cast<cudaStream_t>(stream)>>>(
         rows, V, draft_logits, draft_ids, w.lse_q, w.zq_draft);
     DEER_CUDA(cudaGetLastError());
     return DEER_OK;

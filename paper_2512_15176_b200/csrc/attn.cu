@@ -11,9 +11,6 @@
 // straight from k_blk/v_blk as one more tile handled by the last chunk's block,
 // which also appends them to the cache when asked to.
 
-#include <stdlib.h>
-#include <string.h>
-
 #include "attn.cuh"
 
 namespace attn {
@@ -327,11 +324,8 @@ constexpr int attn_smem_bytes() {
 
 static int mma_row_tiles(int k, int G) { return (G * k + ATT_ROWS - 1) / ATT_ROWS; }
 
-// DEER_ATTN_IMPL=mma forces the warp-level kernel (used to cross-check the tcgen05 one).
-static bool use_umma(int D, int G, float scale) {
-    const char* force = getenv("DEER_ATTN_IMPL");
-    return umma_supported(D, G, scale) && !(force && strcmp(force, "mma") == 0);
-}
+// The tcgen05 kernel takes head_dim 128; the warp-level kernel serves head_dim 64.
+static bool use_umma(int D, int G, float scale) { return umma_supported(D, G, scale); }
 
 }  // namespace attn
 

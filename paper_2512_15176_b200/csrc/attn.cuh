@@ -38,7 +38,7 @@ inline AttnPlan plan_attn(int B, int Hkv, int row_tiles, int max_seq_len) {
     AttnPlan pl;
     pl.row_tiles = row_tiles;
     const long units = (long)B * Hkv * row_tiles;
-    const long target_blocks = 2L * 148;
+    const long target_blocks = 2L * deer_sm_count();
     long per_unit = (target_blocks + units - 1) / units;
     if (per_unit < 1) per_unit = 1;
     long chunk = (max_seq_len + per_unit - 1) / per_unit;

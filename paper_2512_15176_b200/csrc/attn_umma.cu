@@ -55,7 +55,6 @@ constexpr int TMEM_COLS = 512;                 // S0..S3 [0,256)  P0 [256,288)  
 constexpr int P_COL = 256;
 constexpr int O_COL = 384;
 constexpr int MAX_SEGS = 48;                   // segments listed at a time; longer shares go in several rounds
-constexpr int NUM_SMS = 148;
 constexpr float RESCALE_STEP = 8.f;            // raise the running maximum only when a tile exceeds it by 2^8
 // Slot layout.  A K (or V) tile of 64 tokens x 128 dims is 16 KB of 1 KB swizzle atoms (8 tokens x 64 dims).
 //   prefix tile: [page 0..3][token group 0..1][dim half 0..1][8 tokens][128 B] -- what one 5-D TMA box per page
@@ -715,7 +714,7 @@ __global__ void __launch_bounds__(256) attn_umma_merge_kernel(const AttnParams p
 static int pick_blocks(int B, int HR, int HKV, int max_seq_len) {
     const long long t_max = (long long)B * HR * ((max_seq_len + ATT_TILE - 1) / ATT_TILE + 1);
     long long nc = t_max / 8;
-    if (nc > NUM_SMS) nc = NUM_SMS;
+    if (nc > deer_sm_count()) nc = deer_sm_count();
     const int rt = HR / HKV > 0 ? HR / HKV : 1;
     nc = nc / rt * rt;                                    // whole groups of row_tiles blocks
     if (nc < rt) nc = rt;
@@ -783,7 +782,7 @@ int launch_umma(AttnParams p, cudaStream_t st) {
     DEER_CUDA(cudaFuncSetAttribute(block_attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
     block_attn_umma_kernel<<<p.nc, THREADS, SMEM_BYTES, st>>>(tm_q, tm_kb, tm_vb, tm_kp, tm_vp, p);
     DEER_CUDA(cudaGetLastError());
-    if ((long long)p.B * HR * 4 >= 2 * NUM_SMS) attn_umma_merge_kernel<4><<<(unsigned)(p.B * HR * 4), 256, 0, st>>>(p);
+    if ((long long)p.B * HR * 4 >= 2 * deer_sm_count()) attn_umma_merge_kernel<4><<<(unsigned)(p.B * HR * 4), 256, 0, st>>>(p);
     else attn_umma_merge_kernel<1><<<(unsigned)(p.B * HR * 16), 256, 0, st>>>(p);
     DEER_CUDA(cudaGetLastError());
     return DEER_OK;

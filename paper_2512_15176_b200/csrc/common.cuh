@@ -34,6 +34,29 @@ void deer_set_error(const char* fmt, ...);
 
 static inline bool deer_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Streaming multiprocessors of the current device (asked once per device).  Grids and workspaces are sized by it.
+// Where no device can be asked (a host without a GPU sizing a workspace) it is a B200's 148.
+inline int deer_sm_count() {
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        cudaGetLastError();
+        return 148;
+    }
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+            cudaGetLastError();
+            n = 148;
+        }
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+// A tag for one call's arrival words (see arrive_last); never 0, distinct for every call of the process.
+uint32_t deer_next_epoch();
+
 // ---- device helpers --------------------------------------------------------
 #ifdef __CUDACC__
 
@@ -73,6 +96,27 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// "Last block done" without a counter that somebody has to clear.  `word` holds (tag << 32 | arrivals); a caller
+// that finds another tag than its call's `epoch` starts the count anew, so whatever the memory held before (an
+// uninitialised workspace, an older call) does not matter, and the caller that completes `expected` arrivals
+// puts the word back to 0, so that a replay of the same launch (a CUDA graph carries the same epoch) starts
+// clean as well.  Returns true for exactly one caller: the one that arrived last.  Writes made before a
+// __threadfence() by the other callers are visible to it after its own __threadfence().
+__device__ __forceinline__ bool arrive_last(unsigned long long* word, uint32_t epoch, uint32_t expected) {
+    unsigned long long cur = *reinterpret_cast<volatile unsigned long long*>(word);
+    for (;;) {
+        const uint32_t cnt = ((uint32_t)(cur >> 32) == epoch) ? (uint32_t)cur + 1u : 1u;
+        const unsigned long long nxt = ((unsigned long long)epoch << 32) | cnt;
+        const unsigned long long old = atomicCAS(word, cur, nxt);
+        if (old == cur) {
+            if (cnt != expected) return false;
+            *reinterpret_cast<volatile unsigned long long*>(word) = 0ull;
+            return true;
+        }
+        cur = old;                 // another block arrived in between: at most `expected` rounds
+    }
 }
 
 // Record the first data-dependent error seen by any kernel.

@@ -1,6 +1,6 @@
 // Paged-KV manager: the committed prefix x_{1:j} as pages, with reserve (room
 // for the next block) and commit/rollback to the accepted length
-// (Section 3.2 and Algorithm 1's "Update j <- length(x)").
+// (Section 3.2 and Algorithm 1's update of j).
 //
 // Both kernels run as ONE thread block: thread b owns sequence seq_ids[b],
 // a block-wide exclusive scan gives each sequence its offset on the free
@@ -10,6 +10,7 @@
 #include <stdarg.h>
 #include <string.h>
 
+#include <atomic>
 #include <new>
 
 #include "common.cuh"
@@ -25,6 +26,13 @@ void deer_set_error(const char* fmt, ...) {
 }
 
 extern "C" const char* deer_last_error(void) { return g_err; }
+
+uint32_t deer_next_epoch() {
+    static std::atomic<uint32_t> next{1};
+    uint32_t e = next.fetch_add(1, std::memory_order_relaxed);
+    while (e == 0) e = next.fetch_add(1, std::memory_order_relaxed);
+    return e;
+}
 
 // ---- handle ----------------------------------------------------------------
 extern "C" int deer_kv_create(deer_kv** kv, const deer_kv_desc* desc) {

@@ -1,89 +1,25 @@
 // (2) LM head + selection: z = h w^T, p_AR = softmax(z / T) of Eq. 5 reduced
 // on the fly to argmax / log-sum-exp / the draft token's logit.
 //
-// Host entry point, the cross-part finalisation, and kernel dispatch.
+// Host entry points: argument checks and the workspace layout; the kernels are in lmhead_umma.cu.
 
-#include <stdlib.h>
-#include <string.h>
-
-#include "lmhead_mma.cuh"
+#include "lmhead.cuh"
 
 namespace lmhead {
 
 bool umma_supported(int M, int hid, int V);
-int launch_umma(const Params& p, int need_sum, bool allow_pair, int* nparts_out, cudaStream_t st, int* ksplit_out = nullptr);
+int launch_umma(const Params& p, int need_sum, cudaStream_t st, int* ksplit_out = nullptr);
 
-struct FinalizeArgs {
-    const Partial* part;
-    int nparts, M;
-    float inv_t_log2, inv_t;
-    int32_t* out_ids;
-    float* out_max_logprob;
-    float* out_lse;
-};
-
-// One warp per row: the lanes stride over the vocabulary parts, then merge by shuffles.
-__global__ void __launch_bounds__(256) lmhead_finalize_kernel(FinalizeArgs a) {
-    const int m = blockIdx.x * 8 + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (m >= a.M) return;
-    float rm = -INFINITY, rs = 0.f;
-    int32_t ri = 0x7fffffff;
-    bool aborted = false;
-    for (int pt = lane; pt < a.nparts; pt += 32) {
-        const Partial pr = a.part[(size_t)pt * a.M + m];
-        aborted |= (pr.idx == PARTIAL_ABORTED);
-        merge_sel(rm, ri, rs, pr.m, pr.idx, pr.s, a.inv_t_log2);
-    }
-    aborted = __any_sync(0xffffffffu, aborted);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        const float om = __shfl_xor_sync(0xffffffffu, rm, o);
-        const int32_t oi = __shfl_xor_sync(0xffffffffu, ri, o);
-        const float os = __shfl_xor_sync(0xffffffffu, rs, o);
-        merge_sel(rm, ri, rs, om, oi, os, a.inv_t_log2);
-    }
-    if (lane != 0) return;
-    if (a.out_ids) a.out_ids[m] = aborted ? PARTIAL_ABORTED : ri;
-    const float ls = logf(rs);
-    if (a.out_max_logprob) a.out_max_logprob[m] = -ls;          // max z - logsumexp(z), T = 1
-    if (a.out_lse) a.out_lse[m] = rm * a.inv_t + ls;            // logsumexp(z / T)
-}
-
-struct Plan {
-    int bm, m_tiles, nparts;
-};
-
-static Plan plan(int M, int V) {
-    Plan pl;
-    pl.bm = (M <= 32) ? 32 : (M <= 64 ? 64 : 128);
-    pl.m_tiles = (M + pl.bm - 1) / pl.bm;
-    const int resident = 148 * (pl.bm <= 64 ? 2 : 1);
-    int np = resident / pl.m_tiles;
-    if (np < 1) np = 1;
-    const int vt = (V + VT - 1) / VT;
-    if (np > vt) np = vt;
-    pl.nparts = np;
-    return pl;
-}
-
-template <int BM>
-static int launch(const Params& p, const Plan& pl, cudaStream_t st) {
-    constexpr int SM = STAGES * (VT * KT * 2 + BM * KT * 2) + 8 * BM * (int)sizeof(Partial);
-    DEER_CUDA(cudaFuncSetAttribute(lmhead_mma_kernel<BM>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM));
-    dim3 grid(pl.m_tiles, pl.nparts);
-    lmhead_mma_kernel<BM><<<grid, THREADS, SM, st>>>(p);
-    DEER_CUDA(cudaGetLastError());
-    return DEER_OK;
-}
+// Workspace of the selection: one Partial per (vocabulary part, row) for as many parts as there are SMs, then one
+// arrival word per tile of 128 rows.
+static size_t part_bytes(int M) { return ((size_t)deer_sm_count() * M * sizeof(Partial) + 255) / 256 * 256; }
 
 }  // namespace lmhead
 
 extern "C" size_t deer_lmhead_workspace_bytes(int M, int hid, int V) {
     (void)hid;
     if (M <= 0 || V <= 0) return 0;
-    // room for the largest split any kernel variant uses
-    return (size_t)2 * 148 * M * sizeof(lmhead::Partial);
+    return lmhead::part_bytes(M) + (size_t)((M + 127) / 128) * sizeof(unsigned long long);
 }
 
 extern "C" int deer_lmhead_select(const void* h, const void* w, int M, int hid, int V, int mode, float temperature,
@@ -95,7 +31,8 @@ extern "C" int deer_lmhead_select(const void* h, const void* w, int M, int hid, 
     DEER_CHECK_ARG(deer_aligned16(h) && deer_aligned16(w) && deer_aligned16(workspace) && deer_aligned16(out_logits),
                    DEER_ERR_INVALID_ARG, "deer_lmhead_select: pointers must be 16-byte aligned");
     DEER_CHECK_ARG(M >= 0 && V > 0 && hid > 0, DEER_ERR_INVALID_ARG, "deer_lmhead_select: bad sizes");
-    DEER_CHECK_ARG(hid % KT == 0, DEER_ERR_UNSUPPORTED, "deer_lmhead_select: hid must be a multiple of 64");
+    DEER_CHECK_ARG(hid % KT == 0 && V >= 16, DEER_ERR_UNSUPPORTED,
+                   "deer_lmhead_select: hid must be a multiple of 64 and V at least 16");
     DEER_CHECK_ARG(mode == DEER_SEL_ARGMAX || mode == DEER_SEL_ARGMAX_LOGPROB || mode == DEER_SEL_SOFTMAX,
                    DEER_ERR_INVALID_ARG, "deer_lmhead_select: bad mode");
     float t = 1.f;
@@ -112,7 +49,6 @@ extern "C" int deer_lmhead_select(const void* h, const void* w, int M, int hid, 
                    "deer_lmhead_select: workspace of %zu bytes needed, %zu given", need, workspace_bytes);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
-    const Plan pl = plan(M, V);
     Params p;
     p.h = static_cast<const __nv_bfloat16*>(h);
     p.w = static_cast<const __nv_bfloat16*>(w);
@@ -120,6 +56,7 @@ extern "C" int deer_lmhead_select(const void* h, const void* w, int M, int hid, 
     p.hid = hid;
     p.V = V;
     p.inv_t_log2 = LOG2E / t;
+    p.inv_t = 1.f / t;
     p.draft_ids = (mode == DEER_SEL_SOFTMAX) ? draft_ids : nullptr;
     p.out_draft_logit = (mode == DEER_SEL_SOFTMAX) ? out_draft_logit : nullptr;
     p.out_logits = out_logits;
@@ -128,32 +65,12 @@ extern "C" int deer_lmhead_select(const void* h, const void* w, int M, int hid, 
     p.lin_part = nullptr;
     p.max_ksplit = 1;
     p.part = static_cast<Partial*>(workspace);
-    p.nparts = pl.nparts;
-    // DEER_LMHEAD_IMPL=mma forces the warp-level kernel, =single the one-block tcgen05 kernel at every M
-    // (used to cross-check the kernels against each other)
-    const char* force = getenv("DEER_LMHEAD_IMPL");
-    const bool use_umma = umma_supported(M, hid, V) && !(force && strcmp(force, "mma") == 0);
-    const bool allow_pair = !(force && strcmp(force, "single") == 0);
-    int nparts = pl.nparts;
-    int rc;
-    if (use_umma) rc = launch_umma(p, mode != DEER_SEL_ARGMAX, allow_pair, &nparts, st);
-    else if (pl.bm == 32) rc = launch<32>(p, pl, st);
-    else if (pl.bm == 64) rc = launch<64>(p, pl, st);
-    else rc = launch<128>(p, pl, st);
-    if (rc != DEER_OK) return rc;
-
-    FinalizeArgs fa;
-    fa.part = p.part;
-    fa.nparts = nparts;
-    fa.M = M;
-    fa.inv_t_log2 = p.inv_t_log2;
-    fa.inv_t = 1.f / t;
-    fa.out_ids = out_ids;
-    fa.out_max_logprob = (mode == DEER_SEL_ARGMAX_LOGPROB) ? out_max_logprob : nullptr;
-    fa.out_lse = (mode == DEER_SEL_SOFTMAX) ? out_lse : nullptr;
-    lmhead_finalize_kernel<<<(M + 7) / 8, 256, 0, st>>>(fa);
-    DEER_CUDA(cudaGetLastError());
-    return DEER_OK;
+    p.tickets = reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) + part_bytes(M));
+    p.epoch = deer_next_epoch();
+    p.out_ids = out_ids;
+    p.out_max_logprob = (mode == DEER_SEL_ARGMAX_LOGPROB) ? out_max_logprob : nullptr;
+    p.out_lse = (mode == DEER_SEL_SOFTMAX) ? out_lse : nullptr;
+    return launch_umma(p, mode != DEER_SEL_ARGMAX, st);
 }
 
 // ------------------------------------------------------------------------------
@@ -236,9 +153,14 @@ extern "C" int deer_linear(const void* x, const void* w, const void* residual, v
         p.max_ksplit = 1;
     }
     p.part = nullptr;
-    p.nparts = 0;
-    int nparts = 0, ksplit = 1;
-    const int rc = launch_umma(p, 0, true, &nparts, st, &ksplit);
+    p.tickets = nullptr;
+    p.epoch = 0;
+    p.inv_t = 1.f;
+    p.out_ids = nullptr;
+    p.out_max_logprob = nullptr;
+    p.out_lse = nullptr;
+    int ksplit = 1;
+    const int rc = launch_umma(p, 0, st, &ksplit);
     if (rc != DEER_OK) return rc;
     if (ksplit > 1) {
         const long long total = (long long)M * N;

@@ -17,7 +17,8 @@
 
 namespace {
 
-// 2 * 148 vocabulary parts x DEER_STATIC_MAX_ROWS rows x 16 bytes of selection state.
+// Room for 2 * 148 vocabulary parts x DEER_STATIC_MAX_ROWS rows x 16 bytes of selection state (the call uses one
+// part per SM) and the arrival words behind them.  The runtime zero-fills it when the library is loaded.
 constexpr size_t STATIC_SCRATCH_BYTES = (size_t)2 * 148 * DEER_STATIC_MAX_ROWS * 16;
 
 static __device__ __align__(256) unsigned char g_lmhead_scratch[STATIC_SCRATCH_BYTES];
@@ -28,12 +29,17 @@ void* g_scratch_addr[MAX_DEVICES] = {};   // device address of g_lmhead_scratch 
 
 // In host code `g_lmhead_scratch` is only a handle for the runtime, not a
 // device address; the address valid on the current device has to be asked for.
-int scratch_for_current_device(void** out) {
+int scratch_for_current_device(void** out, cudaStream_t st) {
     int dev = -1;
     DEER_CUDA(cudaGetDevice(&dev));
     DEER_CHECK_ARG(dev >= 0 && dev < MAX_DEVICES, DEER_ERR_UNSUPPORTED, "deer_lmhead_select_static: device index %d not supported", dev);
     std::lock_guard<std::mutex> lock(g_mu);
     if (!g_scratch_addr[dev]) {
+        // the look-up is a runtime call that a stream capture must not see: say so instead of spoiling the capture
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        DEER_CUDA(cudaStreamIsCapturing(st, &cap));
+        DEER_CHECK_ARG(cap == cudaStreamCaptureStatusNone, DEER_ERR_UNSUPPORTED,
+                       "deer_lmhead_select_static: the first call on a device must come before any stream capture");
         void* p = nullptr;
         DEER_CUDA(cudaGetSymbolAddress(&p, g_lmhead_scratch));
         DEER_CHECK_ARG(p != nullptr, DEER_ERR_CUDA, "deer_lmhead_select_static: scratch symbol has no device address");
@@ -57,10 +63,10 @@ extern "C" int deer_lmhead_select_static(const void* h, const void* w, int M, in
     DEER_CHECK_ARG(deer_lmhead_workspace_bytes(DEER_STATIC_MAX_ROWS, hid, V) <= STATIC_SCRATCH_BYTES, DEER_ERR_UNSUPPORTED,
                    "deer_lmhead_select_static: built-in scratch too small for this shape");
     void* scratch = nullptr;
-    const int rc = scratch_for_current_device(&scratch);
+    const int rc = scratch_for_current_device(&scratch, static_cast<cudaStream_t>(stream));
     if (rc != DEER_OK) return rc;
-    // Every (vocabulary part, row) slot the finalisation reads is rewritten by this
-    // call's own blocks, so nothing in the shared array has to start at zero.
+    // Every (vocabulary part, row) slot the merge reads is rewritten by this call's own blocks, and the arrival
+    // words are put back to zero by the block that arrives last, so nothing has to be cleared between calls.
     return deer_lmhead_select(h, w, M, hid, V, mode, temperature, draft_ids, out_ids, out_max_logprob, out_lse, out_draft_logit,
                               out_logits, scratch, STATIC_SCRATCH_BYTES, stream);
 }

@@ -5,12 +5,13 @@
 // The five copies in, eight kernels and three copies out are sixteen
 // enqueue calls; issued one by one they cost more host time than the copies
 // take on the bus.  So the sequence is captured once into a CUDA graph, keyed
-// by every argument, and replayed with one launch while the arguments stay
-// the same (a decoding loop calls with the same buffers every step).
-// DEER_STEP_GRAPH=0 turns this off; pageable host buffers and a stream that
-// is already being captured take the plain path too.
+// by every argument (the whole cache descriptor and the whole staging-buffer
+// struct included: a graph holds them by value), and replayed with one launch
+// while the arguments stay the same (a decoding loop calls with the same
+// buffers every step).  A few graphs are kept, so that callers that alternate
+// do not evict each other.  Pageable host buffers, the legacy default stream
+// and a stream that is already being captured take the plain path.
 
-#include <stdlib.h>
 #include <string.h>
 
 #include <mutex>
@@ -19,9 +20,15 @@
 
 namespace {
 
+// Everything the recorded copies and kernels hold by value.  Compared with memcmp, so it is filled field by field
+// into zeroed memory (no padding bytes left undefined).
 struct StepKey {
-    const void* p[16];
-    int i[8];
+    deer_kv_desc kv;
+    deer_step_dev dev;
+    const void* kv_handle;
+    const void* w;
+    const void* host[8];
+    int i[6];
     float scale;
     int device;
 };
@@ -29,10 +36,13 @@ struct StepKey {
 struct StepCache {
     StepKey key;
     cudaGraphExec_t exec = nullptr;
+    unsigned long long used = 0;      // value of g_clock at the last launch: the least recently used entry is replaced
 };
 
+constexpr int N_CACHED = 4;
 std::mutex g_mu;
-StepCache g_cache;
+StepCache g_cache[N_CACHED];
+unsigned long long g_clock = 0;
 
 // A second stream for the copies that the attention does not need (hidden states, draft ids): they cross the bus
 // while the attention kernel runs.  Created on first use; they belong to the device that was current then and are
@@ -118,13 +128,12 @@ extern "C" int deer_verify_step_host(deer_kv* kv, const deer_step_dev* dev, cons
     DEER_CHECK_ARG(B > 0 && k >= 1 && k <= DEER_MAX_BLOCK, DEER_ERR_UNSUPPORTED, "deer_verify_step_host: bad B or k");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
-    const char* env = getenv("DEER_STEP_GRAPH");
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     DEER_CUDA(cudaStreamIsCapturing(st, &cap));
     // the legacy default stream cannot be captured
-    const bool use_graph = !(env && atoi(env) == 0) && st != nullptr && cap == cudaStreamCaptureStatusNone && pinned(q_host) &&
-                           pinned(k_blk_host) && pinned(v_blk_host) && pinned(h_host) && pinned(draft_ids_host) &&
-                           pinned(accept_len_host) && pinned(out_ids_host) && pinned(n_out_host);
+    const bool use_graph = st != nullptr && cap == cudaStreamCaptureStatusNone && pinned(q_host) && pinned(k_blk_host) &&
+                           pinned(v_blk_host) && pinned(h_host) && pinned(draft_ids_host) && pinned(accept_len_host) &&
+                           pinned(out_ids_host) && pinned(n_out_host);
     if (!use_graph) {
         const int rc = enqueue(kv, dev, w, q_host, k_blk_host, v_blk_host, h_host, draft_ids_host, B, k, Hq, hid, V, scale,
                                max_seq_len, accept_len_host, out_ids_host, n_out_host, stream, false);
@@ -135,20 +144,38 @@ extern "C" int deer_verify_step_host(deer_kv* kv, const deer_step_dev* dev, cons
 
     StepKey key;
     memset(&key, 0, sizeof(key));
-    const void* ptrs[] = {kv,          w,           q_host,       k_blk_host,   v_blk_host,    h_host,       draft_ids_host,
-                          accept_len_host, out_ids_host, n_out_host, dev->q,       dev->attn_ws,  dev->lm_ws,   kv->d.k_pool,
-                          kv->d.page_table, dev->seq_ids};
-    for (int j = 0; j < 16; ++j) key.p[j] = ptrs[j];
-    const int ints[] = {B, k, Hq, hid, V, max_seq_len, (int)dev->attn_ws_bytes, (int)dev->lm_ws_bytes};
-    for (int j = 0; j < 8; ++j) key.i[j] = ints[j];
+    {
+        const deer_kv_desc& d = kv->d;
+        key.kv.k_pool = d.k_pool; key.kv.v_pool = d.v_pool; key.kv.page_table = d.page_table; key.kv.seq_len = d.seq_len;
+        key.kv.n_pages = d.n_pages; key.kv.free_stack = d.free_stack; key.kv.free_top = d.free_top; key.kv.status = d.status;
+        key.kv.num_pages = d.num_pages; key.kv.n_kv_heads = d.n_kv_heads; key.kv.head_dim = d.head_dim;
+        key.kv.page_size = d.page_size; key.kv.max_seqs = d.max_seqs; key.kv.max_pages = d.max_pages;
+        key.dev.q = dev->q; key.dev.k_blk = dev->k_blk; key.dev.v_blk = dev->v_blk; key.dev.attn_out = dev->attn_out;
+        key.dev.h = dev->h; key.dev.seq_ids = dev->seq_ids; key.dev.draft_ids = dev->draft_ids;
+        key.dev.target_ids = dev->target_ids; key.dev.accept_len = dev->accept_len; key.dev.out_ids = dev->out_ids;
+        key.dev.n_out = dev->n_out; key.dev.attn_ws = dev->attn_ws; key.dev.attn_ws_bytes = dev->attn_ws_bytes;
+        key.dev.lm_ws = dev->lm_ws; key.dev.lm_ws_bytes = dev->lm_ws_bytes;
+    }
+    key.kv_handle = kv;
+    key.w = w;
+    const void* hosts[8] = {q_host, k_blk_host, v_blk_host, h_host, draft_ids_host, accept_len_host, out_ids_host, n_out_host};
+    for (int j = 0; j < 8; ++j) key.host[j] = hosts[j];
+    const int ints[6] = {B, k, Hq, hid, V, max_seq_len};
+    for (int j = 0; j < 6; ++j) key.i[j] = ints[j];
     key.scale = scale;
     DEER_CUDA(cudaGetDevice(&key.device));
 
     std::lock_guard<std::mutex> lock(g_mu);
-    if (!g_cache.exec || memcmp(&g_cache.key, &key, sizeof(key)) != 0) {
-        if (g_cache.exec) {
-            cudaGraphExecDestroy(g_cache.exec);
-            g_cache.exec = nullptr;
+    StepCache* slot = nullptr;
+    for (StepCache& c : g_cache)
+        if (c.exec && memcmp(&c.key, &key, sizeof(key)) == 0) slot = &c;
+    if (!slot) {
+        slot = &g_cache[0];
+        for (StepCache& c : g_cache)
+            if (!c.exec || (slot->exec && c.used < slot->used)) slot = &c;     // a free entry, else the least recently used
+        if (slot->exec) {
+            cudaGraphExecDestroy(slot->exec);
+            slot->exec = nullptr;
         }
         DEER_CUDA(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
         const int rc = enqueue(kv, dev, w, q_host, k_blk_host, v_blk_host, h_host, draft_ids_host, B, k, Hq, hid, V, scale,
@@ -161,13 +188,14 @@ extern "C" int deer_verify_step_host(deer_kv* kv, const deer_step_dev* dev, cons
             return rc;
         }
         DEER_CUDA(ce);
-        const cudaError_t ci = cudaGraphInstantiate(&g_cache.exec, graph, 0);
+        const cudaError_t ci = cudaGraphInstantiate(&slot->exec, graph, 0);
         cudaGraphDestroy(graph);
-        if (ci != cudaSuccess) g_cache.exec = nullptr;
+        if (ci != cudaSuccess) slot->exec = nullptr;
         DEER_CUDA(ci);
-        g_cache.key = key;
+        slot->key = key;
     }
-    DEER_CUDA(cudaGraphLaunch(g_cache.exec, st));
+    slot->used = ++g_clock;
+    DEER_CUDA(cudaGraphLaunch(slot->exec, st));
     DEER_CUDA(cudaStreamSynchronize(st));
     return DEER_OK;
 }

@@ -137,11 +137,11 @@ class VerifyStep:
         self.accept()
         self.commit()
 
-    #: kernels launched by one run(), by mode (attn + merge, lmhead + finalize, accept, reserve/commit)
+    #: kernels launched by one run(), by mode (attention + merge, LM head, reserve + commit, acceptance)
     def launches_per_step(self) -> int:
         if self.cfg.mask == MASK_BIDIR:
-            return 4
-        return 2 + 2 + 2 + (4 if self.cfg.mode == "sample" else 1)
+            return 3
+        return 2 + 1 + 2 + (4 if self.cfg.mode == "sample" else 1)
 
 
 class DecodeLoop:

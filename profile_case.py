@@ -1,10 +1,10 @@
 """Run one library call a few times on a chosen shape -- the small, self-ending
 program that profiler captures are taken from.
 
-    python -m paper_2512_15176_b200.profile_case lmhead --M 32 --hid 4096 --V 32768 --iters 3
-    python -m paper_2512_15176_b200.profile_case attn --B 8 --Hq 32 --Hkv 8 --k 32 --ctx 8192 --iters 3
-    python -m paper_2512_15176_b200.profile_case qstats --B 4 --k 32 --V 151936 --iters 3
-    python -m paper_2512_15176_b200.profile_case layer --B 1 --k 32 --ctx 4096 --hid 4096 --inter 12288 --iters 20
+    python profile_case.py lmhead --M 32 --hid 4096 --V 32768 --iters 3
+    python profile_case.py attn --B 8 --Hq 32 --Hkv 8 --k 32 --ctx 8192 --iters 3
+    python profile_case.py qstats --B 4 --k 32 --V 151936 --iters 3
+    python profile_case.py layer --B 1 --k 32 --ctx 4096 --hid 4096 --inter 12288 --iters 20
 
 Prints the average CUDA-event time per call and the achieved GB/s over the
 call's algorithmic bytes.
@@ -17,8 +17,13 @@ import math
 import numpy as np
 import torch
 
-from . import binding as L
-from . import workload as W
+import os
+import sys
+
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
+
+from paper_2512_15176_b200 import binding as L  # noqa: E402
+from paper_2512_15176_b200 import workload as W  # noqa: E402
 
 
 def main():
@@ -75,7 +80,7 @@ def main():
         flops = float(W.algorithmic_flops(cfg, lengths)["attn"])
     elif a.what == "layer":
         # one verifier layer (Qwen3-8B shape by default) at M = B k rows, replayed from a CUDA graph
-        from .runner import VerifierLayer
+        from paper_2512_15176_b200.runner import VerifierLayer
         cfg = W.StepConfig("prof", a.B, a.Hq, a.Hkv, a.D, a.k, a.hid, 64, (a.ctx, a.ctx), seed=34, growth=a.k)
         lengths = W.seq_lengths(cfg)
         lay = W.kv_layout(cfg, lengths)

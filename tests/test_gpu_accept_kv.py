@@ -118,6 +118,37 @@ def test_sampling_with_the_extra_row(B, k, V, T):
             np.testing.assert_array_equal(g, w_, err_msg=name)
 
 
+@pytest.mark.parametrize("rv", [0.0, float(np.nextafter(np.float32(1.0), np.float32(0.0)))])
+def test_residual_draw_at_the_ends_of_the_unit_interval(rv):
+    """r = 0 selects the first token of the vocabulary (the smallest v whose cumulative residual is >= 0) and the
+    largest fp32 below 1 the last token that carries residual mass or one next to it; every sequence is made to
+    reject at row 0 (u next to 1 against an alpha far below 1)."""
+    B, k, V = 5, 3, 777
+    cfg = W.StepConfig("r", B, 4, 2, 64, k, 64, V, (0, 0), mode="sample", temperature=1.0, seed=820)
+    ql = W.draft_logits(cfg)
+    zt32 = W.normal(cfg.seed, "zt", (B, k, V), 1.0, dtype=torch.float32).numpy()
+    p0 = np.stack([O.softmax_f64(zt32[b, 0], 1.0) for b in range(B)])
+    q0 = np.stack([O.softmax_f64(ql[b, 0].numpy(), 1.0) for b in range(B)])
+    drafts = np.zeros((B, k), dtype=np.int32)
+    drafts[:, 0] = np.argmax(q0 / p0, axis=1)           # alpha = p/q is smallest there
+    u = torch.full((B, k), 0.999)
+    r = torch.full((B,), rv, dtype=torch.float32)
+    want = O.accept_sample(drafts, zt32, 1.0, ql.numpy(), u.numpy(), r.numpy())
+    assert (want[0] == 0).all()
+    got = _sample(cfg, zt32, ql, drafts, u, r)
+    np.testing.assert_array_equal(got[0], want[0])
+    np.testing.assert_array_equal(got[2], want[2])
+    if rv == 0.0:
+        np.testing.assert_array_equal(got[1], want[1])
+        assert (got[1][:, 0] == 0).all()
+    else:
+        for b in range(B):
+            res, S = O.residual_distribution(p0[b], q0[b])
+            cdf = np.cumsum(res)
+            v = int(got[1][b, 0])
+            assert res[v] > 0 and cdf[v] >= float(np.float32(rv)) * S * (1 - 1e-6), (b, v)
+
+
 def test_sampling_identical_distributions_accept_everything():
     """p == q gives alpha = 1 at every position, so even u next to 1 accepts."""
     cfg = W.StepConfig("z", 2, 4, 2, 64, 2, 64, 500, (0, 0), mode="sample", temperature=1.0, seed=800)

@@ -223,3 +223,65 @@ def test_host_buffer_step_matches_oracle(own_stream):
         assert L.deer_kv_status(kv) == 0
         Hn.kv_state_equal(kv, okv, f"host step {step}")
     Hn.kv_contents_equal(kv, okv, label="host steps")
+
+
+def test_host_buffer_step_notices_a_swapped_device_buffer():
+    """The recorded graph holds every device pointer by value, so a call that differs from the recorded one in a
+    single staging buffer (here the hidden states, then the result arrays) must not replay the old graph: the step
+    has to read the new hidden states and write the new result arrays."""
+    from paper_2512_15176_b200 import binding as L
+    from paper_2512_15176_b200.runner import VerifyStep
+    cfg = W.config(0).with_(growth=64)
+    st = Hn.draw_state(cfg, None, True)
+    kv = Hn.gpu_kv(st)
+    saved = [t.clone() for t in (kv.page_table, kv.seq_len, kv.n_pages, kv.free_stack, kv.free_top)]
+    w = W.lm_head(cfg)
+    w64 = Hn.f64(w)
+    w_dev = w.cuda()
+    msl = int(st.lengths.max()) + 64
+    vs = VerifyStep(cfg, kv, w_dev, msl, store_logits=False)
+    pin = lambda t: t.contiguous().pin_memory()
+    q, kb, vb = Hn.draw_block(cfg, 0, True)
+    hq, hkb, hvb = pin(q), pin(kb), pin(vb)
+    h0, z0, _ = Hn.draw_hidden_with_margin(cfg, w64, 0)
+    h1, z1, _ = Hn.draw_hidden_with_margin(cfg, w64, 1)
+    t0, t1 = (O.select_argmax(z).reshape(cfg.B, cfg.k) for z in (z0, z1))
+    assert (t0 != t1).any()
+    drafts = t0.copy()                       # every row of h0 is accepted in full; against h1 almost nothing is
+    hh, hd = pin(h0), pin(torch.from_numpy(drafts))
+    ha = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
+    ho = torch.empty(cfg.B, cfg.k, dtype=torch.int32).pin_memory()
+    hn = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
+    stream = torch.cuda.Stream()
+
+    def run(h_dev, out_ids_dev):
+        for dst, src in zip((kv.page_table, kv.seq_len, kv.n_pages, kv.free_stack, kv.free_top), saved):
+            dst.copy_(src)
+        torch.cuda.synchronize()
+        sd = L.deer_step_dev(vs.q.data_ptr(), vs.k_blk.data_ptr(), vs.v_blk.data_ptr(), vs.attn_out.data_ptr(), h_dev.data_ptr(),
+                             vs.seq_ids.data_ptr(), vs.draft_ids.data_ptr(), vs.target_ids.data_ptr(), vs.accept_len.data_ptr(),
+                             out_ids_dev.data_ptr(), vs.n_out.data_ptr(), vs.attn_ws.data_ptr(), vs.attn_ws.numel(),
+                             vs.lm_ws.data_ptr(), vs.lm_ws.numel())
+        L.deer_verify_step_host(kv, sd, w_dev, hq, hkb, hvb, hh, hd, cfg.B, cfg.k, cfg.Hq, cfg.hid, cfg.V, vs.scale, msl,
+                                ha, ho, hn, stream=stream)
+        return ha.numpy().copy(), ho.numpy().copy()
+
+    a, out = run(vs.h, vs.out_ids)                      # records a graph
+    want_a, want_out, _ = O.accept_greedy(drafts, t0)
+    np.testing.assert_array_equal(a, want_a)
+    np.testing.assert_array_equal(out, want_out)
+    # same call, other device buffer for the result ids: the old one must stay as it was
+    other_out = torch.full_like(vs.out_ids, -77)
+    vs.out_ids.fill_(-55)
+    torch.cuda.synchronize()
+    a, out = run(vs.h, other_out)
+    np.testing.assert_array_equal(out, want_out)
+    assert (vs.out_ids.cpu().numpy() == -55).all()
+    # same call, other device buffer for the hidden states, new host content
+    hh.copy_(h1)
+    other_h = torch.zeros_like(vs.h)
+    a, out = run(other_h, vs.out_ids)
+    want_a, want_out, _ = O.accept_greedy(drafts, t1)
+    np.testing.assert_array_equal(a, want_a)
+    np.testing.assert_array_equal(out, want_out)
+    assert torch.equal(other_h.cpu(), h1)

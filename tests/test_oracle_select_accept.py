@@ -325,3 +325,68 @@ def test_sampling_bonus_with_one_row_is_plain_sampling():
                 want = v
                 break
         assert out[b, 0] == want
+
+
+# ---------------------------------------------------------------- two corners
+
+def test_inverse_cdf_when_the_cumulative_sum_falls_short_of_the_target():
+    """Hand-built weights whose running sum, rounded term by term, ends below r * total although total is their
+    exact sum: the draw is then the last token that carries weight (trailing zero-weight tokens can never be drawn)."""
+    big, tiny = 1.0, 2.0 ** -54
+    w = np.array([big, tiny, tiny, tiny, tiny, 0.0, 0.0])
+    cdf_end = float(np.cumsum(w)[-1])
+    assert cdf_end == 1.0                              # each tiny term is below half an ulp of 1 and is lost
+    total = math.fsum(w)                               # the exact sum 1 + 2^-52 is representable
+    assert total == 1.0 + 2.0 ** -52 and total > cdf_end
+    assert O.inverse_cdf(w, total, 1.0) == 4           # r * total > cdf[-1]: last index with weight, not 6
+    # the ordinary branch on the same weights
+    assert O.inverse_cdf(w, total, 0.5) == 0
+    assert O.inverse_cdf(w, total, 0.0) == 0
+    # brute force definition on a case without rounding trouble
+    w2 = np.array([0.0, 0.25, 0.0, 0.5, 0.25])
+    for r, want in [(0.0, 0), (0.1, 1), (0.25, 1), (0.26, 3), (0.75, 3), (0.76, 4), (1.0, 4)]:
+        acc, pick = 0.0, None
+        for v, x in enumerate(w2):
+            acc += x
+            if acc >= r * 1.0:
+                pick = v
+                break
+        assert O.inverse_cdf(w2, 1.0, r) == pick == want
+
+
+def test_sampling_with_the_extra_row_and_an_eos_hand_worked():
+    """k = 3 rows = 2 drafts + one more row, vocabulary of 4, worked by hand.
+    Row distributions are chosen so that every acceptance probability is 1 or 0:
+      sequence 0: both drafts have p = q (alpha = 1) -> accepted; the extra row's p = (0.1, 0.2, 0.3, 0.4) and
+                  r = 0.35 picks token 2 (cumulative 0.1, 0.3, 0.6).  Emitted 1, 3, 2.
+      sequence 1: draft 0 accepted; draft 1 = token 0 has p(0) = 0 -> rejected whatever u is; residual of
+                  p = (0, 0.5, 0.5, 0) against q = (0.5, 0.5, 0, 0) is (0, 0, 0.5, 0) -> token 2.  Emitted 2, 2.
+    With eos_id = 3 sequence 0 stops after its second token (the 3): n_out 2, accept_len stays 2; with eos_id = 1
+    it stops after the first: n_out 1 and accept_len is cut to 1.  Sequence 1 never emits 3 or 1."""
+    lg = lambda p: np.log(np.maximum(np.asarray(p, dtype=np.float64), 1e-300))
+    same = [0.25, 0.25, 0.25, 0.25]
+    zt = np.stack([
+        np.stack([lg(same), lg(same), lg([0.1, 0.2, 0.3, 0.4])]),
+        np.stack([lg(same), lg([0.0, 0.5, 0.5, 0.0]), lg(same)]),
+    ])
+    zq = np.stack([
+        np.stack([lg(same), lg(same), lg(same)]),
+        np.stack([lg(same), lg([0.5, 0.5, 0.0, 0.0]), lg(same)]),
+    ])
+    drafts = np.array([[1, 3, 0], [2, 0, 0]], dtype=np.int32)      # column 2 is ignored
+    u = np.full((2, 3), 0.999)
+    r = np.array([0.35, 0.5])
+    a, out, n = O.accept_sample(drafts, zt, 1.0, zq, u, r, eos_id=-1, bonus=True)
+    assert a.tolist() == [2, 1] and n.tolist() == [3, 2]
+    assert out.tolist() == [[1, 3, 2], [2, 2, -1]]
+    a, out, n = O.accept_sample(drafts, zt, 1.0, zq, u, r, eos_id=3, bonus=True)
+    assert a.tolist() == [2, 1] and n.tolist() == [2, 2]
+    assert out.tolist() == [[1, 3, -1], [2, 2, -1]]
+    a, out, n = O.accept_sample(drafts, zt, 1.0, zq, u, r, eos_id=1, bonus=True)
+    assert a.tolist() == [1, 1] and n.tolist() == [1, 2]
+    assert out.tolist() == [[1, -1, -1], [2, 2, -1]]
+    # eos_id = 2: for sequence 0 the extra token itself is the EOS, it is emitted and nothing is cut; sequence 1's
+    # first token (an accepted draft) is the EOS, so its correction is dropped and the accepted draft stays counted
+    a, out, n = O.accept_sample(drafts, zt, 1.0, zq, u, r, eos_id=2, bonus=True)
+    assert a.tolist() == [2, 1] and n.tolist() == [3, 1]
+    assert out.tolist() == [[1, 3, 2], [2, -1, -1]]

@@ -6,11 +6,13 @@ outputs) cannot supply the workspace deer_lmhead_select wants.  The static
 variant keeps that scratch in a fixed array inside the library.  This test
 calls it through the C ABI twice in a row -- the second call finds the first
 call's leftovers in the shared array -- and checks every output against the
-workspace-based entry point.  It is collected last on purpose."""
+workspace-based entry point and against the CPU oracle, and that the device's
+free memory does not move across a call.  It is collected last on purpose."""
 import numpy as np
 import pytest
 import torch
 
+from oracle import deer_oracle as O
 from paper_2512_15176_b200 import workload as W
 
 pytestmark = pytest.mark.gpu
@@ -36,9 +38,22 @@ def test_static_scratch_matches_workspace_entry_point_twice():
         ws = torch.empty(L.deer_lmhead_workspace_bytes(M, hid, V), dtype=torch.uint8, device=dev)
         L.deer_lmhead_select(h, w, mode, T, drafts, ids_a, None, lse_a, dl_a, z_a, ws)
         torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
+        reserved_before = torch.cuda.memory_reserved()
         L.deer_lmhead_select_static(h, w, mode, T, drafts, ids_b, None, lse_b, dl_b, z_b)
         torch.cuda.synchronize()
+        if call > 0:       # the very first call on a device resolves the array's address; later ones touch no allocator
+            assert torch.cuda.mem_get_info()[0] == free_before and torch.cuda.memory_reserved() == reserved_before
         assert torch.equal(ids_a, ids_b)
+        # and against the oracle on the same inputs
+        z64 = O.lm_logits(h.cpu().to(torch.float64).numpy(), w.cpu().to(torch.float64).numpy())
+        want_ids = O.select_argmax(z64)
+        got_ids = ids_b.cpu().numpy()
+        differ = np.flatnonzero(got_ids != want_ids)
+        assert (O.top2_gap(z64[differ]) < 1e-3).all()
+        np.testing.assert_allclose(lse_b.cpu().numpy(), O.logsumexp(z64, float(np.float32(T))), atol=3e-4, rtol=0)
+        np.testing.assert_allclose(dl_b.cpu().numpy(), z64[np.arange(M), drafts.cpu().numpy()], atol=1e-3, rtol=0)
+        np.testing.assert_allclose(z_b.cpu().numpy(), z64, atol=1e-3, rtol=0)
         assert not torch.isnan(lse_b).any() and not torch.isnan(z_b).any()
         np.testing.assert_allclose(lse_b.cpu().numpy(), lse_a.cpu().numpy(), atol=3e-4, rtol=0)
         np.testing.assert_allclose(dl_b.cpu().numpy(), dl_a.cpu().numpy(), atol=1e-3, rtol=0)
@@ -54,6 +69,35 @@ def test_static_scratch_matches_workspace_entry_point_twice():
     torch.cuda.synchronize()
     assert torch.equal(ids_a, ids_b)
     np.testing.assert_allclose(mlp_b.cpu().numpy(), mlp_a.cpu().numpy(), atol=2e-4, rtol=0)
+    z64 = O.lm_logits(h.cpu().to(torch.float64).numpy(), w.cpu().to(torch.float64).numpy())
+    np.testing.assert_allclose(mlp_b.cpu().numpy(), O.max_logprob(z64), atol=2e-4, rtol=0)
+
+
+def test_static_scratch_first_call_inside_a_capture_is_refused_or_already_resolved():
+    """On a device whose array address is still unknown, a call on a capturing stream must refuse (the look-up is not
+    a capturable operation); once an earlier call has resolved it -- the case when the test above ran first -- the
+    same call is simply recorded.  Either way the capture survives."""
+    from paper_2512_15176_b200 import binding as L
+    dev = "cuda"
+    M, hid, V = 8, 64, 128
+    h = W.normal(4243, "h", (M, hid), 1.0).to(dev)
+    w = W.normal(4243, "w", (V, hid), 0.05).to(dev)
+    ids = torch.full((M,), -5, dtype=torch.int32, device=dev)
+    st = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    refused = False
+    with torch.cuda.graph(g, stream=st):
+        try:
+            L.deer_lmhead_select_static(h, w, L.DEER_SEL_ARGMAX, 1.0, None, ids, None, None, None, None)
+        except L.DeerError as e:
+            assert e.code == L.DEER_ERR_UNSUPPORTED
+            refused = True
+    if not refused:
+        g.replay()
+        torch.cuda.synchronize()
+        z64 = O.lm_logits(h.cpu().to(torch.float64).numpy(), w.cpu().to(torch.float64).numpy())
+        assert (ids.cpu().numpy() == O.select_argmax(z64)).all()
 
 
 def test_static_scratch_rejects_more_rows_than_it_holds():
