@@ -20,6 +20,11 @@ import numpy as np
 MASK_CAUSAL = 0
 MASK_BIDIR = 1
 
+# states of a block row in the drafter's partially filled block (block_attention's row_state)
+ROW_ABSENT = -1      # no token there: neither a query nor a key
+ROW_DECODED = 0      # a fixed token: context for the rows that are still masked
+ROW_MASKED = 1       # still a mask token: to be (re-)filled
+
 
 # --------------------------------------------------------------------------
 # paged cache access
@@ -41,12 +46,43 @@ def gather_prefix(pool, page_table_row, n, page_size):
 #     (bidirectional inside the block).
 # --------------------------------------------------------------------------
 
-def block_attention(q, k_blk, v_blk, k_pool, v_pool, page_table, seq_len, seq_ids, mask, scale, page_size=16):
+def block_visibility(k, mask, row_state=None):
+    """allowed[i, j]: may block row i see block row j?  Causal: j <= i.  Bidirectional: every j.  Bidirectional
+    with row states (the drafter's block while it is being filled over several iterations, Section 4 "Generative
+    capabilities"; the drafter-side cache the appendix on the DLLM KV cache looks forward to): a masked row sees
+    every row that holds something (decoded or masked -- the joint fill of Section 3.2); a decoded row sees the
+    decoded rows only, so that what is computed for it never depends on positions that may still change and can
+    be kept as context; an absent row sees nothing and nobody sees it."""
+    allowed = np.ones((k, k), dtype=bool)
+    if mask == MASK_CAUSAL:
+        if row_state is not None:
+            raise ValueError("row states belong to the bidirectional (drafter) mask")
+        for i in range(k):
+            allowed[i, i + 1:] = False
+        return allowed
+    if row_state is None:
+        return allowed
+    st = np.asarray(row_state)
+    for i in range(k):
+        for j in range(k):
+            if st[i] == ROW_MASKED:
+                allowed[i, j] = st[j] != ROW_ABSENT
+            elif st[i] == ROW_DECODED:
+                allowed[i, j] = st[j] == ROW_DECODED
+            else:
+                allowed[i, j] = False
+    return allowed
+
+
+def block_attention(q, k_blk, v_blk, k_pool, v_pool, page_table, seq_len, seq_ids, mask, scale, page_size=16,
+                    row_state=None):
     """q [B,k,Hq,D]; k_blk,v_blk [B,k,Hkv,D]; pools [P,Hkv,page,D] -> [B,k,Hq,D] float64.
 
     Row i of sequence b attends to its committed prefix (cache tokens
     0..n_b-1) and to block rows j with j <= i (causal) or all j (bidirectional).
-    Query head h reads KV head h // (Hq/Hkv)."""
+    Query head h reads KV head h // (Hq/Hkv).
+    row_state [B,k] (bidirectional only): see block_visibility; the output rows of
+    absent positions are zero."""
     q = np.asarray(q, dtype=np.float64)
     k_blk = np.asarray(k_blk, dtype=np.float64)
     v_blk = np.asarray(v_blk, dtype=np.float64)
@@ -62,16 +98,17 @@ def block_attention(q, k_blk, v_blk, k_pool, v_pool, page_table, seq_len, seq_id
         keys = np.concatenate([kp, k_blk[b]], axis=0)       # [n+k, Hkv, D]
         vals = np.concatenate([vp, v_blk[b]], axis=0)
         allowed = np.ones((k, n + k), dtype=bool)
-        if mask == MASK_CAUSAL:
-            for i in range(k):
-                allowed[i, n + i + 1:] = False
+        allowed[:, n:] = block_visibility(k, mask, None if row_state is None else row_state[b])
+        present = np.ones(k, dtype=bool) if row_state is None else np.asarray(row_state[b]) != ROW_ABSENT
+        allowed[~present] = True                      # computed like any row, then zeroed: nothing is defined there
         for h in range(Hq):
             g = h // G
             sc = scale * (q[b, :, h, :] @ keys[:, g, :].T)  # [k, n+k]
             sc = np.where(allowed, sc, -np.inf)
             m = sc.max(axis=1, keepdims=True)
             w = np.exp(sc - m)
-            out[b, :, h, :] = (w @ vals[:, g, :]) / w.sum(axis=1, keepdims=True)
+            o = (w @ vals[:, g, :]) / w.sum(axis=1, keepdims=True)
+            out[b, :, h, :] = np.where(present[:, None], o, 0.0)
     return out
 
 
@@ -180,8 +217,37 @@ def inverse_cdf(weights, total, r):
     return v
 
 
-def accept_sample(draft_ids, target_logits, temperature, draft_logits, u, r, eos_id=-1, bonus=False):
+def truncate_distribution(p, top_k=0, top_p=1.0):
+    """Top-k / nucleus truncation of a probability vector, as samplers apply it to the verifier's distribution at
+    temperature > 0 (the setting of the paper's Table 1 is a temperature; the truncations are the usual
+    companions).  Both are upper level sets of p, so that tokens of equal probability are kept or dropped together:
+      top_k > 0:  keep {v : p[v] >= the top_k-th largest value of p};
+      top_p < 1:  on what is left, renormalised, walk the distinct values downwards, whole tie groups at a time,
+                  and stop after the first group with which the accumulated mass reaches top_p.
+    Returns (the kept part renormalised to sum 1, the boolean keep mask)."""
+    p = np.asarray(p, dtype=np.float64)
+    V = p.shape[0]
+    keep = np.ones(V, dtype=bool)
+    if top_k and 0 < top_k < V:
+        kth = np.sort(p)[V - top_k]
+        keep &= p >= kth
+    if top_p < 1.0:
+        pk = np.where(keep, p, 0.0)
+        pk = pk / pk.sum()
+        order = np.argsort(-pk, kind="stable")
+        cum = np.cumsum(pk[order])
+        first = int(np.searchsorted(cum, top_p, side="left"))        # first position where the running mass >= top_p
+        first = min(first, V - 1)
+        keep &= pk >= pk[order[first]]
+    out = np.where(keep, p, 0.0)
+    return out / out.sum(), keep
+
+
+def accept_sample(draft_ids, target_logits, temperature, draft_logits, u, r, eos_id=-1, bonus=False, top_k=0, top_p=1.0):
     """Speculative rejection sampling over one block per sequence.
+
+    top_k / top_p: p below is softmax(target_logits / T) after truncate_distribution, so the rule is lossless with
+    respect to the truncated verifier distribution; a draft token outside it has alpha = 0.
 
     For i = 0..k-1: p = softmax(target_logits[b,i] / T), q = softmax(draft_logits[b,i]);
     alpha_i = min(1, p[y_i] / q[y_i]) (Eq. 5); accept iff u[b,i] <= alpha_i.  At the
@@ -197,6 +263,7 @@ def accept_sample(draft_ids, target_logits, temperature, draft_logits, u, r, eos
     draft_ids = np.asarray(draft_ids)
     B, k = draft_ids.shape
     kd = k - 1 if bonus else k
+    truncated = bool(top_k) or top_p < 1.0
     accept_len = np.zeros(B, dtype=np.int32)
     out_ids = np.full((B, k), -1, dtype=np.int32)
     n_out = np.zeros(B, dtype=np.int32)
@@ -209,6 +276,10 @@ def accept_sample(draft_ids, target_logits, temperature, draft_logits, u, r, eos
             zq = np.asarray(draft_logits[b, i], dtype=np.float64)
             logp = zp - (zp.max() + np.log(np.exp(zp - zp.max()).sum()))
             logq = zq - (zq.max() + np.log(np.exp(zq - zq.max()).sum()))
+            if truncated:
+                p, _ = truncate_distribution(np.exp(logp), top_k, top_p)
+                with np.errstate(divide="ignore"):
+                    logp = np.log(p)                       # -inf outside the kept set
             log_alpha = min(0.0, logp[y] - logq[y])
             if np.log(np.float64(u[b, i])) <= log_alpha:
                 out_ids[b, i] = y
@@ -226,6 +297,8 @@ def accept_sample(draft_ids, target_logits, temperature, draft_logits, u, r, eos
             break
         if bonus and a == kd:
             p = softmax_f64(target_logits[b, kd], temperature)
+            if truncated:
+                p, _ = truncate_distribution(p, top_k, top_p)
             out_ids[b, kd] = inverse_cdf(p, p.sum(), float(r[b]))
             n += 1
         n, a = _truncate_at_eos(out_ids[b], n, a, eos_id)
@@ -273,12 +346,16 @@ class PagedKV:
                 self.n_pages[s] += 1
         return True
 
-    def append(self, seq_ids, k_blk, v_blk):
-        """Write block rows at token positions seq_len .. seq_len+k-1 (lengths unchanged)."""
+    def append(self, seq_ids, k_blk, v_blk, row_state=None):
+        """Write block rows at token positions seq_len .. seq_len+k-1 (lengths unchanged).  With row states only the
+        decoded rows are written (row i still goes to position seq_len + i): a masked or absent position has no
+        keys and values worth keeping."""
         B, k = k_blk.shape[0], k_blk.shape[1]
         for b in range(B):
             s = int(seq_ids[b])
             for i in range(k):
+                if row_state is not None and row_state[b][i] != ROW_DECODED:
+                    continue
                 t = int(self.seq_len[s]) + i
                 pg = self.page_table[s, t // self.page_size]
                 self.k_pool[pg, :, t % self.page_size, :] = k_blk[b, i]
@@ -331,6 +408,7 @@ class DecodeState:
         that token's, followed by the accepted drafts'."""
         B = self.tokens.shape[0]
         keep = np.zeros(B, dtype=np.int32)
+        self.appended = np.zeros(B, dtype=np.int32)        # tokens that joined each sequence's output in this pass
         for b in range(B):
             if self.finished[b]:
                 continue
@@ -339,6 +417,7 @@ class DecodeState:
             for i in range(m):
                 self.tokens[b, self.n_tokens[b] + i] = out_ids[b][i]
             self.n_tokens[b] += m
+            self.appended[b] = m
             keep[b] = min(int(accept_len[b]), m) + (1 if pending else 0)
             hit_eos = eos_id >= 0 and any(int(out_ids[b][i]) == eos_id for i in range(m))
             if hit_eos or self.n_tokens[b] >= self.max_new:
@@ -386,3 +465,95 @@ def swiglu(gate, up):
     """SiLU(gate) * up with SiLU(g) = g / (1 + exp(-g))."""
     g = np.asarray(gate, dtype=np.float64)
     return g / (1.0 + np.exp(-g)) * np.asarray(up, dtype=np.float64)
+
+
+# --------------------------------------------------------------------------
+# (7) The drafter's side of the loop beyond the single-step fill.
+#     Section 4 ("Generative capabilities") shows the drafter completing a block
+#     over several denoising iterations; the appendix on the DLLM KV cache points
+#     to block-wise caches for diffusion models (confidence-gated parallel
+#     decoding inside a block, the finished block's keys and values kept as
+#     context).  The paper gives neither rule a formula; the ones below are the
+#     published block-diffusion decoding rules it points to, reduced to what the
+#     attention and cache calls need.
+# --------------------------------------------------------------------------
+
+def refill_step(row_state, tokens, ids, logprob, log_threshold):
+    """One iteration of a block re-fill.  For each sequence: every row that is still
+    masked and whose most likely token (ids) has log-probability (logprob) >=
+    log_threshold becomes decoded with that token; if no masked row qualifies, the
+    most confident masked row does (lowest row on ties), so each iteration decodes
+    at least one row while any is masked.  Decoded and absent rows keep their
+    state and token.  Returns (row_state', tokens', masked rows left per sequence).
+    log_threshold = -inf decodes everything at once: the single-step block draft."""
+    st = np.array(row_state, dtype=np.int32)
+    tok = np.array(tokens, dtype=np.int32)
+    B, k = st.shape
+    left = np.zeros(B, dtype=np.int32)
+    for b in range(B):
+        masked = [i for i in range(k) if st[b, i] == ROW_MASKED]
+        if not masked:
+            continue
+        chosen = [i for i in masked if logprob[b][i] >= log_threshold]
+        if not chosen:
+            best = masked[0]
+            for i in masked[1:]:
+                if logprob[b][i] > logprob[b][best]:
+                    best = i
+            chosen = [best]
+        for i in chosen:
+            st[b, i] = ROW_DECODED
+            tok[b, i] = ids[b][i]
+        left[b] = len(masked) - len(chosen)
+    return st, tok, left
+
+
+def refresh_rows(appended, k):
+    """Row states of the pass that brings the drafter's cache up to date after a
+    verify step: the `appended[b]` tokens that joined sequence b's output are
+    decoded rows (they see each other and the drafter's prefix, and their keys and
+    values are written to its cache); the rest of the block is absent."""
+    appended = np.asarray(appended)
+    st = np.full((appended.shape[0], k), ROW_ABSENT, dtype=np.int32)
+    for b in range(appended.shape[0]):
+        st[b, :int(appended[b])] = ROW_DECODED
+    return st
+
+
+# --------------------------------------------------------------------------
+# (8) Routed mixture-of-experts MLP of a Qwen3-MoE-style verifier layer (the
+#     paper's largest verifier, Qwen3-30B-A3B, has one in every layer): a linear
+#     router, softmax over the experts, the top_k experts of each row with their
+#     probabilities renormalised to sum 1, each expert a SiLU-gated MLP, the
+#     weighted sum of their outputs.
+# --------------------------------------------------------------------------
+
+def moe_route(x, w_router, top_k, renormalise=True):
+    """x [M,hid], w_router [E,hid] -> (experts [M,top_k] int32, weights [M,top_k] float64), each row's experts in
+    order of decreasing probability (lower index first among equals)."""
+    logits = np.asarray(x, dtype=np.float64) @ np.asarray(w_router, dtype=np.float64).T
+    logits = logits - logits.max(axis=1, keepdims=True)
+    prob = np.exp(logits)
+    prob = prob / prob.sum(axis=1, keepdims=True)
+    order = np.argsort(-prob, axis=1, kind="stable")[:, :top_k]
+    wts = np.take_along_axis(prob, order, axis=1)
+    if renormalise:
+        wts = wts / wts.sum(axis=1, keepdims=True)
+    return order.astype(np.int32), wts
+
+
+def moe_mlp(x, w_router, w_gate_up, w_down, top_k, renormalise=True):
+    """x [M,hid]; w_router [E,hid]; w_gate_up [E,2I,hid] (gate rows first, then up rows); w_down [E,hid,I]
+    -> y [M,hid] = sum_j weight_j * down_e(silu(gate_e(x)) * up_e(x)) over the row's top_k experts e."""
+    x = np.asarray(x, dtype=np.float64)
+    experts, wts = moe_route(x, w_router, top_k, renormalise)
+    E, twoI, hid = np.asarray(w_gate_up).shape
+    inter = twoI // 2
+    y = np.zeros_like(x)
+    for m in range(x.shape[0]):
+        for j in range(top_k):
+            e = int(experts[m, j])
+            gu = linear(x[m:m + 1], w_gate_up[e])[0]
+            act = swiglu(gu[:inter], gu[inter:])
+            y[m] += wts[m, j] * linear(act[None, :], w_down[e])[0]
+    return y

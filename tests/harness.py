@@ -98,11 +98,22 @@ def check_logits(got_f32, z64, label=""):
     assert err.max() <= 1e-3, f"{label}: logits err max {err.max():.3e} (expected ~1e-5)"
 
 
-def sampling_inputs(cfg, zt32, step=0, r_margin=1e-9, bonus=False):
+R_MARGIN = 1e-4           # r * S keeps this fraction of S away from the edges of the drawn token's cell
+
+
+def truncated_p(z32_row, T, top_k, top_p):
+    p = O.softmax_f64(z32_row, T)
+    if top_k or top_p < 1.0:
+        p, _ = O.truncate_distribution(p, top_k, top_p)
+    return p
+
+
+def sampling_inputs(cfg, zt32, step=0, r_margin=R_MARGIN, bonus=False, top_k=0, top_p=1.0):
     """Drafter logits, sampled drafts, uniforms with cleared margins.
     ``zt32`` are the target logits (fp32 values, [B,k,V]) the oracle will use.
     bonus: the last row holds no draft; when the k-1 drafts before it are all
-    accepted, r is cleared against the edges of that row's own CDF."""
+    accepted, r is cleared against the edges of that row's own CDF.
+    top_k / top_p: the verifier's distribution is truncated first."""
     T = float(np.float32(cfg.temperature))
     ql = W.draft_logits(cfg, step)
     drafts = W.sample_drafts(ql, cfg.seed, step)
@@ -130,12 +141,17 @@ def sampling_inputs(cfg, zt32, step=0, r_margin=1e-9, bonus=False):
             y = int(drafts[b, i])
             zp = zt32[b, i].astype(np.float64) / T
             zq = qn[b, i].astype(np.float64)
-            la = min(0.0, (zp[y] - O.logsumexp(zp[None], 1.0)[0]) - (zq[y] - O.logsumexp(zq[None], 1.0)[0]))
+            if top_k or top_p < 1.0:
+                py = truncated_p(zt32[b, i], T, top_k, top_p)[y]
+                logp_y = math.log(py) if py > 0 else -math.inf
+            else:
+                logp_y = zp[y] - O.logsumexp(zp[None], 1.0)[0]
+            la = min(0.0, logp_y - (zq[y] - O.logsumexp(zq[None], 1.0)[0]))
             while abs(math.log(float(u[b, i])) - la) < ALPHA_MARGIN:
                 u[b, i] = np.float32((int(gen.integers(0, 1 << 24)) + 0.5) / (1 << 24))
                 redraws += 1
             if math.log(float(u[b, i])) > la:          # first rejection: clear r against the residual CDF edges
-                p = O.softmax_f64(zt32[b, i], T)
+                p = truncated_p(zt32[b, i], T, top_k, top_p)
                 qd = O.softmax_f64(qn[b, i], 1.0)
                 res, S = O.residual_distribution(p, qd)
                 wts, tot = (res, S) if S > 0 else (p, p.sum())
@@ -143,7 +159,7 @@ def sampling_inputs(cfg, zt32, step=0, r_margin=1e-9, bonus=False):
                 rejected = True
                 break
         if bonus and not rejected:
-            p = O.softmax_f64(zt32[b, kd], T)
+            p = truncated_p(zt32[b, kd], T, top_k, top_p)
             clear_r(b, p, p.sum())
     return ql, drafts, torch.from_numpy(u), torch.from_numpy(r), redraws
 
@@ -179,3 +195,22 @@ def kv_contents_equal(kv, okv, seqs=None, label=""):
         ok, ov = okv.gather(s)
         np.testing.assert_array_equal(gk, ok, err_msg=f"{label} K contents seq {s}")
         np.testing.assert_array_equal(gv, ov, err_msg=f"{label} V contents seq {s}")
+
+
+def nucleus_margin_ok(z32, T, top_k, top_p, margin=1e-4):
+    """True if, for every row of z32 [M,V], the running mass of the (top-k-renormalised) distribution keeps `margin`
+    away from top_p on both sides of the tie group at which it is reached -- so that summation order cannot move
+    the nucleus's edge."""
+    for row in z32:
+        p = O.softmax_f64(row, T)
+        if top_k:
+            p, _ = O.truncate_distribution(p, top_k, 1.0)
+        vals = np.sort(p[p > 0])[::-1]
+        cum = np.cumsum(vals)
+        i = min(int(np.searchsorted(cum, top_p, side="left")), len(vals) - 1)
+        lo = np.flatnonzero(vals == vals[i])
+        before = cum[lo[0] - 1] if lo[0] > 0 else 0.0
+        incl = cum[lo[-1]]
+        if top_p - before < margin or (incl - top_p < margin and lo[-1] < len(vals) - 1):
+            return False
+    return True

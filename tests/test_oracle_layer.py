@@ -64,3 +64,64 @@ def test_swiglu_values():
     np.testing.assert_allclose(O.swiglu(g, u), want, rtol=1e-14, atol=1e-300)
     t = torch.nn.functional.silu(torch.from_numpy(g)) * torch.from_numpy(u)
     np.testing.assert_allclose(O.swiglu(g, u), t.numpy(), rtol=1e-13)
+
+
+# ---------------------------------------------------------------- routed mixture of experts
+
+def _moe_case(seed, M=5, hid=6, E=4, inter=3):
+    r = np.random.default_rng(seed)
+    return (r.normal(size=(M, hid)), r.normal(size=(E, hid)), r.normal(size=(E, 2 * inter, hid)) * 0.5,
+            r.normal(size=(E, hid, inter)) * 0.5)
+
+
+def test_moe_router_against_scalar_loops():
+    x, wr, _, _ = _moe_case(0)
+    experts, wts = O.moe_route(x, wr, 2)
+    for m in range(x.shape[0]):
+        logit = [sum(x[m, c] * wr[e, c] for c in range(x.shape[1])) for e in range(4)]
+        mx = max(logit)
+        ex = [math.exp(v - mx) for v in logit]
+        prob = [v / sum(ex) for v in ex]
+        order = sorted(range(4), key=lambda e: (-prob[e], e))[:2]
+        assert experts[m].tolist() == order
+        tot = prob[order[0]] + prob[order[1]]
+        np.testing.assert_allclose(wts[m], [prob[order[0]] / tot, prob[order[1]] / tot], atol=1e-14)
+    # without renormalisation the weights are the softmax probabilities themselves
+    _, raw = O.moe_route(x, wr, 2, renormalise=False)
+    assert (raw.sum(axis=1) < 1.0).all()
+    # ties go to the lower expert index
+    e, w = O.moe_route(np.ones((1, 2)), np.array([[1.0, 0.0], [0.0, 1.0], [0.5, 0.5]]), 2)
+    assert e[0].tolist() == [0, 1] and abs(w[0, 0] - 0.5) < 1e-15
+
+
+def test_moe_mlp_against_scalar_loops_and_special_cases():
+    x, wr, wgu, wd = _moe_case(1)
+    M, hid = x.shape
+    E, twoI, _ = wgu.shape
+    inter = twoI // 2
+    y = O.moe_mlp(x, wr, wgu, wd, 2)
+    experts, wts = O.moe_route(x, wr, 2)
+    for m in range(M):
+        acc = [0.0] * hid
+        for j in range(2):
+            e = int(experts[m, j])
+            g = [sum(x[m, c] * wgu[e, i, c] for c in range(hid)) for i in range(inter)]
+            u = [sum(x[m, c] * wgu[e, inter + i, c] for c in range(hid)) for i in range(inter)]
+            a = [g[i] / (1.0 + math.exp(-g[i])) * u[i] for i in range(inter)]
+            for o in range(hid):
+                acc[o] += wts[m, j] * sum(a[i] * wd[e, o, i] for i in range(inter))
+        np.testing.assert_allclose(y[m], acc, atol=1e-12)
+    # one expert with weight 1 is the dense gated MLP
+    dense = O.linear(O.swiglu(O.linear(x, wgu[2])[:, :inter], O.linear(x, wgu[2])[:, inter:]), wd[2])
+    np.testing.assert_allclose(O.moe_mlp(x, wr[2:3], wgu[2:3], wd[2:3], 1), dense, atol=1e-12)
+    # identical experts: the routing does not matter, the weights sum to one
+    same_gu, same_d = np.repeat(wgu[:1], E, axis=0), np.repeat(wd[:1], E, axis=0)
+    dense0 = O.linear(O.swiglu(O.linear(x, wgu[0])[:, :inter], O.linear(x, wgu[0])[:, inter:]), wd[0])
+    np.testing.assert_allclose(O.moe_mlp(x, wr, same_gu, same_d, 3), dense0, atol=1e-12)
+    # all experts chosen without renormalisation: the full softmax mixture
+    full = O.moe_mlp(x, wr, wgu, wd, E, renormalise=False)
+    prob = np.exp(x @ wr.T)
+    prob /= prob.sum(axis=1, keepdims=True)
+    mix = sum(prob[:, e:e + 1] * O.linear(O.swiglu(O.linear(x, wgu[e])[:, :inter], O.linear(x, wgu[e])[:, inter:]), wd[e])
+              for e in range(E))
+    np.testing.assert_allclose(full, mix, atol=1e-12)
