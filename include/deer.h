@@ -218,7 +218,10 @@ int deer_lmhead_select_static(const void* h, const void* w, int M, int hid, int 
  * SAMPLE: alpha_i = min(1, p(y_i)/q(y_i)), p = softmax(target_logits/T),
  *   q = softmax(draft_logits); accept iff u[b][i] <= alpha_i; at the first
  *   rejection one token is drawn from max(0, p - q) normalised, by inverse CDF
- *   in vocabulary order with r[b] (fp64 sums); if that mass is zero, from p.
+ *   in vocabulary order with r[b]; if that mass is zero, from p.  (p and q are
+ *   taken as fp32 exponentials of logit - log-sum-exp, their differences summed
+ *   in fp64: the draw equals an exact evaluation's whenever r * S stays 1e-4 * S
+ *   away from the edges of the drawn token's interval of the cumulative sum S.)
  * No extra token is emitted when all k are accepted (Algorithm 1 as printed).
  * With DEER_ACC_BONUS or-ed into the mode the block's k rows are k-1 drafts
  * followed by one more row whose input was the last draft: column k-1 of
@@ -257,6 +260,37 @@ int deer_accept(int mode, int B, int k, int V,
                 void* workspace, size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------
+ * Top-k / nucleus truncation of the verifier's distribution ahead of the
+ * acceptance rule (the sampling setting of Table 1 is a temperature; these are
+ * its usual companions).  For every row of target_logits, p = softmax(z / T):
+ *   top_k > 0:  keep {v : p[v] >= the top_k-th largest value of p};
+ *   top_p < 1:  of what is left, renormalised, the smallest upper level set
+ *               {v : p[v] >= t} whose mass reaches top_p.
+ * Both are level sets, so tokens of equal probability stay or go together and the
+ * result is one threshold per row: tau[m], the smallest kept logit (token v is
+ * kept iff z[v] >= tau[m]), and lse_trunc[m] = log sum_{kept} exp(z[v] / T), the
+ * log-sum-exp that normalises the kept part.  deer_accept_truncated() then runs
+ * Eq. 5 / Eq. 6 on that truncated distribution: a draft outside it is rejected,
+ * the residual is max(0, p' - q) with p' the truncated, renormalised p.
+ *   target_logits f32 [M][V];  target_lse f32 [M] = logsumexp(z / T) (deer_lmhead_select's out_lse)
+ *   tau, lse_trunc f32 [M]     out
+ * top_k <= 0 or >= V and top_p >= 1 switch the respective truncation off.
+ * No workspace.  Errors: DEER_ERR_INVALID_ARG for null / misaligned pointers,
+ * temperature <= 0 or top_p <= 0.
+ * ---------------------------------------------------------------------- */
+int deer_truncate(int M, int V, const float* target_logits, const float* target_lse, float temperature, int top_k,
+                  float top_p, float* tau, float* lse_trunc, void* stream);
+
+/* deer_accept on a truncated verifier distribution: target_tau f32 [B][k] (deer_truncate's tau) or NULL (= deer_accept),
+ * and target_lse must then be deer_truncate's lse_trunc.  SAMPLE modes only use target_tau. */
+int deer_accept_truncated(int mode, int B, int k, int V,
+                          const int32_t* draft_ids, const int32_t* target_ids,
+                          const float* target_logits, const float* target_lse, const float* target_draft_logit,
+                          const float* target_tau, float temperature, const float* draft_logits, const float* u,
+                          const float* r, int32_t eos_id, int32_t* accept_len, int32_t* out_ids, int32_t* n_out,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------
  * (5) Book-keeping of one pass of Algorithm 1's outer loop (it runs until an
  * EOS is emitted: the tokens chosen in this block join the output, then j is
  * updated).  For every sequence that has not finished:
@@ -274,10 +308,50 @@ int deer_accept(int mode, int B, int k, int V,
  *   n_tokens  i32 [B]           their number           (caller zeroes it before the first pass)
  *   finished  i32 [B]           0 / 1                  (caller zeroes it before the first pass)
  *   keep      i32 [B]           out
+ *   appended  i32 [B] or NULL   out: tokens that joined tokens[b] in this pass (what the drafter's cache has to
+ *                               take in, see deer_refresh_rows)
  * ---------------------------------------------------------------------- */
 int deer_emit(int B, int k, const int32_t* accept_len, const int32_t* out_ids, const int32_t* n_out,
               int32_t eos_id, int32_t max_new, int32_t* tokens, int32_t* n_tokens, int32_t* finished,
-              int32_t* keep, int flags, void* stream);
+              int32_t* keep, int32_t* appended, int flags, void* stream);
+
+/* ------------------------------------------------------------------------
+ * The drafter's block beyond the single-step fill (Section 4, "Generative
+ * capabilities": a block completed over several denoising iterations; the
+ * appendix on the DLLM KV cache: a drafter-side cache of the finished tokens).
+ * The paper gives no formulas for either; these are the block-diffusion
+ * decoding rules it points to, cut down to what attention and cache need.
+ *
+ * Row states (i32 [B][k], bidirectional mask only):
+ *    1  masked   still a mask token: sees the prefix and every row that holds something
+ *    0  decoded  a fixed token: sees the prefix and the decoded rows only, so that
+ *                nothing computed for it depends on rows that may still change
+ *   -1  absent   holds nothing: no key, no query (its output row is unspecified)
+ * deer_block_attn_rows is deer_block_attn with such states (NULL = all rows
+ * masked = deer_block_attn).  With append = 1 only the decoded rows' keys and
+ * values are written, row i at token position n_b + i as always; the caller
+ * commits as many leading rows as are decoded.
+ *
+ * deer_refill: one iteration's decision.  Every masked row whose most likely
+ * token ids[b][i] has log-probability logprob[b][i] >= log_threshold becomes
+ * decoded and tokens[b][i] = ids[b][i]; if a sequence has masked rows but none
+ * qualifies, its most confident masked row does (the lowest row among equals).
+ * left[b] (optional) = rows still masked.  log_threshold = -INFINITY decodes all
+ * at once (the single-step draft of Section 3.2).
+ *
+ * deer_refresh_rows: row_state[b][i] = 0 for i < appended[b], else -1 -- the
+ * states of the pass that brings the drafter's cache up to date after a verify
+ * step: the tokens that joined the output see each other and the drafter's
+ * prefix, their keys and values are appended, and deer_kv_commit(keep =
+ * appended) on the drafter's cache keeps them.
+ * ---------------------------------------------------------------------- */
+int deer_block_attn_rows(deer_kv* kv, const int32_t* seq_ids,
+                         const void* q, const void* k_blk, const void* v_blk, void* out, const int32_t* row_state,
+                         int B, int k, int Hq, int mask, int append, float scale, int max_seq_len,
+                         void* workspace, size_t workspace_bytes, void* stream);
+int deer_refill(int B, int k, const int32_t* ids, const float* logprob, float log_threshold,
+                int32_t* row_state, int32_t* tokens, int32_t* left, void* stream);
+int deer_refresh_rows(int B, int k, const int32_t* appended, int32_t* row_state, void* stream);
 
 /* ------------------------------------------------------------------------
  * (6) The rest of a verifier layer around the block attention.  The paper takes
@@ -317,6 +391,26 @@ int deer_qkv_split_norm_rope(deer_kv* kv, const int32_t* seq_ids, const void* qk
                              const void* q_gamma, const void* k_gamma, int B, int k, int Hq, float eps, float theta,
                              void* stream);
 int deer_swiglu(const void* gate_up, void* y, int M, int I, void* stream);
+
+/* The routed mixture-of-experts MLP of a Qwen3-MoE-style layer (the paper's largest verifier, Qwen3-30B-A3B, has one
+ * in every layer) at M = B k rows:
+ *   probabilities = softmax(x w_router^T) over the E experts (fp32);  each row's top_k experts, lowest index among
+ *   equals, their probabilities renormalised to sum 1;
+ *   y[m] = residual[m] + sum_j weight[m][j] * down_e( silu(gate_e(x[m])) * up_e(x[m]) ),  e = expert[m][j].
+ *   x bf16 [M][hid];  w_router bf16 [E][hid];  w_gate_up bf16 [E][2 I][hid] (an expert's I gate rows, then its I up
+ *   rows);  w_down bf16 [E][hid][I];  residual bf16 [M][hid] or NULL;  y bf16 [M][hid].
+ *   E <= 256, top_k <= min(32, E), hid and I multiples of 64.
+ * The rows are regrouped by expert and both projections run as grouped GEMMs that stream each chosen expert's
+ * weights once; gate, up (each rounded to bf16, as a dense layer would store them), the activations and the expert
+ * outputs are bf16, sums fp32.
+ * deer_moe_route is the first stage alone: experts i32 [M][top_k] in order of falling probability, weights f32
+ * [M][top_k] (renormalise = 0: the softmax probabilities themselves).
+ *   workspace  >= deer_moe_workspace_bytes(...) bytes, 16-byte aligned, contents arbitrary. */
+size_t deer_moe_workspace_bytes(int M, int hid, int E, int I, int top_k);
+int deer_moe_route(const void* x, const void* w_router, int M, int hid, int E, int top_k, int renormalise,
+                   int32_t* experts, float* weights, void* stream);
+int deer_moe_mlp(const void* x, const void* w_router, const void* w_gate_up, const void* w_down, const void* residual,
+                 void* y, int M, int hid, int E, int I, int top_k, void* workspace, size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------
  * One whole greedy verify step with HOST inputs and outputs (Algorithm 1, one

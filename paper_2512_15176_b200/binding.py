@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libdeer.so")
 
 DEER_OK = 0
 DEER_ERR_INVALID_ARG, DEER_ERR_UNSUPPORTED, DEER_ERR_NO_PAGES, DEER_ERR_CUDA, DEER_ERR_WORKSPACE, DEER_ERR_BAD_PAGE = 1, 2, 3, 4, 5, 6
+DEER_ERR_TIMEOUT = 7
 DEER_MASK_CAUSAL, DEER_MASK_BIDIR = 0, 1
 DEER_SEL_ARGMAX, DEER_SEL_ARGMAX_LOGPROB, DEER_SEL_SOFTMAX = 0, 1, 2
 DEER_ACC_GREEDY, DEER_ACC_SAMPLE, DEER_ACC_SAMPLE_PRESTATS, DEER_ACC_BONUS = 0, 1, 2, 4
@@ -28,6 +29,8 @@ EXPORTS = [
     "deer_accept_workspace_bytes", "deer_accept", "deer_verify_step_host",
     "deer_lmhead_static_max_rows", "deer_lmhead_select_static", "deer_emit", "deer_draft_stats",
     "deer_linear_workspace_bytes", "deer_linear", "deer_rmsnorm", "deer_qk_norm_rope", "deer_qkv_split_norm_rope", "deer_swiglu",
+    "deer_truncate", "deer_accept_truncated", "deer_block_attn_rows", "deer_refill", "deer_refresh_rows",
+    "deer_moe_workspace_bytes", "deer_moe_route", "deer_moe_mlp",
 ]
 
 
@@ -87,6 +90,10 @@ def lib() -> ctypes.CDLL:
     L.deer_accept.argtypes = [c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_float,
                               c_void_p, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t,
                               c_void_p]
+    L.deer_accept_truncated.argtypes = [c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                        c_float, c_void_p, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_void_p,
+                                        c_size_t, c_void_p]
+    L.deer_truncate.argtypes = [c_int, c_int, c_void_p, c_void_p, c_float, c_int, c_float, c_void_p, c_void_p, c_void_p]
     L.deer_linear_workspace_bytes.restype = c_size_t
     L.deer_linear_workspace_bytes.argtypes = [c_int] * 3
     L.deer_linear.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_size_t, c_void_p]
@@ -98,7 +105,16 @@ def lib() -> ctypes.CDLL:
     L.deer_swiglu.argtypes = [c_void_p, c_void_p, c_int, c_int, c_void_p]
     L.deer_draft_stats.argtypes = [c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
     L.deer_emit.argtypes = [c_int, c_int, c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p,
-                            c_int, c_void_p]
+                            c_void_p, c_int, c_void_p]
+    L.deer_block_attn_rows.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int, c_int,
+                                       c_int, c_int, c_float, c_int, c_void_p, c_size_t, c_void_p]
+    L.deer_refill.argtypes = [c_int, c_int, c_void_p, c_void_p, c_float, c_void_p, c_void_p, c_void_p, c_void_p]
+    L.deer_refresh_rows.argtypes = [c_int, c_int, c_void_p, c_void_p, c_void_p]
+    L.deer_moe_workspace_bytes.restype = c_size_t
+    L.deer_moe_workspace_bytes.argtypes = [c_int] * 5
+    L.deer_moe_route.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p]
+    L.deer_moe_mlp.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_int,
+                               c_void_p, c_size_t, c_void_p]
     L.deer_verify_step_host.argtypes = [c_void_p, POINTER(deer_step_dev), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                         c_void_p, c_int, c_int, c_int, c_int, c_int, c_float, c_int, c_void_p, c_void_p,
                                         c_void_p, c_void_p]
@@ -240,6 +256,23 @@ def deer_accept(mode, B, k, V, draft_ids, target_ids, target_logits, target_lse,
                              _stream(stream)))
 
 
+def deer_truncate(target_logits, target_lse, temperature, top_k, top_p, tau, lse_trunc, stream=None):
+    V = target_logits.shape[-1]
+    M = target_logits.numel() // V
+    _check(lib().deer_truncate(M, V, _ptr(target_logits), _ptr(target_lse), float(temperature), int(top_k), float(top_p),
+                               _ptr(tau), _ptr(lse_trunc), _stream(stream)))
+
+
+def deer_accept_truncated(mode, B, k, V, draft_ids, target_ids, target_logits, target_lse, target_draft_logit, target_tau,
+                          temperature, draft_logits, u, r, eos_id, accept_len, out_ids, n_out, workspace, stream=None):
+    _check(lib().deer_accept_truncated(int(mode), B, k, V, _ptr(draft_ids), _ptr(target_ids), _ptr(target_logits),
+                                       _ptr(target_lse), _ptr(target_draft_logit), _ptr(target_tau), float(temperature),
+                                       _ptr(draft_logits), _ptr(u), _ptr(r), int(eos_id), _ptr(accept_len), _ptr(out_ids),
+                                       _ptr(n_out), _ptr(workspace),
+                                       workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                                       _stream(stream)))
+
+
 def deer_linear_workspace_bytes(M, K, N) -> int:
     return lib().deer_linear_workspace_bytes(M, K, N)
 
@@ -273,15 +306,52 @@ def deer_swiglu(gate_up, y, stream=None):
     _check(lib().deer_swiglu(_ptr(gate_up), _ptr(y), M, I, _stream(stream)))
 
 
+def deer_moe_workspace_bytes(M, hid, E, I, top_k) -> int:
+    return lib().deer_moe_workspace_bytes(M, hid, E, I, top_k)
+
+
+def deer_moe_route(x, w_router, top_k, experts, weights, renormalise=True, stream=None):
+    M, hid = x.shape
+    _check(lib().deer_moe_route(_ptr(x), _ptr(w_router), M, hid, w_router.shape[0], int(top_k), 1 if renormalise else 0,
+                                _ptr(experts), _ptr(weights), _stream(stream)))
+
+
+def deer_moe_mlp(x, w_router, w_gate_up, w_down, y, top_k, workspace, residual=None, stream=None):
+    M, hid = x.shape
+    E, two_i, _ = w_gate_up.shape
+    _check(lib().deer_moe_mlp(_ptr(x), _ptr(w_router), _ptr(w_gate_up), _ptr(w_down), _ptr(residual), _ptr(y), M, hid, E, two_i // 2,
+                              int(top_k), _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
 def deer_draft_stats(B, k, V, draft_ids, draft_logits, workspace, stream=None):
     _check(lib().deer_draft_stats(B, k, V, _ptr(draft_ids), _ptr(draft_logits), _ptr(workspace),
                                   workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
-def deer_emit(accept_len, out_ids, n_out, eos_id, tokens, n_tokens, finished, keep, flags=0, stream=None):
+def deer_emit(accept_len, out_ids, n_out, eos_id, tokens, n_tokens, finished, keep, flags=0, stream=None, appended=None):
     B, k = out_ids.shape
     _check(lib().deer_emit(B, k, _ptr(accept_len), _ptr(out_ids), _ptr(n_out), int(eos_id), tokens.shape[1], _ptr(tokens),
-                           _ptr(n_tokens), _ptr(finished), _ptr(keep), int(flags), _stream(stream)))
+                           _ptr(n_tokens), _ptr(finished), _ptr(keep), _ptr(appended), int(flags), _stream(stream)))
+
+
+def deer_block_attn_rows(kv: KVCache, seq_ids, q, k_blk, v_blk, out, row_state, mask, append, scale, max_seq_len, workspace,
+                         stream=None):
+    B, k, Hq, D = q.shape
+    _check(lib().deer_block_attn_rows(kv.handle, _ptr(seq_ids), _ptr(q), _ptr(k_blk), _ptr(v_blk), _ptr(out), _ptr(row_state),
+                                      B, k, Hq, int(mask), int(append), float(scale), int(max_seq_len), _ptr(workspace),
+                                      workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                                      _stream(stream)))
+
+
+def deer_refill(ids, logprob, log_threshold, row_state, tokens, left=None, stream=None):
+    B, k = row_state.shape
+    _check(lib().deer_refill(B, k, _ptr(ids), _ptr(logprob), float(log_threshold), _ptr(row_state), _ptr(tokens), _ptr(left),
+                             _stream(stream)))
+
+
+def deer_refresh_rows(appended, row_state, stream=None):
+    B, k = row_state.shape
+    _check(lib().deer_refresh_rows(B, k, _ptr(appended), _ptr(row_state), _stream(stream)))
 
 
 def deer_verify_step_host(kv: KVCache, dev: deer_step_dev, w, q_host, k_blk_host, v_blk_host, h_host, draft_ids_host,

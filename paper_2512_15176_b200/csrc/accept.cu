@@ -5,9 +5,9 @@
 // SAMPLE: (a) one streaming pass over the drafter logits for log-sum-exp and
 // the draft token's logit of every block row; (b) a per-sequence scan for the
 // first rejection, log alpha_i = min(0, log p(y_i) - log q(y_i)) against log u;
-// (c) for each rejected sequence the residual max(0, p - q) of that one row in
-// fp64, split over NS thread blocks, then an inverse-CDF search in vocabulary
-// order.  Only (a) touches more than a few rows.
+// (c) for each rejected sequence the residual max(0, p - q) of that one row,
+// split over NS thread blocks, then an inverse-CDF search in vocabulary order.
+// (b) and (c) are one kernel.  Only (a) touches more than a few rows.
 
 #include "common.cuh"
 
@@ -21,6 +21,8 @@ __global__ void accept_greedy_kernel(int B, int k, int kd, const int32_t* __rest
                                      int32_t eos_id, int32_t* __restrict__ accept_len, int32_t* __restrict__ out_ids,
                                      int32_t* __restrict__ n_out) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    pdl_trigger();
+    pdl_wait();
     if (b >= B) return;
     const int32_t* d = draft + (size_t)b * k;
     const int32_t* t = target + (size_t)b * k;
@@ -48,10 +50,15 @@ __global__ void accept_greedy_kernel(int B, int k, int kd, const int32_t* __rest
 template <int THREADS, int DEPTH>
 __global__ void __launch_bounds__(THREADS) draft_row_stats_kernel(int rows, int V, const float* __restrict__ q_logits,
                                                                   const int32_t* __restrict__ draft, float* __restrict__ lse_q,
-                                                                  float* __restrict__ zq_draft) {
+                                                                  float* __restrict__ zq_draft, int* __restrict__ done, int n_done) {
     constexpr int NW = THREADS / 32;
     __shared__ float sm[NW], ss[NW];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    pdl_trigger();
+    pdl_wait();
+    // the arrival counters of the acceptance kernel that follows on this workspace start at zero
+    if (blockIdx.x == 0)
+        for (int j = threadIdx.x; j < n_done; j += THREADS) done[j] = 0;
     for (int row = blockIdx.x; row < rows; row += gridDim.x) {
         const float* z = q_logits + (size_t)row * V;
         float m = -INFINITY, s = 0.f;
@@ -112,59 +119,34 @@ __global__ void __launch_bounds__(THREADS) draft_row_stats_kernel(int rows, int 
     }
 }
 
-// ---------------------------------------------------------------- sample (b)
-// One warp per sequence, lane i = block row i.
-__global__ void __launch_bounds__(128) accept_scan_kernel(int B, int k, int kd, const int32_t* __restrict__ draft,
-                                                          const float* __restrict__ lse_p, const float* __restrict__ zp_draft,
-                                                          float inv_t, const float* __restrict__ lse_q,
-                                                          const float* __restrict__ zq_draft, const float* __restrict__ u,
-                                                          int32_t* __restrict__ accept_len, int32_t* __restrict__ out_ids,
-                                                          int32_t* __restrict__ n_out, int32_t* __restrict__ rej_pos,
-                                                          int32_t* __restrict__ from_p, int32_t* __restrict__ done) {
-    const int b = blockIdx.x * 4 + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (b >= B) return;
-    bool acc = true;
-    int y = -1;
-    if (lane < kd) {
-        const size_t r = (size_t)b * k + lane;
-        y = draft[r];
-        const float log_alpha = fminf(0.f, (zp_draft[r] * inv_t - lse_p[r]) - (zq_draft[r] - lse_q[r]));
-        acc = logf(u[r]) <= log_alpha;
-    }
-    const unsigned rejected = ~__ballot_sync(0xffffffffu, acc);
-    const int a = rejected ? __ffs(rejected) - 1 : kd;    // lanes >= kd always vote "accepted"
-    if (lane < k) out_ids[(size_t)b * k + lane] = lane < a ? y : -1;
-    if (lane == 0) {
-        accept_len[b] = a;
-        n_out[b] = a < k ? a + 1 : k;
-        rej_pos[b] = a < k ? a : -1;    // the row a token is drawn from: the first rejection, or the extra row
-        from_p[b] = (a == kd) ? 1 : 0;  // nothing was proposed for that row: the token comes from p itself
-        done[b] = 0;                    // slices of the residual pass finished so far
-    }
-}
-
-// ---------------------------------------------------------------- sample (c)
-// The residual of the one rejected row of a sequence, in fp64: p(v) = exp(z_p/T - lse_p) / Sp with Sp the fp64 sum of
-// the numerators (lse_p is only fp32-accurate), likewise q.  The numerators are computed once (the fp64 exponential is
-// what this path costs) and kept in the workspace for the second pass.
-struct ResidualArgs {
-    int B, k, V, slice;
-    const int32_t* rej_pos;
-    const int32_t* from_p;        // [B] 1: draw from p (the extra row after k-1 accepted drafts), q counts as 0
+// ---------------------------------------------------------------- sample (b) + (c)
+// One kernel, NS thread blocks per sequence.  Every block first repeats the sequence's scan (warp 0, lane i =
+// block row i: log alpha_i against log u_i, Eq. 5) and so knows the first rejected row by itself; block 0 writes
+// the accepted prefix.  Then each block sums the residual max(0, p - q) of that row (Eq. 6) over its slice of the
+// vocabulary, and the block that arrives last draws the token by inverse CDF in vocabulary order.
+//   p(v) = exp(z_p[v]/T - lse_p) (0 below the truncation threshold, if there is one), q(v) = exp(z_q[v] - lse_q):
+// the exponentials in fp32 (expf, 2 ulp), their differences summed in fp64.  lse_p and lse_q are fp32 values,
+// so p and q carry a common relative error of ~1e-6 each; the cumulative residual is off by a few 1e-6 of its
+// total at most, and the draw agrees with an exact evaluation whenever r * S keeps 1e-4 * S away from the edges
+// of the drawn token's cell.
+struct SampleArgs {
+    int B, k, kd, V, slice;
+    const int32_t* draft;
     const float* target_logits;   // [B][k][V]
     const float* draft_logits;    // [B][k][V]
-    const float* lse_p;
+    const float* lse_p;           // [B][k]  logsumexp(z_p / T) (over the kept tokens, if truncated)
+    const float* zp_draft;        // [B][k]  z_p[draft]
+    const float* tau;             // [B][k] or null: tokens with z_p < tau have p = 0
     const float* lse_q;
-    double temperature;
+    const float* zq_draft;
+    float inv_t;
+    const float* u;
     const float* r;
-    double* e_p;                  // [B][V]  exp(z_p/T - lse_p) of the rejected row
-    double* e_q;                  // [B][V]  exp(z_q - lse_q)
-    double* sums;                 // [B][NS][4]: sum e_p, sum e_q, residual mass of the slice, unused
-    int32_t* done;                // [B] slices finished (zeroed by the scan kernel)
-    int32_t* out_ids;
+    double* sums;                 // [B][NS][2]: residual mass, p mass of the slice
+    int* done;                    // [B] slices finished (zeroed by draft_row_stats_kernel)
     int32_t eos_id;
     int32_t* accept_len;
+    int32_t* out_ids;
     int32_t* n_out;
 };
 
@@ -181,7 +163,7 @@ __device__ __forceinline__ double block_sum(double v, double* sh) {
 }
 
 // Algorithm 1's EOS break: nothing is emitted after the first EOS (one thread per sequence).
-__device__ void cut_at_eos(const ResidualArgs& a, int b) {
+__device__ void cut_at_eos(const SampleArgs& a, int b) {
     int32_t* o = a.out_ids + (size_t)b * a.k;
     const int n = a.n_out[b];
     for (int j = 0; j < n; ++j)
@@ -193,111 +175,87 @@ __device__ void cut_at_eos(const ResidualArgs& a, int b) {
         }
 }
 
-// Pass 1: the fp64 normalisers, one (slice, sequence) per block.  Four tokens per thread and step where the
-// rows are 16-byte aligned, so that eight exponentials are in flight per thread.
-__global__ void __launch_bounds__(RES_THREADS) residual_norm_kernel(ResidualArgs a) {
-    __shared__ double sh[32];
-    const int b = blockIdx.y, sl = blockIdx.x;
-    const int i = a.rej_pos[b];
-    if (i < 0) return;
-    const size_t row = (size_t)b * a.k + i;
-    const float* zp = a.target_logits + row * a.V;
-    const float* zq = a.draft_logits + row * a.V;
-    const double lp = (double)a.lse_p[row], lq = (double)a.lse_q[row], it = 1.0 / a.temperature;
-    const int v0 = sl * a.slice, v1 = min(a.V, v0 + a.slice);
-    double sp = 0.0, sq = 0.0;
-    double* ep = a.e_p + (size_t)b * a.V;
-    double* eq = a.e_q + (size_t)b * a.V;
-    int v = v0 + threadIdx.x;
-    if (a.from_p[b]) {
-        // the extra row: only p is needed
-        for (; v < v1; v += RES_THREADS) {
-            const double x = exp((double)zp[v] * it - lp);
-            ep[v] = x;
-            eq[v] = 0.0;
-            sp += x;
-        }
-    } else if ((a.V & 3) == 0) {
-        // v0 and V are multiples of 4, so v1 - v0 is as well
-        for (int q = v0 + 4 * threadIdx.x; q < v1; q += 4 * RES_THREADS) {
-            const float4 p4 = __ldg(reinterpret_cast<const float4*>(zp + q));
-            const float4 q4 = __ldg(reinterpret_cast<const float4*>(zq + q));
-            const double x0 = exp((double)p4.x * it - lp), x1 = exp((double)p4.y * it - lp);
-            const double x2 = exp((double)p4.z * it - lp), x3 = exp((double)p4.w * it - lp);
-            const double y0 = exp((double)q4.x - lq), y1 = exp((double)q4.y - lq);
-            const double y2 = exp((double)q4.z - lq), y3 = exp((double)q4.w - lq);
-            *reinterpret_cast<double2*>(ep + q) = make_double2(x0, x1);
-            *reinterpret_cast<double2*>(ep + q + 2) = make_double2(x2, x3);
-            *reinterpret_cast<double2*>(eq + q) = make_double2(y0, y1);
-            *reinterpret_cast<double2*>(eq + q + 2) = make_double2(y2, y3);
-            sp += (x0 + x1) + (x2 + x3);
-            sq += (y0 + y1) + (y2 + y3);
-        }
-        v = v1;
-    }
-    for (; v < v1; v += RES_THREADS) {
-        const double x = exp((double)zp[v] * it - lp), y = exp((double)zq[v] - lq);
-        ep[v] = x;
-        eq[v] = y;
-        sp += x;
-        sq += y;
-    }
-    sp = block_sum(sp, sh);
-    sq = block_sum(sq, sh);
-    if (threadIdx.x == 0) {
-        a.sums[((size_t)b * NS + sl) * 4 + 0] = sp;
-        a.sums[((size_t)b * NS + sl) * 4 + 1] = sq;
-    }
-}
-
-// Pass 2: residual mass of each slice; the block that finishes a sequence's last slice then draws the token:
-// inverse CDF in vocabulary order, the smallest v whose cumulative residual reaches r * (total residual mass),
-// from p itself if that mass is 0.
-__global__ void __launch_bounds__(RES_THREADS) residual_pick_kernel(ResidualArgs a) {
+__global__ void __launch_bounds__(RES_THREADS) accept_sample_kernel(SampleArgs a) {
     constexpr int NW = RES_THREADS / 32;
     __shared__ double sh[32];
     __shared__ double s_mass[NS], s_psum[NS];
     __shared__ double warp_tot[NW];
-    __shared__ int s_last, s_hit;
+    __shared__ int s_acc, s_last, s_hit;
     const int b = blockIdx.y, sl = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int i = a.rej_pos[b];
+    pdl_trigger();
+    pdl_wait();
+
+    // ---- the scan: first rejected row of this sequence ----
+    if (warp == 0) {
+        bool acc = true;
+        int y = -1;
+        if (lane < a.kd) {
+            const size_t row = (size_t)b * a.k + lane;
+            y = a.draft[row];
+            const float zp = a.zp_draft[row];
+            float log_p = zp * a.inv_t - a.lse_p[row];
+            if (a.tau && zp < a.tau[row]) log_p = -INFINITY;        // outside the kept set: never accepted
+            const float log_alpha = fminf(0.f, log_p - (a.zq_draft[row] - a.lse_q[row]));
+            acc = logf(a.u[row]) <= log_alpha;
+        }
+        const unsigned rejected = ~__ballot_sync(0xffffffffu, acc);
+        const int n_acc = rejected ? __ffs(rejected) - 1 : a.kd;    // lanes >= kd always vote "accepted"
+        if (lane == 0) s_acc = n_acc;
+        if (sl == 0) {
+            if (lane < a.k) a.out_ids[(size_t)b * a.k + lane] = lane < n_acc ? y : -1;
+            if (lane == 0) {
+                a.accept_len[b] = n_acc;
+                a.n_out[b] = n_acc < a.k ? n_acc + 1 : a.k;
+            }
+        }
+    }
+    __syncthreads();
+    const int n_acc = s_acc;
+    const int i = n_acc < a.k ? n_acc : -1;       // the row a token is drawn from: the first rejection, or the extra row
+    const bool from_p = (n_acc == a.kd);          // nothing was proposed for that row: the token comes from p itself
     if (i < 0) {
         if (sl == 0 && tid == 0 && a.eos_id >= 0) cut_at_eos(a, b);
         return;
     }
-    const double* ep = a.e_p + (size_t)b * a.V;
-    const double* eq = a.e_q + (size_t)b * a.V;
-    double Sp = 0.0, Sq = 0.0;
-#pragma unroll
-    for (int j = 0; j < NS; ++j) {
-        Sp += a.sums[((size_t)b * NS + j) * 4 + 0];
-        Sq += a.sums[((size_t)b * NS + j) * 4 + 1];
-    }
-    const double ip = 1.0 / Sp, iq = a.from_p[b] ? 0.0 : 1.0 / Sq;
-    auto resid2 = [&](double x, double y) {
-        const double res = x * ip - y * iq;
-        return res > 0.0 ? res : 0.0;
-    };
+    const size_t row = (size_t)b * a.k + i;
+    const float* __restrict__ zp = a.target_logits + row * a.V;
+    const float* __restrict__ zq = a.draft_logits + row * a.V;
+    const float lp = a.lse_p[row], lq = a.lse_q[row], it = a.inv_t;
+    const float tau = a.tau ? a.tau[row] : -INFINITY;
+    auto p_of = [&](float z) { return z >= tau ? expf(fmaf(z, it, -lp)) : 0.f; };
+    auto q_of = [&](float z) { return from_p ? 0.f : expf(z - lq); };
+    auto resid = [&](float x, float y) { return fmaxf(x - y, 0.f); };
+
+    // ---- residual mass and p mass of this block's slice ----
     {
         const int v0 = sl * a.slice, v1 = min(a.V, v0 + a.slice);
-        double acc = 0.0;
+        double acc = 0.0, accp = 0.0;
         int v = v0 + tid;
-        if ((a.V & 1) == 0) {
-            // slices start at multiples of 4 and V is even: pairs stay inside the slice and 16-byte aligned
-            for (int q = v0 + 2 * tid; q < v1; q += 2 * RES_THREADS) {
-                const double2 x = *reinterpret_cast<const double2*>(ep + q);
-                const double2 y = *reinterpret_cast<const double2*>(eq + q);
-                acc += resid2(x.x, y.x) + resid2(x.y, y.y);
+        if ((a.V & 3) == 0) {
+            // v0 and V are multiples of 4, so v1 - v0 is as well
+            for (int q = v0 + 4 * tid; q < v1; q += 4 * RES_THREADS) {
+                const float4 p4 = __ldg(reinterpret_cast<const float4*>(zp + q));
+                const float4 q4 = __ldg(reinterpret_cast<const float4*>(zq + q));
+                const float x0 = p_of(p4.x), x1 = p_of(p4.y), x2 = p_of(p4.z), x3 = p_of(p4.w);
+                const float y0 = q_of(q4.x), y1 = q_of(q4.y), y2 = q_of(q4.z), y3 = q_of(q4.w);
+                acc += ((double)resid(x0, y0) + (double)resid(x1, y1)) + ((double)resid(x2, y2) + (double)resid(x3, y3));
+                accp += ((double)x0 + (double)x1) + ((double)x2 + (double)x3);
             }
             v = v1;
         }
-        for (; v < v1; v += RES_THREADS) acc += resid2(ep[v], eq[v]);
+        for (; v < v1; v += RES_THREADS) {
+            const float x = p_of(zp[v]);
+            acc += (double)resid(x, q_of(zq[v]));
+            accp += (double)x;
+        }
         acc = block_sum(acc, sh);
+        accp = block_sum(accp, sh);
         if (tid == 0) {
-            a.sums[((size_t)b * NS + sl) * 4 + 2] = acc;
+            a.sums[((size_t)b * NS + sl) * 2 + 0] = acc;
+            a.sums[((size_t)b * NS + sl) * 2 + 1] = accp;
             __threadfence();
-            s_last = (atomicAdd(a.done + b, 1) == NS - 1) ? 1 : 0;
+            s_last = (atomicAdd(a.done + b, 1) == NS - 1) ? 1 : 0;     // zeroed by the pass over the drafter's logits
         }
         __syncthreads();
         if (!s_last) return;
@@ -306,23 +264,26 @@ __global__ void __launch_bounds__(RES_THREADS) residual_pick_kernel(ResidualArgs
     // ---- the last block of the sequence: locate the slice, then the token inside it ----
     const volatile double* vs = a.sums;
     if (tid < NS) {
-        s_mass[tid] = vs[((size_t)b * NS + tid) * 4 + 2];
-        s_psum[tid] = vs[((size_t)b * NS + tid) * 4 + 0];
+        s_mass[tid] = vs[((size_t)b * NS + tid) * 2 + 0];
+        s_psum[tid] = vs[((size_t)b * NS + tid) * 2 + 1];
     }
     __syncthreads();
-    double S = 0.0;
+    double S = 0.0, Sp = 0.0;
 #pragma unroll
-    for (int j = 0; j < NS; ++j) S += s_mass[j];
-    const bool use_p = !(S > 0.0);
-    const double target = (double)a.r[b] * (use_p ? 1.0 : S);
+    for (int j = 0; j < NS; ++j) {
+        S += s_mass[j];
+        Sp += s_psum[j];
+    }
+    const bool use_p = !(S > 0.0);              // no residual mass at all: draw from p itself
+    const double target = (double)a.r[b] * (use_p ? Sp : S);
     double base = 0.0;
     int hs = 0;
     for (; hs < NS - 1; ++hs) {
-        const double m = use_p ? s_psum[hs] * ip : s_mass[hs];
+        const double m = use_p ? s_psum[hs] : s_mass[hs];
         if (base + m >= target) break;
         base += m;
     }
-    auto weight = [&](int v) { return use_p ? ep[v] * ip : resid2(ep[v], eq[v]); };
+    auto weight = [&](int v) { return (double)(use_p ? p_of(zp[v]) : resid(p_of(zp[v]), q_of(zq[v]))); };
     // Warp w owns a contiguous span of the slice, walked 32 consecutive tokens at a time (coalesced).
     const int v0 = hs * a.slice, v1 = min(a.V, v0 + a.slice);
     const int span = ((v1 - v0 + NW - 1) / NW + 31) / 32 * 32;
@@ -386,11 +347,14 @@ __global__ void __launch_bounds__(RES_THREADS) residual_pick_kernel(ResidualArgs
 __global__ void emit_kernel(int B, int k, const int32_t* __restrict__ accept_len, const int32_t* __restrict__ out_ids,
                             const int32_t* __restrict__ n_out, int32_t eos_id, int32_t max_new, int32_t* __restrict__ tokens,
                             int32_t* __restrict__ n_tokens, int32_t* __restrict__ finished, int32_t* __restrict__ keep,
-                            int pending) {
+                            int32_t* __restrict__ appended, int pending) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    pdl_trigger();
+    pdl_wait();
     if (b >= B) return;
     if (finished[b]) {
         keep[b] = 0;
+        if (appended) appended[b] = 0;
         return;
     }
     const int have = n_tokens[b];
@@ -405,26 +369,66 @@ __global__ void emit_kernel(int B, int k, const int32_t* __restrict__ accept_len
         eos |= (eos_id >= 0 && t == eos_id);
     }
     n_tokens[b] = have + m;
+    if (appended) appended[b] = m;
     const int a = accept_len[b];
     keep[b] = (a < m ? (a < 0 ? 0 : a) : m) + pending;    // pending: row 0 was the token emitted last; it stays too
     if (eos || have + m >= max_new) finished[b] = 1;
 }
 
+// ---------------------------------------------------------------- the drafter's block between iterations
+// One thread per sequence: the re-fill rule (masked rows whose best token is confident enough become decoded; if
+// none is, the most confident one does).
+__global__ void refill_kernel(int B, int k, const int32_t* __restrict__ ids, const float* __restrict__ logprob, float log_threshold,
+                              int32_t* __restrict__ row_state, int32_t* __restrict__ tokens, int32_t* __restrict__ left) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    pdl_trigger();
+    pdl_wait();
+    if (b >= B) return;
+    int32_t* st = row_state + (size_t)b * k;
+    int n_masked = 0, n_chosen = 0, best = -1;
+    float best_lp = -INFINITY;
+    for (int i = 0; i < k; ++i) {
+        if (st[i] != 1) continue;
+        ++n_masked;
+        const float lp = logprob[(size_t)b * k + i];
+        if (best < 0 || lp > best_lp) {           // the first row wins among equals
+            best = i;
+            best_lp = lp;
+        }
+        if (lp >= log_threshold) {
+            st[i] = 0;
+            tokens[(size_t)b * k + i] = ids[(size_t)b * k + i];
+            ++n_chosen;
+        }
+    }
+    if (n_masked > 0 && n_chosen == 0) {
+        st[best] = 0;
+        tokens[(size_t)b * k + best] = ids[(size_t)b * k + best];
+        n_chosen = 1;
+    }
+    if (left) left[b] = n_masked - n_chosen;
+}
+
+__global__ void refresh_rows_kernel(int B, int k, const int32_t* __restrict__ appended, int32_t* __restrict__ row_state) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    pdl_trigger();
+    pdl_wait();
+    if (idx >= B * k) return;
+    const int b = idx / k, i = idx % k;
+    row_state[idx] = i < appended[b] ? 0 : -1;
+}
+
 struct SampleWs {
     float* lse_q;
     float* zq_draft;
-    int32_t* rej_pos;
-    int32_t* from_p;
-    double* e_p;
-    double* e_q;
     double* sums;
-    int32_t* done;
+    int* done;
     size_t bytes;
 };
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-SampleWs carve(void* base, int B, int k, int V) {
+SampleWs carve(void* base, int B, int k) {
     SampleWs w;
     size_t off = 0;
     auto take = [&](size_t bytes) {
@@ -434,38 +438,53 @@ SampleWs carve(void* base, int B, int k, int V) {
     };
     w.lse_q = static_cast<float*>(take((size_t)B * k * sizeof(float)));
     w.zq_draft = static_cast<float*>(take((size_t)B * k * sizeof(float)));
-    w.rej_pos = static_cast<int32_t*>(take((size_t)B * sizeof(int32_t)));
-    w.from_p = static_cast<int32_t*>(take((size_t)B * sizeof(int32_t)));
-    w.e_p = static_cast<double*>(take((size_t)B * V * sizeof(double)));
-    w.e_q = static_cast<double*>(take((size_t)B * V * sizeof(double)));
-    w.sums = static_cast<double*>(take((size_t)B * NS * 4 * sizeof(double)));
-    w.done = static_cast<int32_t*>(take((size_t)B * sizeof(int32_t)));
+    w.sums = static_cast<double*>(take((size_t)B * NS * 2 * sizeof(double)));
+    w.done = static_cast<int*>(take((size_t)B * sizeof(int)));
     w.bytes = off;
     return w;
 }
 
 }  // namespace
 
+extern "C" int deer_refill(int B, int k, const int32_t* ids, const float* logprob, float log_threshold, int32_t* row_state,
+                           int32_t* tokens, int32_t* left, void* stream) {
+    DEER_CHECK_ARG(ids && logprob && row_state && tokens, DEER_ERR_INVALID_ARG, "deer_refill: null argument");
+    DEER_CHECK_ARG(k >= 1 && k <= DEER_MAX_BLOCK, DEER_ERR_UNSUPPORTED, "deer_refill: k must be in [1, 32]");
+    DEER_CHECK_ARG(B >= 0, DEER_ERR_INVALID_ARG, "deer_refill: B must not be negative");
+    if (B == 0) return DEER_OK;
+    DEER_CUDA(launch_pdl(refill_kernel, dim3((B + 127) / 128), dim3(128), 0, static_cast<cudaStream_t>(stream), B, k, ids, logprob,
+                         log_threshold, row_state, tokens, left));
+    return DEER_OK;
+}
+
+extern "C" int deer_refresh_rows(int B, int k, const int32_t* appended, int32_t* row_state, void* stream) {
+    DEER_CHECK_ARG(appended && row_state, DEER_ERR_INVALID_ARG, "deer_refresh_rows: null argument");
+    DEER_CHECK_ARG(k >= 1 && k <= DEER_MAX_BLOCK, DEER_ERR_UNSUPPORTED, "deer_refresh_rows: k must be in [1, 32]");
+    DEER_CHECK_ARG(B >= 0, DEER_ERR_INVALID_ARG, "deer_refresh_rows: B must not be negative");
+    if (B == 0) return DEER_OK;
+    DEER_CUDA(launch_pdl(refresh_rows_kernel, dim3((B * k + 127) / 128), dim3(128), 0, static_cast<cudaStream_t>(stream), B, k, appended,
+                         row_state));
+    return DEER_OK;
+}
+
 extern "C" int deer_emit(int B, int k, const int32_t* accept_len, const int32_t* out_ids, const int32_t* n_out, int32_t eos_id,
-                         int32_t max_new, int32_t* tokens, int32_t* n_tokens, int32_t* finished, int32_t* keep, int flags,
-                         void* stream) {
+                         int32_t max_new, int32_t* tokens, int32_t* n_tokens, int32_t* finished, int32_t* keep,
+                         int32_t* appended, int flags, void* stream) {
     DEER_CHECK_ARG((flags & ~DEER_EMIT_PENDING) == 0, DEER_ERR_INVALID_ARG, "deer_emit: unknown flags");
     DEER_CHECK_ARG(accept_len && out_ids && n_out && (tokens || max_new == 0) && n_tokens && finished && keep, DEER_ERR_INVALID_ARG,
                    "deer_emit: null argument");
     DEER_CHECK_ARG(k >= 1 && k <= DEER_MAX_BLOCK, DEER_ERR_UNSUPPORTED, "deer_emit: k must be in [1, 32]");
     DEER_CHECK_ARG(B >= 0 && max_new >= 0, DEER_ERR_INVALID_ARG, "deer_emit: B and max_new must not be negative");
     if (B == 0) return DEER_OK;
-    emit_kernel<<<(B + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(B, k, accept_len, out_ids, n_out, eos_id, max_new,
-                                                                               tokens, n_tokens, finished, keep,
-                                                                               (flags & DEER_EMIT_PENDING) ? 1 : 0);
-    DEER_CUDA(cudaGetLastError());
+    DEER_CUDA(launch_pdl(emit_kernel, dim3((B + 127) / 128), dim3(128), 0, static_cast<cudaStream_t>(stream), B, k, accept_len, out_ids,
+                         n_out, eos_id, max_new, tokens, n_tokens, finished, keep, appended, (flags & DEER_EMIT_PENDING) ? 1 : 0));
     return DEER_OK;
 }
 
 extern "C" size_t deer_accept_workspace_bytes(int mode, int B, int k, int V) {
     mode &= ~DEER_ACC_BONUS;
     if ((mode != DEER_ACC_SAMPLE && mode != DEER_ACC_SAMPLE_PRESTATS) || B <= 0 || k <= 0 || V <= 0) return 0;
-    return carve(nullptr, B, k, V).bytes;
+    return carve(nullptr, B, k).bytes;
 }
 
 extern "C" int deer_draft_stats(int B, int k, int V, const int32_t* draft_ids, const float* draft_logits, void* workspace,
@@ -479,7 +498,7 @@ extern "C" int deer_draft_stats(int B, int k, int V, const int32_t* draft_ids, c
     const size_t need = deer_accept_workspace_bytes(DEER_ACC_SAMPLE, B, k, V);
     DEER_CHECK_ARG(workspace && workspace_bytes >= need, DEER_ERR_WORKSPACE,
                    "deer_draft_stats: workspace of %zu bytes needed, %zu given", need, workspace_bytes);
-    const SampleWs w = carve(workspace, B, k, V);
+    const SampleWs w = carve(workspace, B, k);
     // Meant to run beside the attention kernel, whose blocks take 56 K of an SM's 64 K registers and most of its
     // shared memory.  Two things let a block of this kernel share an SM with one of those: at most one block per SM
     // (one block of 256 threads and 32 registers per SM, striding over the rows; a block per row filled the SMs first and
@@ -488,9 +507,8 @@ extern "C" int deer_draft_stats(int B, int k, int V, const int32_t* draft_ids, c
     // 496 us instead of 283).
     const int rows = B * k, sms = deer_sm_count();
     DEER_CUDA(cudaFuncSetAttribute(draft_row_stats_kernel<256, 4>, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
-    draft_row_stats_kernel<256, 4><<<rows < sms ? rows : sms, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        rows, V, draft_logits, draft_ids, w.lse_q, w.zq_draft);
-    DEER_CUDA(cudaGetLastError());
+    DEER_CUDA(launch_pdl(draft_row_stats_kernel<256, 4>, dim3(rows < sms ? rows : sms), dim3(256), 0, static_cast<cudaStream_t>(stream),
+                         rows, V, draft_logits, draft_ids, w.lse_q, w.zq_draft, w.done, B));
     return DEER_OK;
 }
 
@@ -499,6 +517,16 @@ extern "C" int deer_accept(int mode, int B, int k, int V, const int32_t* draft_i
                            float temperature, const float* draft_logits, const float* u, const float* r, int32_t eos_id,
                            int32_t* accept_len, int32_t* out_ids, int32_t* n_out, void* workspace, size_t workspace_bytes,
                            void* stream) {
+    return deer_accept_truncated(mode, B, k, V, draft_ids, target_ids, target_logits, target_lse, target_draft_logit, nullptr,
+                                 temperature, draft_logits, u, r, eos_id, accept_len, out_ids, n_out, workspace, workspace_bytes,
+                                 stream);
+}
+
+extern "C" int deer_accept_truncated(int mode, int B, int k, int V, const int32_t* draft_ids, const int32_t* target_ids,
+                                     const float* target_logits, const float* target_lse, const float* target_draft_logit,
+                                     const float* target_tau, float temperature, const float* draft_logits, const float* u,
+                                     const float* r, int32_t eos_id, int32_t* accept_len, int32_t* out_ids, int32_t* n_out,
+                                     void* workspace, size_t workspace_bytes, void* stream) {
     const int kd = (mode & DEER_ACC_BONUS) ? k - 1 : k;     // drafts under test
     mode &= ~DEER_ACC_BONUS;
     DEER_CHECK_ARG(mode == DEER_ACC_GREEDY || mode == DEER_ACC_SAMPLE || mode == DEER_ACC_SAMPLE_PRESTATS, DEER_ERR_INVALID_ARG,
@@ -510,8 +538,8 @@ extern "C" int deer_accept(int mode, int B, int k, int V, const int32_t* draft_i
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (mode == DEER_ACC_GREEDY) {
         DEER_CHECK_ARG(target_ids, DEER_ERR_INVALID_ARG, "deer_accept: target_ids is required in GREEDY mode");
-        accept_greedy_kernel<<<(B + 127) / 128, 128, 0, st>>>(B, k, kd, draft_ids, target_ids, eos_id, accept_len, out_ids, n_out);
-        DEER_CUDA(cudaGetLastError());
+        DEER_CUDA(launch_pdl(accept_greedy_kernel, dim3((B + 127) / 128), dim3(128), 0, st, B, k, kd, draft_ids, target_ids, eos_id,
+                             accept_len, out_ids, n_out));
         return DEER_OK;
     }
     DEER_CHECK_ARG(target_logits && target_lse && target_draft_logit && draft_logits && u && r, DEER_ERR_INVALID_ARG,
@@ -522,41 +550,35 @@ extern "C" int deer_accept(int mode, int B, int k, int V, const int32_t* draft_i
     const size_t need = deer_accept_workspace_bytes(mode, B, k, V);
     DEER_CHECK_ARG(workspace && workspace_bytes >= need, DEER_ERR_WORKSPACE,
                    "deer_accept: workspace of %zu bytes needed, %zu given", need, workspace_bytes);
-    const SampleWs w = carve(workspace, B, k, V);
+    const SampleWs w = carve(workspace, B, k);
 
     if (mode == DEER_ACC_SAMPLE) {       // otherwise deer_draft_stats has left them in the workspace
-        draft_row_stats_kernel<256, 2><<<B * k, 256, 0, st>>>(B * k, V, draft_logits, draft_ids, w.lse_q, w.zq_draft);
-        DEER_CUDA(cudaGetLastError());
+        DEER_CUDA(launch_pdl(draft_row_stats_kernel<256, 2>, dim3(B * k), dim3(256), 0, st, B * k, V, draft_logits, draft_ids, w.lse_q,
+                             w.zq_draft, w.done, B));
     }
-    accept_scan_kernel<<<(B + 3) / 4, 128, 0, st>>>(B, k, kd, draft_ids, target_lse, target_draft_logit, 1.f / temperature,
-                                                     w.lse_q, w.zq_draft, u, accept_len, out_ids, n_out, w.rej_pos,
-                                                     w.from_p, w.done);
-    DEER_CUDA(cudaGetLastError());
-
-    ResidualArgs a;
+    SampleArgs a;
     a.B = B;
     a.k = k;
+    a.kd = kd;
     a.V = V;
     a.slice = ((V + NS - 1) / NS + 3) / 4 * 4;
-    a.rej_pos = w.rej_pos;
-    a.from_p = w.from_p;
+    a.draft = draft_ids;
     a.target_logits = target_logits;
     a.draft_logits = draft_logits;
     a.lse_p = target_lse;
+    a.zp_draft = target_draft_logit;
+    a.tau = target_tau;
     a.lse_q = w.lse_q;
-    a.temperature = (double)temperature;
+    a.zq_draft = w.zq_draft;
+    a.inv_t = 1.f / temperature;
+    a.u = u;
     a.r = r;
-    a.e_p = w.e_p;
-    a.e_q = w.e_q;
     a.sums = w.sums;
     a.done = w.done;
-    a.out_ids = out_ids;
     a.eos_id = eos_id;
     a.accept_len = accept_len;
+    a.out_ids = out_ids;
     a.n_out = n_out;
-    residual_norm_kernel<<<dim3(NS, B), RES_THREADS, 0, st>>>(a);
-    DEER_CUDA(cudaGetLastError());
-    residual_pick_kernel<<<dim3(NS, B), RES_THREADS, 0, st>>>(a);
-    DEER_CUDA(cudaGetLastError());
+    DEER_CUDA(launch_pdl(accept_sample_kernel, dim3(NS, B), dim3(RES_THREADS), 0, st, a));
     return DEER_OK;
 }

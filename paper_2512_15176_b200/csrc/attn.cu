@@ -42,6 +42,8 @@ __global__ void __launch_bounds__(ATT_THREADS, 1) block_attn_kernel(AttnParams p
     const int b = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int Hkv = p.kv.n_kv_heads;
+    pdl_trigger();
+    pdl_wait();
 
     const int s = p.seq_ids[b];
     if (s < 0 || s >= p.kv.max_seqs) {
@@ -64,10 +66,14 @@ __global__ void __launch_bounds__(ATT_THREADS, 1) block_attn_kernel(AttnParams p
     const __nv_bfloat16* kpool = static_cast<const __nv_bfloat16*>(p.kv.k_pool);
     const __nv_bfloat16* vpool = static_cast<const __nv_bfloat16*>(p.kv.v_pool);
 
-    // ---- append the block's K/V rows to the cache (one block per (b, kvh)) ----
+    uint32_t present, decoded;
+    row_state_sets(p.row_state, b, p.k, lane, &present, &decoded);
+
+    // ---- append the block's K/V rows to the cache (one block per (b, kvh)); with row states the decoded rows only ----
     if (p.append && last && rt == 0) {
         for (int idx = tid; idx < p.k * PIECES; idx += ATT_THREADS) {
             const int j = idx / PIECES, pc = idx % PIECES;
+            if (p.row_state && !((decoded >> j) & 1u)) continue;
             const int t = n + j;
             const int lp = t >> 4;
             const int pg = (lp < p.kv.max_pages) ? pt_row[lp] : -1;
@@ -119,7 +125,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 1) block_attn_kernel(AttnParams p
                 for (int it = 0; it < ATT_TILE * PIECES / ATT_THREADS; ++it) {
                     const int idx = tid + it * ATT_THREADS;
                     const int row = idx / PIECES, pc = idx % PIECES;
-                    const int bytes = (row < p.k) ? 16 : 0;
+                    const int bytes = (row < p.k && ((present >> row) & 1u)) ? 16 : 0;     // rows that hold nothing read as zero
                     const size_t off = ((size_t)(b * p.k + (row < p.k ? row : 0)) * Hkv + kvh) * D + pc * 8;
                     cp_async16(kdst + tile_off<D>(row, pc), p.k_blk + off, bytes);
                     cp_async16(vdst + tile_off<D>(row, pc), p.v_blk + off, bytes);
@@ -156,6 +162,8 @@ __global__ void __launch_bounds__(ATT_THREADS, 1) block_attn_kernel(AttnParams p
     const int row_lo = rt * ATT_ROWS + warp * 16 + g8;   // global row (within the KV head) of accumulator rows g and g+8
     const int row_hi = row_lo + 8;
     const int i_lo = row_lo % p.k, i_hi = row_hi % p.k;
+    const uint32_t cols_lo = visible_rows(p.mask, i_lo, p.row_state ? p.row_state[(size_t)b * p.k + i_lo] : 1, present, decoded);
+    const uint32_t cols_hi = visible_rows(p.mask, i_hi, p.row_state ? p.row_state[(size_t)b * p.k + i_hi] : 1, present, decoded);
 
     float o[ND][4];
 #pragma unroll
@@ -196,9 +204,9 @@ __global__ void __launch_bounds__(ATT_THREADS, 1) block_attn_kernel(AttnParams p
             for (int e = 0; e < 2; ++e) {
                 const int col = nt * 8 + t4 * 2 + e;
                 bool ok_lo = col < valid, ok_hi = col < valid;
-                if (is_block && p.mask == DEER_MASK_CAUSAL) {
-                    ok_lo = ok_lo && (col <= i_lo);
-                    ok_hi = ok_hi && (col <= i_hi);
+                if (is_block) {                       // valid = k <= 32 here, so col < 32 wherever ok is still true
+                    ok_lo = ok_lo && ((cols_lo >> (col & 31)) & 1u);
+                    ok_hi = ok_hi && ((cols_hi >> (col & 31)) & 1u);
                 }
                 sc[nt][e] = ok_lo ? sc[nt][e] * p.scale_log2 : -INFINITY;
                 sc[nt][2 + e] = ok_hi ? sc[nt][2 + e] * p.scale_log2 : -INFINITY;
@@ -287,6 +295,8 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(AttnParams p, __nv_bflo
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const size_t n_rows = (size_t)p.B * p.k * p.Hq;
     const size_t orow = (size_t)blockIdx.x * 8 + warp;
+    pdl_trigger();
+    pdl_wait();
     if (orow >= n_rows) return;
     const int b = (int)(orow / ((size_t)p.k * p.Hq));
     const int s = p.seq_ids[b];
@@ -347,7 +357,16 @@ extern "C" size_t deer_block_attn_workspace_bytes(int B, int k, int Hq, int Hkv,
 extern "C" int deer_block_attn(deer_kv* kv, const int32_t* seq_ids, const void* q, const void* k_blk, const void* v_blk,
                                void* out, int B, int k, int Hq, int mask, int append, float scale, int max_seq_len,
                                void* workspace, size_t workspace_bytes, void* stream) {
+    return deer_block_attn_rows(kv, seq_ids, q, k_blk, v_blk, out, nullptr, B, k, Hq, mask, append, scale, max_seq_len, workspace,
+                                workspace_bytes, stream);
+}
+
+extern "C" int deer_block_attn_rows(deer_kv* kv, const int32_t* seq_ids, const void* q, const void* k_blk, const void* v_blk,
+                                    void* out, const int32_t* row_state, int B, int k, int Hq, int mask, int append, float scale,
+                                    int max_seq_len, void* workspace, size_t workspace_bytes, void* stream) {
     DEER_CHECK_ARG(kv && seq_ids && q && k_blk && v_blk && out, DEER_ERR_INVALID_ARG, "deer_block_attn: null argument");
+    DEER_CHECK_ARG(!row_state || mask == DEER_MASK_BIDIR, DEER_ERR_INVALID_ARG,
+                   "deer_block_attn_rows: row states belong to the bidirectional mask");
     DEER_CHECK_ARG(deer_aligned16(q) && deer_aligned16(k_blk) && deer_aligned16(v_blk) && deer_aligned16(out) &&
                        deer_aligned16(workspace),
                    DEER_ERR_INVALID_ARG, "deer_block_attn: pointers must be 16-byte aligned");
@@ -369,6 +388,7 @@ extern "C" int deer_block_attn(deer_kv* kv, const int32_t* seq_ids, const void* 
     AttnParams p;
     p.kv = kv->d;
     p.seq_ids = seq_ids;
+    p.row_state = row_state;
     p.q = static_cast<const __nv_bfloat16*>(q);
     p.k_blk = static_cast<const __nv_bfloat16*>(k_blk);
     p.v_blk = static_cast<const __nv_bfloat16*>(v_blk);
@@ -403,15 +423,13 @@ extern "C" int deer_block_attn(deer_kv* kv, const int32_t* seq_ids, const void* 
     } else if (D == 128) {
         constexpr int SM = attn_smem_bytes<128>();
         DEER_CUDA(cudaFuncSetAttribute(block_attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM));
-        block_attn_kernel<128><<<grid, ATT_THREADS, SM, st>>>(p);
-        DEER_CUDA(cudaGetLastError());
-        attn_merge_kernel<128><<<merge_blocks, 256, 0, st>>>(p, static_cast<__nv_bfloat16*>(out));
+        DEER_CUDA(launch_pdl(block_attn_kernel<128>, grid, dim3(ATT_THREADS), (size_t)SM, st, p));
+        DEER_CUDA(launch_pdl(attn_merge_kernel<128>, dim3(merge_blocks), dim3(256), 0, st, p, static_cast<__nv_bfloat16*>(out)));
     } else {
         constexpr int SM = attn_smem_bytes<64>();
         DEER_CUDA(cudaFuncSetAttribute(block_attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM));
-        block_attn_kernel<64><<<grid, ATT_THREADS, SM, st>>>(p);
-        DEER_CUDA(cudaGetLastError());
-        attn_merge_kernel<64><<<merge_blocks, 256, 0, st>>>(p, static_cast<__nv_bfloat16*>(out));
+        DEER_CUDA(launch_pdl(block_attn_kernel<64>, grid, dim3(ATT_THREADS), (size_t)SM, st, p));
+        DEER_CUDA(launch_pdl(attn_merge_kernel<64>, dim3(merge_blocks), dim3(256), 0, st, p, static_cast<__nv_bfloat16*>(out)));
     }
     DEER_CUDA(cudaGetLastError());
     return DEER_OK;

@@ -9,9 +9,29 @@ namespace attn {
 constexpr int ATT_TILE = 64;      // tokens per pipeline stage (4 pages)
 constexpr float LOG2E = 1.4426950408889634f;
 
+#ifdef __CUDACC__
+// Block rows that block row i may see, as a bit per row.  Causal: rows 0..i.  Bidirectional: all k; with row
+// states a masked row sees the rows that hold something, a decoded row the decoded rows, and an absent row (whose
+// output nobody reads) is treated like a masked one.  `present` / `decoded` are the bit sets of the sequence's rows
+// with state >= 0 / == 0 (all ones without row states).
+__device__ __forceinline__ uint32_t visible_rows(int mask, int i, int state_i, uint32_t present, uint32_t decoded) {
+    if (mask == DEER_MASK_CAUSAL) return i >= 31 ? 0xffffffffu : (2u << i) - 1u;
+    return state_i == 0 ? decoded : present;
+}
+// Warp-collective: the two bit sets for sequence b (lane j looks at row j).
+__device__ __forceinline__ void row_state_sets(const int32_t* row_state, int b, int k, int lane, uint32_t* present, uint32_t* decoded) {
+    int st = 1;
+    if (row_state) st = lane < k ? row_state[(size_t)b * k + lane] : -1;
+    else if (lane >= k) st = -1;
+    *present = __ballot_sync(0xffffffffu, st >= 0);
+    *decoded = row_state ? __ballot_sync(0xffffffffu, st == 0) : *present;
+}
+#endif
+
 struct AttnParams {
     deer_kv_desc kv;
     const int32_t* seq_ids;
+    const int32_t* row_state;  // [B][k] or null: 1 masked, 0 decoded, -1 absent (bidirectional mask only)
     const __nv_bfloat16* q;
     const __nv_bfloat16* k_blk;
     const __nv_bfloat16* v_blk;

@@ -194,26 +194,9 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const int jg = j / p.row_tiles, rt_blk = j % p.row_tiles;  // group of blocks that walk the same share; my row tile
     const int ncg = p.nc / p.row_tiles;                        // groups (nc is a multiple of row_tiles)
 
-    // ---- this block's share of the flattened tile list ----
-    long long T = 0;
-    for (int b = lane; b < p.B; b += 32) {
-        const int tiles = seq_tiles(p, b, nullptr, nullptr);
-        T += tiles;
-        // a sequence that cannot be used has no tiles, so no block will write its units' merge entries: do it here
-        if (tiles == 0 && j == 0 && warp == 0)
-            for (int hr = 0; hr < HR; ++hr) p.unit_parts[(size_t)b * HR + hr] = make_int2(-1, -1);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) T += __shfl_xor_sync(0xffffffffu, T, o);
-    T *= Hkv;                                                  // list entries: (sequence, KV head) x tiles
-    const long long share_lo = share_begin(T, jg, ncg), share_hi = share_begin(T, jg + 1, ncg);
-    if (j == 0 && tid == 0) *p.total_tiles = T;                // for the merge kernel
-    if (share_hi <= share_lo) return;                          // nothing to do (fewer tiles than blocks)
-
+    // ---- what needs no input: barriers, tensor-map prefetch ----
     const uint32_t bar_base = smem_u32(bars);
     auto bar = [&](int idx) { return bar_base + 8u * idx; };
-
-    // ---- set-up ---------------------------------------------------------------
     if (tid == 0) {
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(BAR_Q_FULL + i), 1);
@@ -238,6 +221,25 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         prefetch_tensormap(&tm_kpool);
         prefetch_tensormap(&tm_vpool);
     }
+    pdl_trigger();
+    pdl_wait();                                                // lengths, page table, the block's rows: written by what ran before
+
+    // ---- this block's share of the flattened tile list ----
+    long long T = 0;
+    for (int b = lane; b < p.B; b += 32) {
+        const int tiles = seq_tiles(p, b, nullptr, nullptr);
+        T += tiles;
+        // a sequence that cannot be used has no tiles, so no block will write its units' merge entries: do it here
+        if (tiles == 0 && j == 0 && warp == 0)
+            for (int hr = 0; hr < HR; ++hr) p.unit_parts[(size_t)b * HR + hr] = make_int2(-1, -1);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) T += __shfl_xor_sync(0xffffffffu, T, o);
+    T *= Hkv;                                                  // list entries: (sequence, KV head) x tiles
+    const long long share_lo = share_begin(T, jg, ncg), share_hi = share_begin(T, jg + 1, ncg);
+    if (j == 0 && tid == 0) *p.total_tiles = T;                // for the merge kernel
+    if (share_hi <= share_lo) return;                          // nothing to do (fewer tiles than blocks)
+
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
     tcgen05_fence_before();
     __syncthreads();
@@ -411,13 +413,19 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 const int i_blk = i0 + row / p.G;             // block row of this query row
                 const bool row_valid = row < ni * p.G;
                 const int last_tile = (g.n + ATT_TILE - 1) / ATT_TILE;
+                uint32_t present, decoded;
+                row_state_sets(p.row_state, g.b, p.k, lane, &present, &decoded);
+                const uint32_t my_cols = visible_rows(p.mask, i_blk, (p.row_state && row_valid) ? p.row_state[(size_t)g.b * p.k + i_blk] : 1,
+                                                      present, decoded);
 
-                // append the block's K/V rows to the cache (once per (sequence, KV head): with the block tile of row tile 0)
+                // append the block's K/V rows to the cache (once per (sequence, KV head): with the block tile of row tile 0);
+                // with row states the decoded rows only
                 if (p.append && rt == 0 && g.t_b == last_tile + 1) {
                     constexpr int PIECES = HD / 8;
                     const int32_t* pt_row = p.kv.page_table + (size_t)g.s * p.kv.max_pages;
                     for (int idx = wtid; idx < p.k * PIECES; idx += 128) {
                         const int jr = idx / PIECES, pc = idx % PIECES;
+                        if (p.row_state && !((decoded >> jr) & 1u)) continue;
                         const int t = g.n + jr;
                         const int lp = t >> 4;
                         const int pg = (lp < p.kv.max_pages) ? pt_row[lp] : -1;
@@ -451,12 +459,14 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     // columns this row may see: the valid tokens of a prefix tile, or the block rows the mask allows
                     const bool is_block = (t == last_tile);
                     const int tile_valid = is_block ? p.k : min(ATT_TILE, g.n - t * ATT_TILE);
-                    int limit = tile_valid;
-                    if (is_block && p.mask == DEER_MASK_CAUSAL) limit = min(p.k, i_blk + 1);
-                    if (limit < ATT_TILE) {                   // ragged or masked tile: hide the columns this row may not see
+                    if (is_block) {                           // the block rows' own tile: k <= 32 columns, a bit per column
 #pragma unroll
                         for (int c = 0; c < ATT_TILE; ++c)
-                            if (c >= limit) sr[c] = 0xff800000u;   // -inf
+                            if (c >= 32 || c >= p.k || !((my_cols >> (c & 31)) & 1u)) sr[c] = 0xff800000u;   // -inf
+                    } else if (tile_valid < ATT_TILE) {       // ragged prefix tile: hide the columns beyond the sequence
+#pragma unroll
+                        for (int c = 0; c < ATT_TILE; ++c)
+                            if (c >= tile_valid) sr[c] = 0xff800000u;
                     }
                     float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains: one warp per scheduler needs the ILP
 #pragma unroll
@@ -526,6 +536,13 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                             const int off = is_block ? half * KV_HALF + tk * 128
                                                      : (tk >> 4) * 4096 + ((tk >> 3) & 1) * 2048 + half * 1024 + (tk & 7) * 128;
                             *reinterpret_cast<uint4*>(vt + off + pc * 16) = make_uint4(0, 0, 0, 0);
+                        }
+                        if (is_block && p.row_state) {        // so do the rows of positions that hold nothing
+                            for (int idx = wtid; idx < p.k * 16; idx += 128) {
+                                const int tk = idx >> 4, half = (idx >> 3) & 1, pc = idx & 7;
+                                if (!((present >> tk) & 1u))
+                                    *reinterpret_cast<uint4*>(vt + half * KV_HALF + tk * 128 + pc * 16) = make_uint4(0, 0, 0, 0);
+                            }
                         }
                         fence_proxy_async_smem();
                     }
@@ -628,6 +645,8 @@ __global__ void __launch_bounds__(256) attn_umma_merge_kernel(const AttnParams p
     const int unit = blockIdx.x / BPU;
     const int Hkv = p.kv.n_kv_heads, HR = Hkv * p.row_tiles;
     const int b = unit / HR, hr = unit % HR;
+    pdl_trigger();
+    pdl_wait();                                                   // the attention kernel's partial results
     // written by the block that holds the unit's first tile (by block 0 for a sequence that was skipped)
     const int2 parts = p.unit_parts[unit];
     if (parts.x < 0) return;
@@ -780,11 +799,11 @@ int launch_umma(AttnParams p, cudaStream_t st) {
         if (rc != DEER_OK) return rc;
     }
     DEER_CUDA(cudaFuncSetAttribute(block_attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
-    block_attn_umma_kernel<<<p.nc, THREADS, SMEM_BYTES, st>>>(tm_q, tm_kb, tm_vb, tm_kp, tm_vp, p);
-    DEER_CUDA(cudaGetLastError());
-    if ((long long)p.B * HR * 4 >= 2 * deer_sm_count()) attn_umma_merge_kernel<4><<<(unsigned)(p.B * HR * 4), 256, 0, st>>>(p);
-    else attn_umma_merge_kernel<1><<<(unsigned)(p.B * HR * 16), 256, 0, st>>>(p);
-    DEER_CUDA(cudaGetLastError());
+    DEER_CUDA(launch_pdl(block_attn_umma_kernel, dim3(p.nc), dim3(THREADS), (size_t)SMEM_BYTES, st, tm_q, tm_kb, tm_vb, tm_kp, tm_vp, p));
+    if ((long long)p.B * HR * 4 >= 2 * deer_sm_count())
+        DEER_CUDA(launch_pdl(attn_umma_merge_kernel<4>, dim3((unsigned)(p.B * HR * 4)), dim3(256), 0, st, p));
+    else
+        DEER_CUDA(launch_pdl(attn_umma_merge_kernel<1>, dim3((unsigned)(p.B * HR * 16)), dim3(256), 0, st, p));
     return DEER_OK;
 }
 

@@ -54,8 +54,21 @@ inline int deer_sm_count() {
     return cached[dev];
 }
 
-// A tag for one call's arrival words (see arrive_last); never 0, distinct for every call of the process.
-uint32_t deer_next_epoch();
+// Launches `kernel` so that it may overlap the tail of the kernel before it in the stream (see pdl_wait below).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 // ---- device helpers --------------------------------------------------------
 #ifdef __CUDACC__
@@ -98,26 +111,14 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// "Last block done" without a counter that somebody has to clear.  `word` holds (tag << 32 | arrivals); a caller
-// that finds another tag than its call's `epoch` starts the count anew, so whatever the memory held before (an
-// uninitialised workspace, an older call) does not matter, and the caller that completes `expected` arrivals
-// puts the word back to 0, so that a replay of the same launch (a CUDA graph carries the same epoch) starts
-// clean as well.  Returns true for exactly one caller: the one that arrived last.  Writes made before a
-// __threadfence() by the other callers are visible to it after its own __threadfence().
-__device__ __forceinline__ bool arrive_last(unsigned long long* word, uint32_t epoch, uint32_t expected) {
-    unsigned long long cur = *reinterpret_cast<volatile unsigned long long*>(word);
-    for (;;) {
-        const uint32_t cnt = ((uint32_t)(cur >> 32) == epoch) ? (uint32_t)cur + 1u : 1u;
-        const unsigned long long nxt = ((unsigned long long)epoch << 32) | cnt;
-        const unsigned long long old = atomicCAS(word, cur, nxt);
-        if (old == cur) {
-            if (cnt != expected) return false;
-            *reinterpret_cast<volatile unsigned long long*>(word) = 0ull;
-            return true;
-        }
-        cur = old;                 // another block arrived in between: at most `expected` rounds
-    }
-}
+// Programmatic dependent launch.  A kernel launched with launch_pdl() may become resident while the kernel before
+// it in the stream is still running: its blocks set up what needs no input (barriers, tensor memory, tensor-map
+// prefetch) and then sit in pdl_wait() until that kernel has completed and its writes are visible.  pdl_trigger()
+// in a running kernel lets the next one be launched from that point on.  Every kernel of the library executes
+// pdl_wait() in every thread before its first read of global memory, so the completion of a kernel implies the
+// completion of everything before it; both instructions do nothing in a kernel launched the plain way.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // Record the first data-dependent error seen by any kernel.
 __device__ __forceinline__ void deer_report(int32_t* status, int32_t code) {

@@ -10,7 +10,6 @@
 #include <stdarg.h>
 #include <string.h>
 
-#include <atomic>
 #include <new>
 
 #include "common.cuh"
@@ -26,13 +25,6 @@ void deer_set_error(const char* fmt, ...) {
 }
 
 extern "C" const char* deer_last_error(void) { return g_err; }
-
-uint32_t deer_next_epoch() {
-    static std::atomic<uint32_t> next{1};
-    uint32_t e = next.fetch_add(1, std::memory_order_relaxed);
-    while (e == 0) e = next.fetch_add(1, std::memory_order_relaxed);
-    return e;
-}
 
 // ---- handle ----------------------------------------------------------------
 extern "C" int deer_kv_create(deer_kv** kv, const deer_kv_desc* desc) {
@@ -103,6 +95,8 @@ kv_reserve_kernel(deer_kv_desc d, const int32_t* __restrict__ seq_ids, int B, in
     __shared__ int total;
     __shared__ int bad;
     const int b = threadIdx.x;
+    pdl_trigger();
+    pdl_wait();
     if (b == 0) bad = 0;
     __syncthreads();
     int s = -1, have = 0, need_pages = 0;
@@ -140,6 +134,8 @@ kv_commit_kernel(deer_kv_desc d, const int32_t* __restrict__ seq_ids, const int3
     __shared__ int warp_sums[32];
     __shared__ int total;
     const int b = threadIdx.x;
+    pdl_trigger();
+    pdl_wait();
     int s = -1, have = 0, need_pages = 0;
     if (b < B) {
         s = seq_ids[b];
@@ -185,8 +181,7 @@ extern "C" int deer_kv_reserve(deer_kv* kv, const int32_t* seq_ids, int B, int k
     DEER_CHECK_ARG(B >= 0 && B <= KV_THREADS, DEER_ERR_UNSUPPORTED, "deer_kv_reserve: B must be in [0, %d]", KV_THREADS);
     DEER_CHECK_ARG(k >= 0 && k <= DEER_MAX_BLOCK, DEER_ERR_UNSUPPORTED, "deer_kv_reserve: k must be in [0, 32]");
     if (B == 0) return DEER_OK;
-    kv_reserve_kernel<<<1, KV_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(kv->d, seq_ids, B, k);
-    DEER_CUDA(cudaGetLastError());
+    DEER_CUDA(launch_pdl(kv_reserve_kernel, dim3(1), dim3(KV_THREADS), 0, static_cast<cudaStream_t>(stream), kv->d, seq_ids, B, k));
     return DEER_OK;
 }
 
@@ -195,7 +190,6 @@ extern "C" int deer_kv_commit(deer_kv* kv, const int32_t* seq_ids, const int32_t
     DEER_CHECK_ARG(B >= 0 && B <= KV_THREADS, DEER_ERR_UNSUPPORTED, "deer_kv_commit: B must be in [0, %d]", KV_THREADS);
     DEER_CHECK_ARG(k >= 0 && k <= DEER_MAX_BLOCK, DEER_ERR_UNSUPPORTED, "deer_kv_commit: k must be in [0, 32]");
     if (B == 0) return DEER_OK;
-    kv_commit_kernel<<<1, KV_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(kv->d, seq_ids, keep, B, k);
-    DEER_CUDA(cudaGetLastError());
+    DEER_CUDA(launch_pdl(kv_commit_kernel, dim3(1), dim3(KV_THREADS), 0, static_cast<cudaStream_t>(stream), kv->d, seq_ids, keep, B, k));
     return DEER_OK;
 }

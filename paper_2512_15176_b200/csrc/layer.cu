@@ -19,6 +19,8 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const __nv_bfloat16* __res
                                                       __nv_bfloat16* __restrict__ y, int hid, float eps) {
     __shared__ float part[8];
     const size_t row = blockIdx.x;
+    pdl_trigger();
+    pdl_wait();
     const __nv_bfloat16* xr = x + row * hid;
     float ss = 0.f;
     for (int c = threadIdx.x; c < hid; c += 256) {
@@ -49,6 +51,8 @@ __global__ void __launch_bounds__(128) qk_norm_rope_kernel(deer_kv_desc kv, cons
                                                            int D, float eps, double log2_theta) {
     const int lane = threadIdx.x & 31;
     const long long item = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
+    pdl_trigger();
+    pdl_wait();
     const long long nq = (long long)B * k * Hq, nk = (long long)B * k * Hkv;
     if (item >= nq + nk + (qkv ? nk : 0)) return;
     if (item >= nq + nk) {                                        // a V head: copy out of the packed rows
@@ -110,6 +114,8 @@ __global__ void __launch_bounds__(128) qk_norm_rope_kernel(deer_kv_desc kv, cons
 __global__ void __launch_bounds__(256) swiglu_kernel(const __nv_bfloat16* __restrict__ gu, __nv_bfloat16* __restrict__ y, int I,
                                                      long long total) {
     const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+    pdl_trigger();
+    pdl_wait();
     if (idx >= total) return;
     const long long m = idx / I;
     const int c = (int)(idx % I);
@@ -123,10 +129,8 @@ extern "C" int deer_rmsnorm(const void* x, const void* gamma, void* y, int M, in
     DEER_CHECK_ARG(x && gamma && y, DEER_ERR_INVALID_ARG, "deer_rmsnorm: null argument");
     DEER_CHECK_ARG(M >= 0 && hid > 0 && eps >= 0.f, DEER_ERR_INVALID_ARG, "deer_rmsnorm: bad sizes");
     if (M == 0) return DEER_OK;
-    rmsnorm_kernel<<<M, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const __nv_bfloat16*>(x),
-                                                                      static_cast<const __nv_bfloat16*>(gamma),
-                                                                      static_cast<__nv_bfloat16*>(y), hid, eps);
-    DEER_CUDA(cudaGetLastError());
+    DEER_CUDA(launch_pdl(rmsnorm_kernel, dim3(M), dim3(256), 0, static_cast<cudaStream_t>(stream), static_cast<const __nv_bfloat16*>(x),
+                         static_cast<const __nv_bfloat16*>(gamma), static_cast<__nv_bfloat16*>(y), hid, eps));
     return DEER_OK;
 }
 
@@ -140,12 +144,11 @@ static int qk_norm_rope(deer_kv* kv, const int32_t* seq_ids, const void* qkv, vo
     if (B == 0) return DEER_OK;
     const int Hkv = kv->d.n_kv_heads, D = kv->d.head_dim;
     const long long items = (long long)B * k * (Hq + Hkv + (qkv ? Hkv : 0));
-    qk_norm_rope_kernel<<<(unsigned)((items + 3) / 4), 128, 0, static_cast<cudaStream_t>(stream)>>>(
-        kv->d, seq_ids, static_cast<const __nv_bfloat16*>(qkv), static_cast<__nv_bfloat16*>(q), static_cast<__nv_bfloat16*>(k_blk),
-        static_cast<__nv_bfloat16*>(v_blk),
-        static_cast<const __nv_bfloat16*>(q_gamma), static_cast<const __nv_bfloat16*>(k_gamma), B, k, Hq, Hkv, D, eps,
-        log2((double)theta));
-    DEER_CUDA(cudaGetLastError());
+    DEER_CUDA(launch_pdl(qk_norm_rope_kernel, dim3((unsigned)((items + 3) / 4)), dim3(128), 0, static_cast<cudaStream_t>(stream), kv->d,
+                         seq_ids, static_cast<const __nv_bfloat16*>(qkv), static_cast<__nv_bfloat16*>(q),
+                         static_cast<__nv_bfloat16*>(k_blk), static_cast<__nv_bfloat16*>(v_blk),
+                         static_cast<const __nv_bfloat16*>(q_gamma), static_cast<const __nv_bfloat16*>(k_gamma), B, k, Hq, Hkv, D, eps,
+                         log2((double)theta)));
     return DEER_OK;
 }
 
@@ -166,8 +169,7 @@ extern "C" int deer_swiglu(const void* gate_up, void* y, int M, int I, void* str
     DEER_CHECK_ARG(M >= 0 && I > 0, DEER_ERR_INVALID_ARG, "deer_swiglu: bad sizes");
     if (M == 0) return DEER_OK;
     const long long total = (long long)M * I;
-    swiglu_kernel<<<(unsigned)((total + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const __nv_bfloat16*>(gate_up), static_cast<__nv_bfloat16*>(y), I, total);
-    DEER_CUDA(cudaGetLastError());
+    DEER_CUDA(launch_pdl(swiglu_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, static_cast<cudaStream_t>(stream),
+                         static_cast<const __nv_bfloat16*>(gate_up), static_cast<__nv_bfloat16*>(y), I, total));
     return DEER_OK;
 }

@@ -1,25 +1,61 @@
 // (2) LM head + selection: z = h w^T, p_AR = softmax(z / T) of Eq. 5 reduced
 // on the fly to argmax / log-sum-exp / the draft token's logit.
 //
-// Host entry points: argument checks and the workspace layout; the kernels are in lmhead_umma.cu.
+// Host entry points, the cross-part finalisation and the linear layer's reduction; the tensor-core kernels are
+// in lmhead_umma.cu.
 
 #include "lmhead.cuh"
 
 namespace lmhead {
 
 bool umma_supported(int M, int hid, int V);
-int launch_umma(const Params& p, int need_sum, cudaStream_t st, int* ksplit_out = nullptr);
+int launch_umma(const Params& p, int need_sum, int* nparts_out, cudaStream_t st, int* ksplit_out = nullptr);
 
-// Workspace of the selection: one Partial per (vocabulary part, row) for as many parts as there are SMs, then one
-// arrival word per tile of 128 rows.
-static size_t part_bytes(int M) { return ((size_t)deer_sm_count() * M * sizeof(Partial) + 255) / 256 * 256; }
+struct FinalizeArgs {
+    const Partial* part;
+    int nparts, M;
+    float inv_t_log2, inv_t;
+    int32_t* out_ids;
+    float* out_max_logprob;
+    float* out_lse;
+};
+
+// One warp per row: the lanes stride over the vocabulary parts, then merge by shuffles.
+__global__ void __launch_bounds__(256) lmhead_finalize_kernel(FinalizeArgs a) {
+    pdl_trigger();
+    const int m = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    pdl_wait();                                   // the partials of the LM-head kernel
+    if (m >= a.M) return;
+    float rm = -INFINITY, rs = 0.f;
+    int32_t ri = 0x7fffffff;
+    bool aborted = false;
+    for (int pt = lane; pt < a.nparts; pt += 32) {
+        const Partial pr = a.part[(size_t)pt * a.M + m];
+        aborted |= (pr.idx == PARTIAL_ABORTED);
+        merge_sel(rm, ri, rs, pr.m, pr.idx, pr.s, a.inv_t_log2);
+    }
+    aborted = __any_sync(0xffffffffu, aborted);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, rm, o);
+        const int32_t oi = __shfl_xor_sync(0xffffffffu, ri, o);
+        const float os = __shfl_xor_sync(0xffffffffu, rs, o);
+        merge_sel(rm, ri, rs, om, oi, os, a.inv_t_log2);
+    }
+    if (lane != 0) return;
+    if (a.out_ids) a.out_ids[m] = aborted ? PARTIAL_ABORTED : ri;
+    const float ls = logf(rs);
+    if (a.out_max_logprob) a.out_max_logprob[m] = -ls;          // max z - logsumexp(z), T = 1
+    if (a.out_lse) a.out_lse[m] = rm * a.inv_t + ls;            // logsumexp(z / T)
+}
 
 }  // namespace lmhead
 
 extern "C" size_t deer_lmhead_workspace_bytes(int M, int hid, int V) {
     (void)hid;
     if (M <= 0 || V <= 0) return 0;
-    return lmhead::part_bytes(M) + (size_t)((M + 127) / 128) * sizeof(unsigned long long);
+    return (size_t)deer_sm_count() * M * sizeof(lmhead::Partial);     // one Partial per (vocabulary part, row), a part per SM at most
 }
 
 extern "C" int deer_lmhead_select(const void* h, const void* w, int M, int hid, int V, int mode, float temperature,
@@ -56,7 +92,6 @@ extern "C" int deer_lmhead_select(const void* h, const void* w, int M, int hid, 
     p.hid = hid;
     p.V = V;
     p.inv_t_log2 = LOG2E / t;
-    p.inv_t = 1.f / t;
     p.draft_ids = (mode == DEER_SEL_SOFTMAX) ? draft_ids : nullptr;
     p.out_draft_logit = (mode == DEER_SEL_SOFTMAX) ? out_draft_logit : nullptr;
     p.out_logits = out_logits;
@@ -65,12 +100,21 @@ extern "C" int deer_lmhead_select(const void* h, const void* w, int M, int hid, 
     p.lin_part = nullptr;
     p.max_ksplit = 1;
     p.part = static_cast<Partial*>(workspace);
-    p.tickets = reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) + part_bytes(M));
-    p.epoch = deer_next_epoch();
-    p.out_ids = out_ids;
-    p.out_max_logprob = (mode == DEER_SEL_ARGMAX_LOGPROB) ? out_max_logprob : nullptr;
-    p.out_lse = (mode == DEER_SEL_SOFTMAX) ? out_lse : nullptr;
-    return launch_umma(p, mode != DEER_SEL_ARGMAX, st);
+    int nparts = 0;
+    const int rc = launch_umma(p, mode != DEER_SEL_ARGMAX, &nparts, st);
+    if (rc != DEER_OK) return rc;
+
+    FinalizeArgs fa;
+    fa.part = p.part;
+    fa.nparts = nparts;
+    fa.M = M;
+    fa.inv_t_log2 = p.inv_t_log2;
+    fa.inv_t = 1.f / t;
+    fa.out_ids = out_ids;
+    fa.out_max_logprob = (mode == DEER_SEL_ARGMAX_LOGPROB) ? out_max_logprob : nullptr;
+    fa.out_lse = (mode == DEER_SEL_SOFTMAX) ? out_lse : nullptr;
+    DEER_CUDA(launch_pdl(lmhead_finalize_kernel, dim3((M + 7) / 8), dim3(256), 0, st, fa));
+    return DEER_OK;
 }
 
 // ------------------------------------------------------------------------------
@@ -89,6 +133,8 @@ __global__ void __launch_bounds__(256) linear_reduce_kernel(const float* __restr
                                                             const __nv_bfloat16* __restrict__ residual,
                                                             __nv_bfloat16* __restrict__ y) {
     const long long i = ((long long)blockIdx.x * 256 + threadIdx.x) * 2;
+    pdl_trigger();
+    pdl_wait();                                   // the partial products of the kernel before
     if (i >= total) return;
     float s0 = 0.f, s1 = 0.f;
     if (i + 1 < total && (total & 1) == 0) {
@@ -153,19 +199,13 @@ extern "C" int deer_linear(const void* x, const void* w, const void* residual, v
         p.max_ksplit = 1;
     }
     p.part = nullptr;
-    p.tickets = nullptr;
-    p.epoch = 0;
-    p.inv_t = 1.f;
-    p.out_ids = nullptr;
-    p.out_max_logprob = nullptr;
-    p.out_lse = nullptr;
-    int ksplit = 1;
-    const int rc = launch_umma(p, 0, st, &ksplit);
+    int nparts = 0, ksplit = 1;
+    const int rc = launch_umma(p, 0, &nparts, st, &ksplit);
     if (rc != DEER_OK) return rc;
     if (ksplit > 1) {
         const long long total = (long long)M * N;
-        linear_reduce_kernel<<<(unsigned)((total / 2 + 256) / 256), 256, 0, st>>>(p.lin_part, ksplit, total, p.residual, p.out_bf16);
-        DEER_CUDA(cudaGetLastError());
+        DEER_CUDA(launch_pdl(linear_reduce_kernel, dim3((unsigned)((total / 2 + 256) / 256)), dim3(256), 0, st,
+                             (const float*)p.lin_part, ksplit, total, p.residual, p.out_bf16));
     }
     return DEER_OK;
 }

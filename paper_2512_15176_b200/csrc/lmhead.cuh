@@ -23,7 +23,6 @@ struct Params {
     const __nv_bfloat16* w;      // [V][hid]
     int M, hid, V;
     float inv_t_log2;            // log2(e) / T
-    float inv_t;                 // 1 / T
     const int32_t* draft_ids;    // [M] or null
     float* out_draft_logit;      // [M] or null
     float* out_logits;           // [M][V] or null
@@ -32,11 +31,6 @@ struct Params {
     float* lin_part;             // linear layer: room for max_ksplit partial products [M][V] fp32, or null
     int max_ksplit;
     Partial* part;               // [nparts][M]
-    unsigned long long* tickets; // [row tiles] arrival words of the blocks that share a row tile (selection only)
-    uint32_t epoch;              // this call's tag in those words (never 0)
-    int32_t* out_ids;            // [M]  selection outputs, written by the block that arrives last at its row tile
-    float* out_max_logprob;      // [M] or null
-    float* out_lse;              // [M] or null
 };
 
 __device__ __forceinline__ void merge_sel(float& m, int32_t& idx, float& s, float m2, int32_t idx2, float s2, float inv_t_log2) {

@@ -18,11 +18,11 @@
 //
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (+ TMEM owner),
 // warps 2..5 = epilogue (one TMEM lane quarter each).  The blocks that share a
-// row tile leave their (max, argmax, sum exp) per row in the workspace; the one
-// that arrives last merges them and writes the call's outputs, so there is no
-// second kernel.  All waits are bounded: a wait that runs out raises the block's
-// abort flag, every role leaves its loop, TMEM is freed and the kernel returns;
-// the rows of such a block get the id -2 (linear-layer mode: its tiles stay
+// row tile leave their (max, argmax, sum exp) per row in the workspace; a small
+// second kernel, launched so that it is resident before this one ends, merges
+// them.  All waits are bounded: a wait that runs out raises the block's abort
+// flag, every role leaves its loop, TMEM is freed and the kernel returns; the
+// rows of such a block get the id -2 (linear-layer mode: its tiles stay
 // unwritten).
 
 #include "lmhead.cuh"
@@ -63,12 +63,6 @@ struct Args {
     int ksplit;              // linear-layer mode, few output columns: the contraction is cut into ksplit ranges, one per
     float* lin_part;         // blockIdx.y / nparts; the partial sums go to lin_part[ksplit][M][V] (fp32) and are added up after
     Partial* part;           // [nparts][M]
-    unsigned long long* tickets;   // [row tiles of 128] arrival words of the blocks sharing a row tile
-    uint32_t epoch;          // this call's tag in them
-    float inv_t;             // 1 / T
-    int32_t* out_ids;        // [M]
-    float* out_max_logprob;  // [M] or null: max z - logsumexp(z)
-    float* out_lse;          // [M] or null: logsumexp(z / T)
 };
 
 // One 16-column slice of an accumulator row: optional store, draft-token pick, running selection.
@@ -194,7 +188,7 @@ constexpr int STAGING_BYTES = 4 * 2 * 4096;   // per epilogue warp two 32-row x 
 template <bool PAIR>
 __device__ __forceinline__ void epilogue(const Args& a, const CUtensorMap* tm_z, int quarter, int lane, int m0, int part,
                                          const Tiles& tl, uint32_t tmem_base, uint32_t tfull0,
-                                         uint32_t tempty0, uint32_t staging, volatile int* abort_flag, volatile int* last_flag) {
+                                         uint32_t tempty0, uint32_t staging, volatile int* abort_flag) {
     const int row = quarter * 32 + lane;
     const int grow = m0 + row;
     const bool row_ok = grow < a.M;
@@ -254,64 +248,14 @@ __device__ __forceinline__ void epilogue(const Args& a, const CUtensorMap* tm_z,
         }
     }
     if (lane == 0) bulk_wait<0>();               // the staging area outlives every store that reads it
-    if (a.out_bf16 || m0 >= a.M) return;            // block-uniform: a linear layer, or a pair's second tile beyond M
-    if (row_ok) {
+    if (row_ok && !a.out_bf16) {
         Partial pr;
         pr.m = run_m;
         pr.idx = run_i;
         pr.s = a.need_sum ? run_s : 1.f;
         pr.pad = 0;
-        if (*abort_flag) pr.idx = PARTIAL_ABORTED;     // the merge below turns this into an id of -2
+        if (*abort_flag) pr.idx = PARTIAL_ABORTED;     // the finalisation turns this into ids of -2
         a.part[(size_t)part * a.M + grow] = pr;
-    }
-    // ---- the block that arrives last at this row tile merges the parts of its rows ----
-    __threadfence();
-    asm volatile("bar.sync 1, 128;" ::: "memory");     // the four epilogue warps
-    if (quarter == 0 && lane == 0) *last_flag = arrive_last(a.tickets + m0 / BM, a.epoch, (uint32_t)a.nparts) ? 1 : 0;
-    asm volatile("bar.sync 1, 128;" ::: "memory");
-    if (!*last_flag) return;
-    __threadfence();
-    const int rows = min(BM, a.M - m0);
-    constexpr int RQ = 4;                              // rows a warp merges at a time: their loads are in flight together
-    for (int r0 = quarter * RQ; r0 < rows; r0 += 4 * RQ) {
-        float rm[RQ], rs[RQ];
-        int32_t ri[RQ];
-        bool aborted = false;
-#pragma unroll
-        for (int q = 0; q < RQ; ++q) {
-            rm[q] = -INFINITY;
-            rs[q] = 0.f;
-            ri[q] = 0x7fffffff;
-        }
-        for (int pt = lane; pt < a.nparts; pt += 32) {
-            int4 raw[RQ];
-#pragma unroll
-            for (int q = 0; q < RQ; ++q)
-                raw[q] = __ldcg(reinterpret_cast<const int4*>(a.part + (size_t)pt * a.M + m0 + min(r0 + q, rows - 1)));
-#pragma unroll
-            for (int q = 0; q < RQ; ++q) {
-                aborted |= (raw[q].y == PARTIAL_ABORTED);
-                merge_sel(rm[q], ri[q], rs[q], __int_as_float(raw[q].x), raw[q].y, __int_as_float(raw[q].z), a.c2);
-            }
-        }
-        aborted = __any_sync(0xffffffffu, aborted);
-#pragma unroll
-        for (int q = 0; q < RQ; ++q) {
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                const float om = __shfl_xor_sync(0xffffffffu, rm[q], o);
-                const int32_t oi = __shfl_xor_sync(0xffffffffu, ri[q], o);
-                const float os = __shfl_xor_sync(0xffffffffu, rs[q], o);
-                merge_sel(rm[q], ri[q], rs[q], om, oi, os, a.c2);
-            }
-            const int m = m0 + r0 + q;
-            if (lane == 0 && r0 + q < rows) {
-                a.out_ids[m] = aborted ? PARTIAL_ABORTED : ri[q];
-                const float ls = logf(rs[q]);
-                if (a.out_max_logprob) a.out_max_logprob[m] = -ls;          // max z - logsumexp(z), T = 1
-                if (a.out_lse) a.out_lse[m] = rm[q] * a.inv_t + ls;          // logsumexp(z / T)
-            }
-        }
     }
 }
 
@@ -356,13 +300,20 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
         *abort_flag = 0;
         mbar_init_fence();
     }
+    if (warp == 0 && lane == 0) {
+        prefetch_tensormap(&tm_h);
+        prefetch_tensormap(&tm_w_hi);
+        prefetch_tensormap(&tm_w_lo);
+    }
     if (warp == 1) {
         tmem_alloc(smem_u32(tmem_slot), 512);
     }
+    pdl_trigger();
     tcgen05_fence_before();
     __syncthreads();
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();                                   // everything above needed no input; h (and what follows) does
 
     // Accumulator rows at or beyond h_box_rows are never read back, and row i of an MMA depends on row i
     // of its 128-row operand only, so the h atom holds just h_box_rows rows: the rest of the 16 KB the
@@ -420,7 +371,7 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
     } else {
         // ---------------- epilogue: 4 warps, one TMEM lane quarter each ----------------
         epilogue<false>(a, &tm_z, warp & 3, lane, m0, part, tl, tmem_base, tfull_bar(0), tempty_bar(0),
-                        smem_base + (uint32_t)(a.stages * stage_bytes), abort_flag, abort_flag + 1);
+                        smem_base + (uint32_t)(a.stages * stage_bytes), abort_flag);
     }
 
     // ---- tear-down ------------------------------------------------------------
@@ -486,12 +437,19 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
         *abort_flag = 0;
         mbar_init_fence();
     }
+    if (warp == 0 && lane == 0) {
+        prefetch_tensormap(&tm_h);
+        prefetch_tensormap(&tm_w_hi);
+        prefetch_tensormap(&tm_w_lo);
+    }
     if (warp == 1) tmem_alloc_pair(smem_u32(tmem_slot), 512);
+    pdl_trigger();
     tcgen05_fence_before();
     __syncthreads();
     cluster_sync();                              // the peer's barriers exist before anything signals them
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();                                   // everything above needed no input; h (and what follows) does
 
     if (warp == 0) {
         // ---------------- TMA producer (each block: its 128 rows of h, its half of the weight tile) ----------------
@@ -549,7 +507,7 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
     } else {
         // ---------------- epilogue: 4 warps in each block, one TMEM lane quarter each ----------------
         epilogue<true>(a, &tm_z, warp & 3, lane, m0, part, tl, tmem_base, tfull_bar(0), tempty_bar(0),
-                       smem_base + (uint32_t)(a.stages * stage_bytes), abort_flag, abort_flag + 1);
+                       smem_base + (uint32_t)(a.stages * stage_bytes), abort_flag);
     }
 
     // ---- tear-down: neither block leaves while the other may still signal it or read its shared memory ----
@@ -580,9 +538,9 @@ static int make_operand_map(CUtensorMap* tm, const void* base, uint64_t rows, ui
 
 bool umma_supported(int M, int hid, int V) { return M > 0 && hid % umma::BK == 0 && hid >= umma::BK && V >= 16; }
 
-// Launches the tcgen05 kernel (selection: outputs written by the kernel itself; linear layer: *ksplit_out tells
-// whether partial products are left to be summed).
-int launch_umma(const Params& p, int need_sum, cudaStream_t st, int* ksplit_out) {
+// Launches the tcgen05 kernel.  Selection: *nparts_out vocabulary parts per row are left for the finalisation;
+// linear layer: *ksplit_out tells whether partial products are left to be summed.
+int launch_umma(const Params& p, int need_sum, int* nparts_out, cudaStream_t st, int* ksplit_out) {
     using namespace umma;
     const int sms = deer_sm_count();
     // more than 128 block rows: pairs of blocks share the weight tiles (256 rows per pair)
@@ -635,12 +593,6 @@ int launch_umma(const Params& p, int need_sum, cudaStream_t st, int* ksplit_out)
     a.ksplit = ksplit;
     a.lin_part = p.lin_part;
     a.part = p.part;
-    a.tickets = p.tickets;
-    a.epoch = p.epoch;
-    a.inv_t = p.inv_t;
-    a.out_ids = p.out_ids;
-    a.out_max_logprob = p.out_max_logprob;
-    a.out_lse = p.out_lse;
     CUtensorMap tm_h, tm_w_hi, tm_w_lo;
     int rc = make_operand_map(&tm_h, p.h, (uint64_t)p.M, (uint64_t)p.hid, (uint32_t)a.h_box_rows);
     if (rc != DEER_OK) return rc;
@@ -661,12 +613,13 @@ int launch_umma(const Params& p, int need_sum, cudaStream_t st, int* ksplit_out)
     if (ksplit_out) *ksplit_out = ksplit;
     if (pair) {
         DEER_CUDA(cudaFuncSetAttribute(lmhead_umma_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
-        lmhead_umma_pair_kernel<<<grid, umma::THREADS, smem_bytes, st>>>(tm_h, tm_w_hi, tm_w_lo, tm_z, a);
+        DEER_CUDA(launch_pdl(lmhead_umma_pair_kernel, grid, dim3(umma::THREADS), (size_t)smem_bytes, st, tm_h, tm_w_hi, tm_w_lo, tm_z, a));
     } else {
         DEER_CUDA(cudaFuncSetAttribute(lmhead_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
-        lmhead_umma_kernel<<<grid, umma::THREADS, smem_bytes, st>>>(tm_h, tm_w_hi, tm_w_lo, tm_z, a);
+        DEER_CUDA(launch_pdl(lmhead_umma_kernel, grid, dim3(umma::THREADS), (size_t)smem_bytes, st, tm_h, tm_w_hi, tm_w_lo, tm_z, a));
     }
     DEER_CUDA(cudaGetLastError());
+    *nparts_out = nparts;
     return DEER_OK;
 }
 

@@ -59,6 +59,10 @@ class VerifyStep:
         self.side = torch.cuda.Stream(device=dev) if (sample and overlap_draft_stats) else None
         self._stats_forked = False
         self.bonus = False              # the k rows are k-1 drafts + one more row (deer_accept's DEER_ACC_BONUS)
+        # sampling: top-k / nucleus truncation of the verifier's distribution ahead of the acceptance (0 / 1.0 = off)
+        self.top_k, self.top_p = 0, 1.0
+        self.tau = torch.empty(M, dtype=f32, device=dev) if sample else None
+        self.lse_trunc = torch.empty(M, dtype=f32, device=dev) if sample else None
 
     # ---- inputs -------------------------------------------------------------
     def load(self, q=None, k_blk=None, v_blk=None, h=None, draft_ids=None, q_logits=None, u=None, r=None):
@@ -111,10 +115,16 @@ class VerifyStep:
             self._stats_forked = False
         extra = L.DEER_ACC_BONUS if self.bonus else 0
         if c.mode == "sample":
-            L.deer_accept((L.DEER_ACC_SAMPLE_PRESTATS if prestats else L.DEER_ACC_SAMPLE) | extra, c.B, c.k, c.V, self.draft_ids, None,
-                          self.logits, self.lse, self.draft_logit,
-                          c.temperature, self.q_logits, self.u, self.r, self.eos_id, self.accept_len, self.out_ids, self.n_out,
-                          self.acc_ws)
+            mode = (L.DEER_ACC_SAMPLE_PRESTATS if prestats else L.DEER_ACC_SAMPLE) | extra
+            if self.top_k > 0 or self.top_p < 1.0:
+                L.deer_truncate(self.logits, self.lse, c.temperature, self.top_k, self.top_p, self.tau, self.lse_trunc)
+                L.deer_accept_truncated(mode, c.B, c.k, c.V, self.draft_ids, None, self.logits, self.lse_trunc, self.draft_logit,
+                                        self.tau, c.temperature, self.q_logits, self.u, self.r, self.eos_id, self.accept_len,
+                                        self.out_ids, self.n_out, self.acc_ws)
+            else:
+                L.deer_accept(mode, c.B, c.k, c.V, self.draft_ids, None, self.logits, self.lse, self.draft_logit,
+                              c.temperature, self.q_logits, self.u, self.r, self.eos_id, self.accept_len, self.out_ids,
+                              self.n_out, self.acc_ws)
         else:
             L.deer_accept(L.DEER_ACC_GREEDY | extra, c.B, c.k, c.V, self.draft_ids, self.target_ids, None, None, None, 1.0, None,
                           None, None, self.eos_id, self.accept_len, self.out_ids, self.n_out, None)
@@ -140,8 +150,8 @@ class VerifyStep:
     #: kernels launched by one run(), by mode (attention + merge, LM head, reserve + commit, acceptance)
     def launches_per_step(self) -> int:
         if self.cfg.mask == MASK_BIDIR:
-            return 3
-        return 2 + 1 + 2 + (4 if self.cfg.mode == "sample" else 1)
+            return 4
+        return 2 + 2 + 2 + (2 if self.cfg.mode == "sample" else 1)
 
 
 class DecodeLoop:
@@ -165,6 +175,8 @@ class DecodeLoop:
         self.finished = torch.zeros(B, dtype=torch.int32, device=dev)
         self.keep = torch.zeros(B, dtype=torch.int32, device=dev)
 
+        self.appended = torch.zeros(B, dtype=torch.int32, device=dev)
+
     def one_pass(self):
         vs = self.vs
         vs.reserve()
@@ -172,8 +184,69 @@ class DecodeLoop:
         vs.lmhead()
         vs.accept()
         L.deer_emit(vs.accept_len, vs.out_ids, vs.n_out, self.eos_id, self.tokens, self.n_tokens, self.finished, self.keep,
-                    L.DEER_EMIT_PENDING if self.pending else 0)
+                    L.DEER_EMIT_PENDING if self.pending else 0, appended=self.appended)
         L.deer_kv_commit(vs.kv, vs.seq_ids, self.keep, vs.cfg.k)
+
+
+class DrafterBlock:
+    """The drafter's side of a pass (Section 3.2's block proposal, Section 4's several
+    denoising iterations, and the drafter-side cache the appendix on the DLLM KV cache
+    looks forward to) on the library's calls.  ``fill()`` runs iterations of
+    bidirectional block attention over the drafter's own paged cache -> LM head
+    (argmax + its log-probability) -> ``deer_refill`` until every row is decoded or
+    ``max_iters`` is reached, entirely on the device; the decoded tokens are the
+    draft block.  ``refresh(appended)`` brings the drafter's cache up to date after
+    the verify step: the tokens that joined the output are attended as decoded rows,
+    their keys and values appended, and the cache commits ``appended`` rows.
+    There is no drafter model here: the per-iteration query/key/value rows and hidden
+    states are inputs (``load``)."""
+
+    def __init__(self, cfg: StepConfig, kv: L.KVCache, w: torch.Tensor, max_seq_len: int, device="cuda"):
+        self.cfg, self.kv, self.w, self.max_seq_len = cfg, kv, w, int(max_seq_len)
+        B, k, Hq, Hkv, D, M = cfg.B, cfg.k, cfg.Hq, cfg.Hkv, cfg.D, cfg.M
+        bf, i32, f32 = torch.bfloat16, torch.int32, torch.float32
+        self.seq_ids = torch.arange(B, dtype=i32, device=device)
+        self.q = torch.empty(B, k, Hq, D, dtype=bf, device=device)
+        self.k_blk = torch.empty(B, k, Hkv, D, dtype=bf, device=device)
+        self.v_blk = torch.empty(B, k, Hkv, D, dtype=bf, device=device)
+        self.attn_out = torch.empty(B, k, Hq, D, dtype=bf, device=device)
+        self.h = torch.empty(M, cfg.hid, dtype=bf, device=device)
+        self.ids = torch.empty(B, k, dtype=i32, device=device)
+        self.logprob = torch.empty(B, k, dtype=f32, device=device)
+        self.row_state = torch.ones(B, k, dtype=i32, device=device)
+        self.tokens = torch.full((B, k), -1, dtype=i32, device=device)
+        self.left = torch.zeros(B, dtype=i32, device=device)
+        self.attn_ws = _ws(L.deer_block_attn_workspace_bytes(B, k, Hq, Hkv, D, self.max_seq_len), device)
+        self.lm_ws = _ws(L.deer_lmhead_workspace_bytes(M, cfg.hid, cfg.V), device)
+        self.scale = 1.0 / math.sqrt(D)
+
+    def load(self, q=None, k_blk=None, v_blk=None, h=None):
+        for dst, src in ((self.q, q), (self.k_blk, k_blk), (self.v_blk, v_blk), (self.h, h)):
+            if src is not None:
+                dst.copy_(src.to(dst.dtype).reshape(dst.shape), non_blocking=True)
+
+    def start_block(self):
+        """A fresh block: every row masked, no token yet."""
+        self.row_state.fill_(1)
+        self.tokens.fill_(-1)
+
+    def iteration(self, log_threshold: float):
+        """One denoising iteration on the current row states (inputs as loaded)."""
+        L.deer_block_attn_rows(self.kv, self.seq_ids, self.q, self.k_blk, self.v_blk, self.attn_out, self.row_state,
+                               L.DEER_MASK_BIDIR, False, self.scale, self.max_seq_len, self.attn_ws)
+        L.deer_lmhead_select(self.h, self.w, L.DEER_SEL_ARGMAX_LOGPROB, 1.0, None, self.ids, self.logprob, None, None, None,
+                             self.lm_ws)
+        L.deer_refill(self.ids, self.logprob, log_threshold, self.row_state, self.tokens, self.left)
+
+    def refresh(self, appended: torch.Tensor):
+        """After the verify step: the drafter's keys and values of the tokens that joined the output (inputs as
+        loaded: their rows first) go into its cache."""
+        k = self.cfg.k
+        L.deer_refresh_rows(appended, self.row_state)
+        L.deer_kv_reserve(self.kv, self.seq_ids, k)
+        L.deer_block_attn_rows(self.kv, self.seq_ids, self.q, self.k_blk, self.v_blk, self.attn_out, self.row_state,
+                               L.DEER_MASK_BIDIR, True, self.scale, self.max_seq_len, self.attn_ws)
+        L.deer_kv_commit(self.kv, self.seq_ids, appended, k)
 
 
 class VerifierLayer:

@@ -73,7 +73,13 @@ def test_host_side_argument_validation(lib):
     assert lib.deer_accept(1, 1, 8, 100, fake, None, None, None, None, 1.0, None, None, None, -1, fake, fake, fake, None, 0, None) == L.DEER_ERR_INVALID_ARG
     assert lib.deer_accept(0, 0, 8, 100, fake, fake, None, None, None, 1.0, None, None, None, -1, fake, fake, fake, None, 0, None) == L.DEER_OK
     assert lib.deer_accept_workspace_bytes(0, 16, 32, 151936) == 0
-    assert lib.deer_accept_workspace_bytes(1, 16, 32, 151936) > 2 * 16 * 151936 * 8
+    need = lib.deer_accept_workspace_bytes(1, 16, 32, 151936)
+    assert 2 * 16 * 32 * 4 < need < (1 << 20)          # per-row statistics and per-slice sums; no copy of a vocabulary row
+    # truncation: null outputs, non-positive temperature or top_p
+    assert lib.deer_truncate(4, 100, fake, fake, 1.0, 5, 0.9, None, fake, None) == L.DEER_ERR_INVALID_ARG
+    assert lib.deer_truncate(4, 100, fake, fake, 0.0, 5, 0.9, fake, fake, None) == L.DEER_ERR_INVALID_ARG
+    assert lib.deer_truncate(4, 100, fake, fake, 1.0, 5, 0.0, fake, fake, None) == L.DEER_ERR_INVALID_ARG
+    assert lib.deer_truncate(0, 100, fake, fake, 1.0, 5, 0.9, fake, fake, None) == L.DEER_OK
 
 
 def test_workload_is_deterministic_and_shaped():
