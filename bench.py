@@ -272,10 +272,13 @@ class Flusher:
         self.rd.max()
 
 
-def measure(cfg, steps, warmup, dev, peaks, flush, world=1, rank=0, with_e2e=False, clock_sampler=None, device_weights=False):
+def measure(cfg, steps, warmup, dev, peaks, flush, world=1, rank=0, with_e2e=False, clock_sampler=None, device_weights=False,
+            consecutive=False):
     """Times ``steps`` steps of ``cfg`` on the current device.  Returns a dict with the step time (events at the two
     ends of the step's graph), the phase split (a second graph with events between the phases), the roofline of the
-    LM-head call and of the whole step."""
+    LM-head call and of the whole step.  ``consecutive``: the timed steps follow one another on the same cache --
+    every step commits what it accepted, the contexts grow, and each step gets freshly planted drafts -- instead of
+    starting from the same state each time."""
     from paper_2512_15176_b200 import binding as L
     from paper_2512_15176_b200.runner import VerifyStep
     import torch.distributed as dist
@@ -289,7 +292,8 @@ def measure(cfg, steps, warmup, dev, peaks, flush, world=1, rank=0, with_e2e=Fal
     del kp, vp
     saved = [t.clone() for t in (kv.page_table, kv.seq_len, kv.n_pages, kv.free_stack, kv.free_top)]
     w = head_weights(cfg, dev, device_weights)
-    vs = VerifyStep(cfg, kv, w, int(lengths.max()), device=dev, store_logits=None if cfg.mode == "sample" else False)
+    max_seq_len = int(lengths.max()) + cfg.growth           # consecutive steps grow the contexts
+    vs = VerifyStep(cfg, kv, w, max_seq_len, device=dev, store_logits=None if cfg.mode == "sample" else False)
     q, kb, vb = W.block_qkv(cfg)
     h = W.hidden(cfg)
     vs.load(q, kb, vb, h)
@@ -313,6 +317,11 @@ def measure(cfg, steps, warmup, dev, peaks, flush, world=1, rank=0, with_e2e=Fal
         drafts = W.plant_drafts(cfg, target, W.planted_prefix_lengths(cfg))
         vs.load(draft_ids=drafts)
     bidir = cfg.mask == W.MASK_BIDIR
+    step_drafts = None
+    if consecutive and greedy and not bidir:
+        # the hidden states stay, so the targets do; every step gets its own planted prefix lengths
+        step_drafts = torch.stack([torch.from_numpy(W.plant_drafts(cfg, target, W.planted_prefix_lengths(cfg, s), s))
+                                   for s in range(steps)]).to(dev)
 
     def phase_attn():
         if not bidir:
@@ -369,8 +378,16 @@ def measure(cfg, steps, warmup, dev, peaks, flush, world=1, rank=0, with_e2e=Fal
     torch.cuda.synchronize()
     wall0 = time.perf_counter()
     step_ms = []
-    for _ in range(steps):
-        replay(g_step)
+    if step_drafts is not None:
+        restore()
+    for s_i in range(steps):
+        if step_drafts is not None:
+            vs.draft_ids.copy_(step_drafts[s_i])
+            flush()
+            g_step.replay()
+            torch.cuda.synchronize()
+        else:
+            replay(g_step)
         step_ms.append(ev_step[0].elapsed_time(ev_step[3]))
     torch.cuda.synchronize()
     wall = time.perf_counter() - wall0
@@ -405,7 +422,7 @@ def measure(cfg, steps, warmup, dev, peaks, flush, world=1, rank=0, with_e2e=Fal
             torch.cuda.synchronize()
             t0 = time.perf_counter()
             L.deer_verify_step_host(kv, sd, w, hq, hkb, hvb, hh, hd, cfg.B, cfg.k, cfg.Hq, cfg.hid, cfg.V, vs.scale,
-                                    int(lengths.max()), ha, ho, hn, stream=es)
+                                    max_seq_len, ha, ho, hn, stream=es)
             dt = time.perf_counter() - t0
             if s >= 3:
                 e2e_s += dt
@@ -444,6 +461,7 @@ def measure(cfg, steps, warmup, dev, peaks, flush, world=1, rank=0, with_e2e=Fal
                    "accept_commit_ms": acc_s * 1e3, "step_ms_with_phase_events": float(m[:, 2].mean())},
         "gpu_launches": steps * vs.launches_per_step(),
         "kv_status": status, "accepted_tokens_last_step": accepted, "wall_s_timed_loop": wall,
+        "consecutive_steps": bool(step_drafts is not None),
         "flops_per_step": fl["total"], "clocks": clocks,
     }
     if greedy and with_e2e:
@@ -452,6 +470,73 @@ def measure(cfg, steps, warmup, dev, peaks, flush, world=1, rank=0, with_e2e=Fal
     del vs, kv, w
     torch.cuda.empty_cache()
     return out
+
+
+def measure_layer(name, dev, peaks, flush, B, k, ctx, hid, Hq, Hkv, D, inter, moe=None, layers=1, steps=20):
+    """One verifier layer (or a short stack) around the block attention at the M = B k rows of a draft block, on the
+    fused calls, replayed from a CUDA graph with L2 flushed between replays.  The floor is the time the weights
+    (for a routed MLP: the experts the rows really chose) and the live KV take at the measured HBM peak."""
+    from paper_2512_15176_b200 import binding as L
+    from paper_2512_15176_b200.runner import VerifierStack
+    cfg = W.StepConfig(name, B, Hq, Hkv, D, k, hid, 64, (ctx, ctx), seed=34, growth=k)
+    lengths = W.seq_lengths(cfg)
+    lay = W.kv_layout(cfg, lengths)
+    i32 = lambda a: torch.from_numpy(a.copy()).to(device=dev, dtype=torch.int32).contiguous()
+    shared = [i32(a) for a in (lay.page_table, lay.seq_len, lay.n_pages, lay.free_stack, lay.free_top)]
+    mk = lambda n, shape, sig: W.normal(34, n, shape, sig, device=str(dev))
+    QD, KD = Hq * D, Hkv * D
+    kvs, weights, w_bytes = [], [], 0
+    for l in range(layers):
+        kp, vp = W.kv_pools(cfg.with_(seed=34 + l), lay.num_pages, device=str(dev), sigma=1.0)
+        kvs.append(L.KVCache(kp, vp, *shared))
+        w = {"ln1": mk(f"ln1{l}", (hid,), 1.0), "ln2": mk(f"ln2{l}", (hid,), 1.0), "q_norm": mk(f"qn{l}", (D,), 1.0),
+             "k_norm": mk(f"kn{l}", (D,), 1.0), "wqkv": mk(f"wqkv{l}", (QD + 2 * KD, hid), hid ** -0.5),
+             "wo": mk(f"wo{l}", (hid, QD), QD ** -0.5)}
+        if moe:
+            E, top_k = moe
+            w.update({"w_router": mk(f"wr{l}", (E, hid), hid ** -0.5 * 3.0), "w_gate_up": mk(f"wgue{l}", (E, 2 * inter, hid), hid ** -0.5),
+                      "w_down": mk(f"wde{l}", (E, hid, inter), inter ** -0.5)})
+        else:
+            w.update({"wgu": mk(f"wgu{l}", (2 * inter, hid), hid ** -0.5), "wd": mk(f"wd{l}", (hid, inter), inter ** -0.5)})
+        weights.append(w)
+    x = mk("x", (cfg.M, hid), 1.0)
+    stack = VerifierStack(cfg, kvs, weights, ctx + k, inter, fused=True, moe=moe)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())           # the weights and pools were drawn on the current stream
+    with torch.cuda.stream(side):
+        for _ in range(3):
+            stack.forward(x)
+        side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            stack.forward(x)
+    torch.cuda.synchronize()
+    # bytes the layers must move: dense weights once, the chosen experts' matrices once, the live KV once
+    for l, w in enumerate(weights):
+        w_bytes += sum(t.numel() * 2 for n, t in w.items() if n in ("wqkv", "wo", "wgu", "wd", "w_router"))
+        if moe:
+            e_ids = torch.empty(cfg.M, moe[1], dtype=torch.int32, device=dev)
+            e_w = torch.empty(cfg.M, moe[1], dtype=torch.float32, device=dev)
+            L.deer_moe_route(stack.layers[l].xn2, w["w_router"], moe[1], e_ids, e_w)
+            torch.cuda.synchronize()
+            w_bytes += int(torch.unique(e_ids).numel()) * 3 * inter * hid * 2
+    kv_bytes = layers * W.algorithmic_bytes(cfg, lengths)["attn"]
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for e0, e1 in ev:
+        flush()
+        e0.record()
+        g.replay()
+        e1.record()
+    torch.cuda.synchronize()
+    ms = float(np.mean([e0.elapsed_time(e1) for e0, e1 in ev]))
+    floor_ms = (w_bytes + kv_bytes) / (peaks["hbm_gbs"] * 1e9) * 1e3
+    status = [L.deer_kv_status(kv) for kv in kvs]
+    del stack, kvs, weights
+    torch.cuda.empty_cache()
+    return {"config": {"workload": name, "B": B, "k": k, "ctx": ctx, "hid": hid, "Hq": Hq, "Hkv": Hkv, "D": D, "inter": inter,
+                       "experts": list(moe) if moe else None, "layers": layers, "calls": "fused"},
+            "ms_per_layer": ms / layers, "bytes_per_layer": (w_bytes + kv_bytes) / layers,
+            "gbs": (w_bytes + kv_bytes) / ms / 1e6, "frac_of_hbm_floor": floor_ms / ms, "kv_status": max(status)}
 
 
 def run_ours(args, cfg):
@@ -480,6 +565,13 @@ def run_ours(args, cfg):
             r = measure(c, extra_steps, 3, dev, peaks, flush, clock_sampler=ClockSampler(local), device_weights=True)
             r.pop("flops_per_step", None)
             others[name] = r
+        # the rest of a verifier layer around the attention, per layer: Qwen3-8B's dense layer and Qwen3-30B-A3B's
+        # routed one, at one sequence's block and at sixteen
+        others["layer-qwen3-8b-B1"] = measure_layer("layer-qwen3-8b", dev, peaks, flush, 1, 32, 4096, 4096, 32, 8, 128, 12288, layers=2)
+        others["layer-qwen3-30b-a3b-B1"] = measure_layer("layer-qwen3-30b-a3b", dev, peaks, flush, 1, 32, 4096, 2048, 32, 4, 128, 768,
+                                                         moe=(128, 8), layers=2)
+        others["layer-qwen3-30b-a3b-B16"] = measure_layer("layer-qwen3-30b-a3b", dev, peaks, flush, 16, 32, 4096, 2048, 32, 4, 128, 768,
+                                                          moe=(128, 8), layers=1)
     if rank != 0:
         if world > 1:
             import torch.distributed as dist
@@ -515,8 +607,9 @@ def run_ours(args, cfg):
 # ---------------------------------------------------------------------------
 
 def run_sweep(args):
-    """All 96 points (batch x context x block size x mask), each timed for ``--steps`` steps of the single-step
-    graph; writes profiles/sweep.md and prints one JSON line with the table's rows."""
+    """All 96 points (batch x context x block size x mask).  A causal point runs ``--steps`` (default here: 64)
+    consecutive verify steps on one cache, committing every step; a bidirectional point the drafter's block fill
+    that many times (it commits nothing).  Writes the table to --sweep-out and prints one JSON line with its rows."""
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
     from paper_2512_15176_b200 import binding as L
@@ -528,10 +621,10 @@ def run_sweep(args):
         for B in (1, 4, 16, 64):
             for ctx in (1024, 4096, 16384, 32768):
                 for k in (8, 16, 32):
-                    cfg = W.sweep_config(B, ctx, k, mask, steps=1)
+                    cfg = W.sweep_config(B, ctx, k, mask, steps=args.steps + 8)
                     if mask == W.MASK_BIDIR:
                         cfg = cfg.with_(mode="argmax_logprob")
-                    r = measure(cfg, args.steps, 3, dev, peaks, flush, device_weights=True)
+                    r = measure(cfg, args.steps, 3, dev, peaks, flush, device_weights=True, consecutive=True)
                     rows.append({"B": B, "ctx": ctx, "k": k, "mask": mname, "ms_per_step": r["ms_per_step"],
                                  "tokens_per_s": r["value"], "attn_ms": r["phases"]["attn_ms"],
                                  "attn_frac_of_floor": r["phases"]["attn_frac_of_floor"], "lmhead_ms": r["phases"]["lmhead_ms"],
@@ -541,9 +634,11 @@ def run_sweep(args):
     path = os.path.join(ROOT, args.sweep_out)
     with open(path, "w") as f:
         f.write("# Sweep: batch x context x block size x mask (32q/8kv heads, head_dim 128, hidden 4096, vocabulary 151936)\n\n")
-        f.write(f"`python bench.py --sweep --steps {args.steps}` on one B200; ragged lengths in [ctx/2, ctx], greedy acceptance "
-                "with planted prefixes (causal) or argmax + max log-probability (bidirectional block fill); one CUDA graph per "
-                "step, L2 flushed between steps.  Peaks: HBM %.1f GB/s, bf16 %.1f TFLOP/s sustained (%s).  `of floor` = time "
+        f.write(f"`python bench.py --sweep --steps {args.steps}` on one B200; ragged lengths in [ctx/2, ctx]; causal points: "
+                f"{args.steps} consecutive verify steps on one cache (greedy acceptance, geometric planted prefixes drawn anew "
+                "every step, every step commits, the contexts grow); bidirectional points: the drafter's block fill (argmax + "
+                "max log-probability; commits nothing); one CUDA graph per step, L2 flushed between steps; times are means "
+                "over the steps.  Peaks: HBM %.1f GB/s, bf16 %.1f TFLOP/s sustained (%s).  `of floor` = time "
                 "the algorithmic bytes / flops take at those peaks over the measured time.\n\n" %
                 (peaks["hbm_gbs"], peaks["bf16_tflops_sustained"], peaks["source"]))
         f.write("| mask | B | ctx | k | step us | verified tok/s | attention us | attn of floor | LM head us | LM head of peak | accept+commit us | step of floor |\n")
@@ -559,7 +654,7 @@ def run_sweep(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=None, help="timed steps (default 200; 64 with --sweep)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=1, help="workload index 0..3 (1 = Qwen3-8B-shaped verify step)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -571,6 +666,8 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="time every point of the sweep and write the table")
     ap.add_argument("--sweep-out", default="profiles/sweep.md")
     args = ap.parse_args()
+    if args.steps is None:
+        args.steps = 64 if args.sweep else 200
     if args.sweep:
         run_sweep(args)
         return

@@ -392,6 +392,25 @@ int deer_qkv_split_norm_rope(deer_kv* kv, const int32_t* seq_ids, const void* qk
                              void* stream);
 int deer_swiglu(const void* gate_up, void* y, int M, int I, void* stream);
 
+/* A projection and the row-wise step that follows it in the layer, as one call each (fewer kernels: at the few rows of a
+ * draft block the layer is bound by launches as much as by the weight stream).  Same arithmetic and the same bf16
+ * roundings as the separate calls.
+ * deer_linear_qkv_rope: the fused Q/K/V projection of x bf16 [B k][hid] by w_qkv bf16 [(Hq + 2 Hkv) D][hid], then
+ *   deer_qkv_split_norm_rope on its result.
+ * deer_linear_residual_norm: y = x w^T + residual (bf16 [M][N], residual may be NULL), and, if gamma != NULL,
+ *   y_norm = RMSNorm(y) * gamma -- the output or down projection together with the normalisation that opens the
+ *   next sub-layer.
+ * deer_linear_swiglu: y bf16 [M][I] = silu(g) * u with (g, u) = the columns (2 c, 2 c + 1) of x w_pairs^T; w_pairs bf16
+ *   [2 I][hid] holds channel c's gate row at 2 c and its up row at 2 c + 1 (a layout the caller prepares once).
+ *   workspace  >= deer_layer_workspace_bytes(M, K, N) bytes (N = the projection's output columns), 16-byte aligned. */
+size_t deer_layer_workspace_bytes(int M, int K, int N);
+int deer_linear_qkv_rope(deer_kv* kv, const int32_t* seq_ids, const void* x, const void* w_qkv, void* q, void* k_blk, void* v_blk,
+                         const void* q_gamma, const void* k_gamma, int B, int k, int Hq, int hid, float eps, float theta,
+                         void* workspace, size_t workspace_bytes, void* stream);
+int deer_linear_residual_norm(const void* x, const void* w, const void* residual, const void* gamma, void* y, void* y_norm,
+                              int M, int K, int N, float eps, void* workspace, size_t workspace_bytes, void* stream);
+int deer_linear_swiglu(const void* x, const void* w_pairs, void* y, int M, int K, int I, void* stream);
+
 /* The routed mixture-of-experts MLP of a Qwen3-MoE-style layer (the paper's largest verifier, Qwen3-30B-A3B, has one
  * in every layer) at M = B k rows:
  *   probabilities = softmax(x w_router^T) over the E experts (fp32);  each row's top_k experts, lowest index among

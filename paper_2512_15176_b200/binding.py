@@ -31,6 +31,7 @@ EXPORTS = [
     "deer_linear_workspace_bytes", "deer_linear", "deer_rmsnorm", "deer_qk_norm_rope", "deer_qkv_split_norm_rope", "deer_swiglu",
     "deer_truncate", "deer_accept_truncated", "deer_block_attn_rows", "deer_refill", "deer_refresh_rows",
     "deer_moe_workspace_bytes", "deer_moe_route", "deer_moe_mlp",
+    "deer_layer_workspace_bytes", "deer_linear_qkv_rope", "deer_linear_residual_norm", "deer_linear_swiglu",
 ]
 
 
@@ -110,6 +111,13 @@ def lib() -> ctypes.CDLL:
                                        c_int, c_int, c_float, c_int, c_void_p, c_size_t, c_void_p]
     L.deer_refill.argtypes = [c_int, c_int, c_void_p, c_void_p, c_float, c_void_p, c_void_p, c_void_p, c_void_p]
     L.deer_refresh_rows.argtypes = [c_int, c_int, c_void_p, c_void_p, c_void_p]
+    L.deer_layer_workspace_bytes.restype = c_size_t
+    L.deer_layer_workspace_bytes.argtypes = [c_int] * 3
+    L.deer_linear_qkv_rope.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                       c_int, c_int, c_int, c_int, c_float, c_float, c_void_p, c_size_t, c_void_p]
+    L.deer_linear_residual_norm.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int, c_int,
+                                            c_float, c_void_p, c_size_t, c_void_p]
+    L.deer_linear_swiglu.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p]
     L.deer_moe_workspace_bytes.restype = c_size_t
     L.deer_moe_workspace_bytes.argtypes = [c_int] * 5
     L.deer_moe_route.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p]
@@ -304,6 +312,30 @@ def deer_qkv_split_norm_rope(kv: "KVCache", seq_ids, qkv, q, k_blk, v_blk, q_gam
 def deer_swiglu(gate_up, y, stream=None):
     M, I = y.shape
     _check(lib().deer_swiglu(_ptr(gate_up), _ptr(y), M, I, _stream(stream)))
+
+
+def deer_layer_workspace_bytes(M, K, N) -> int:
+    return lib().deer_layer_workspace_bytes(M, K, N)
+
+
+def deer_linear_qkv_rope(kv: "KVCache", seq_ids, x, w_qkv, q, k_blk, v_blk, q_gamma, k_gamma, eps, theta, workspace, stream=None):
+    B, k, Hq, _ = q.shape
+    _check(lib().deer_linear_qkv_rope(kv.handle, _ptr(seq_ids), _ptr(x), _ptr(w_qkv), _ptr(q), _ptr(k_blk), _ptr(v_blk), _ptr(q_gamma),
+                                      _ptr(k_gamma), B, k, Hq, x.shape[1], float(eps), float(theta), _ptr(workspace),
+                                      workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def deer_linear_residual_norm(x, w, y, residual=None, gamma=None, y_norm=None, eps=1e-6, workspace=None, stream=None):
+    M, K = x.shape
+    _check(lib().deer_linear_residual_norm(_ptr(x), _ptr(w), _ptr(residual), _ptr(gamma), _ptr(y), _ptr(y_norm), M, K, w.shape[0],
+                                           float(eps), _ptr(workspace),
+                                           workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                                           _stream(stream)))
+
+
+def deer_linear_swiglu(x, w_pairs, y, stream=None):
+    M, K = x.shape
+    _check(lib().deer_linear_swiglu(_ptr(x), _ptr(w_pairs), _ptr(y), M, K, y.shape[1], _stream(stream)))
 
 
 def deer_moe_workspace_bytes(M, hid, E, I, top_k) -> int:

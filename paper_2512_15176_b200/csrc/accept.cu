@@ -13,7 +13,7 @@
 
 namespace {
 
-constexpr int NS = 32;             // vocabulary slices per rejected row
+constexpr int NS = 128;            // vocabulary slices per rejected row (NS <= RES_THREADS)
 constexpr int RES_THREADS = 256;
 
 // ---------------------------------------------------------------- greedy

@@ -25,8 +25,9 @@
 // gets a tcgen05.mma accepted only every ~100 cycles whatever its size, so
 // three warps issue -- even S tiles, odd S tiles, O -- and their streams
 // interleave on the tensor pipe.  The softmax warps hold one row per thread (no
-// shuffles) and keep a running maximum that is only raised when a tile exceeds
-// it by 2^8 (the accumulator in TMEM is rescaled then, which is rare).
+// shuffles); the exponentials of a segment are taken against its first tile's
+// row maximum, which is raised only when a later tile's exponentials outgrow
+// 2^32 (the accumulator in TMEM is rescaled then, which is rare).
 //
 // Warp roles: warp 0 = TMA producer, warps 1-2 = issuers of S (warp 1 owns the
 // TMEM allocation), warp 3 = issuer of O, warps 4..7 = softmax (one TMEM lane
@@ -55,7 +56,7 @@ constexpr int TMEM_COLS = 512;                 // S0..S3 [0,256)  P0 [256,288)  
 constexpr int P_COL = 256;
 constexpr int O_COL = 384;
 constexpr int MAX_SEGS = 48;                   // segments listed at a time; longer shares go in several rounds
-constexpr float RESCALE_STEP = 8.f;            // raise the running maximum only when a tile exceeds it by 2^8
+constexpr float RESCALE_SUM = 4294967296.f;    // 2^32: a row sum over one tile beyond this raises the running maximum
 // Slot layout.  A K (or V) tile of 64 tokens x 128 dims is 16 KB of 1 KB swizzle atoms (8 tokens x 64 dims).
 //   prefix tile: [page 0..3][token group 0..1][dim half 0..1][8 tokens][128 B] -- what one 5-D TMA box per page
 //                writes; atoms of one dim half are 2 KB apart along the tokens, the two halves 1 KB apart.
@@ -468,56 +469,70 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         for (int c = 0; c < ATT_TILE; ++c)
                             if (c >= tile_valid) sr[c] = 0xff800000u;
                     }
-                    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains: one warp per scheduler needs the ILP
+                    // Row maximum of this tile (log2 domain, scaled); four chains: one warp per scheduler needs the ILP.
+                    auto tile_max = [&]() -> float {
+                        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                    for (int c = 0; c < ATT_TILE; c += 4) {
-                        mx4[0] = fmaxf(mx4[0], __uint_as_float(sr[c]));
-                        mx4[1] = fmaxf(mx4[1], __uint_as_float(sr[c + 1]));
-                        mx4[2] = fmaxf(mx4[2], __uint_as_float(sr[c + 2]));
-                        mx4[3] = fmaxf(mx4[3], __uint_as_float(sr[c + 3]));
-                    }
-                    float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-                    mx *= p.scale_log2;                       // scale > 0, so the maximum commutes with it
-                    if (!(mx > -INFINITY)) mx = 0.f;          // lanes without a query row
+                        for (int c = 0; c < ATT_TILE; c += 4) {
+                            mx4[0] = fmaxf(mx4[0], __uint_as_float(sr[c]));
+                            mx4[1] = fmaxf(mx4[1], __uint_as_float(sr[c + 1]));
+                            mx4[2] = fmaxf(mx4[2], __uint_as_float(sr[c + 2]));
+                            mx4[3] = fmaxf(mx4[3], __uint_as_float(sr[c + 3]));
+                        }
+                        float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                        mx *= p.scale_log2;                   // scale > 0, so the maximum commutes with it
+                        return (mx > -INFINITY) ? mx : 0.f;   // lanes without a query row, rows that see nothing here
+                    };
+                    // P = 2^(s * scale - m), two bf16 per TMEM column, and the row's sum over this tile
+                    uint32_t pr[ATT_TILE / 2];
+                    float tile_sum;
+                    auto exponentials = [&]() {
+                        float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+                        const float neg_m = -m_run;
+#pragma unroll
+                        for (int c = 0; c < ATT_TILE; c += 2) {
+                            const float p0 = ex2_approx(fmaf(__uint_as_float(sr[c]), p.scale_log2, neg_m));
+                            const float p1 = ex2_approx(fmaf(__uint_as_float(sr[c + 1]), p.scale_log2, neg_m));
+                            sum4[(c >> 1) & 3] += p0 + p1;
+                            pr[c >> 1] = pack_bf16(p0, p1);
+                        }
+                        tile_sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+                    };
 
+                    // The reference point m of a segment is its first tile's row maximum.  Subtracting a maximum only
+                    // keeps the exponentials in range -- the quotient O / l does not depend on m -- so later tiles
+                    // are taken against the same m without looking for their maximum, and m is raised (O and l
+                    // rescaled, as any online softmax does) only when a row's sum over a tile shows that its
+                    // exponentials have grown past 2^32 (or are not finite): rare, and then the tile is redone.
                     // o_done completes one phase per tile, and a parity wait can only tell the current phase from the
                     // one before it: every phase is waited for, in order -- phase it-1 during tile it.
                     bool o_synced = (it == 0);
-                    if (t == g.t_a) {
-                        m_run = mx;                           // a segment starts a new accumulation
-                    } else if (__any_sync(0xffffffffu, mx > m_run + RESCALE_STEP)) {
-                        // raise the maximum: O and the row sum shrink by 2^(old - new); O must be final up to the last tile
-                        const float m_new = fmaxf(m_run, mx);
+                    if (t == g.t_a) m_run = tile_max();       // a segment starts a new accumulation
+                    exponentials();
+                    if (__any_sync(0xffffffffu, !(tile_sum < RESCALE_SUM))) {
+                        const float m_new = fmaxf(m_run, tile_max());
                         const float alpha = ex2_approx(m_run - m_new);
-                        const bool od = mbar_wait(bar(BAR_O_DONE), (uint32_t)(it - 1) & 1u, abort_flag);
+                        const bool od = o_synced || mbar_wait(bar(BAR_O_DONE), (uint32_t)(it - 1) & 1u, abort_flag);
                         if (!__all_sync(0xffffffffu, od)) { alive = false; break; }
                         o_synced = true;
                         tcgen05_fence_after();
+                        if (t != g.t_a) {                     // O holds the segment's tiles so far: shrink it by 2^(old - new)
 #pragma unroll
-                        for (int cc = 0; cc < HD / 32; ++cc) {
-                            uint32_t orow[32];
-                            TMEM_LD_X32(t_lane + O_COL + cc * 32, orow);
-                            tmem_wait_ld();
+                            for (int cc = 0; cc < HD / 32; ++cc) {
+                                uint32_t orow[32];
+                                TMEM_LD_X32(t_lane + O_COL + cc * 32, orow);
+                                tmem_wait_ld();
 #pragma unroll
-                            for (int c = 0; c < 32; ++c) orow[c] = __float_as_uint(__uint_as_float(orow[c]) * alpha);
-                            TMEM_ST_X32(t_lane + O_COL + cc * 32, orow);
+                                for (int c = 0; c < 32; ++c) orow[c] = __float_as_uint(__uint_as_float(orow[c]) * alpha);
+                                TMEM_ST_X32(t_lane + O_COL + cc * 32, orow);
+                            }
+                            tmem_wait_st();
                         }
-                        tmem_wait_st();
                         l_run *= alpha;
                         m_run = m_new;
+                        exponentials();
                     }
-                    // P = 2^(s * scale - m), two bf16 per TMEM column, in this tile's P buffer
-                    uint32_t pr[ATT_TILE / 2];
-                    float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-                    const float neg_m = -m_run;
-#pragma unroll
-                    for (int c = 0; c < ATT_TILE; c += 2) {
-                        const float p0 = ex2_approx(fmaf(__uint_as_float(sr[c]), p.scale_log2, neg_m));
-                        const float p1 = ex2_approx(fmaf(__uint_as_float(sr[c + 1]), p.scale_log2, neg_m));
-                        sum4[(c >> 1) & 3] += p0 + p1;
-                        pr[c >> 1] = pack_bf16(p0, p1);
-                    }
-                    l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+                    l_run += tile_sum;
                     if (!o_synced) {                          // normally long complete; also frees this P buffer (tile it-2)
                         const bool od = mbar_wait(bar(BAR_O_DONE), (uint32_t)(it - 1) & 1u, abort_flag);
                         if (!__all_sync(0xffffffffu, od)) { alive = false; break; }

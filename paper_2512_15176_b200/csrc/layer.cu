@@ -41,9 +41,12 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const __nv_bfloat16* __res
 // One warp per (block row, head) of q or k: optional RMSNorm over the head's D values, then the rotation of the
 // pairs (d, d + D/2) by pos * theta^(-2d/D).  In place.
 // With `qkv` (the packed output [B k][(Hq + 2 Hkv) D] of one fused projection) the values are read from there and
-// q, k_blk, v_blk are written (v copied as it is); without it q and k_blk are transformed in place.
+// q, k_blk, v_blk are written (v copied as it is); without it q and k_blk are transformed in place.  With `part`
+// the packed output does not exist yet: it is the sum of `ksplit` fp32 partial products [ksplit][B k][(Hq + 2 Hkv) D]
+// (the projection's contraction was cut into ranges), summed here and rounded to bf16 as the projection would have.
 __global__ void __launch_bounds__(128) qk_norm_rope_kernel(deer_kv_desc kv, const int32_t* __restrict__ seq_ids,
-                                                           const __nv_bfloat16* __restrict__ qkv,
+                                                           const __nv_bfloat16* __restrict__ qkv, const float* __restrict__ part,
+                                                           int ksplit,
                                                            __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ kb,
                                                            __nv_bfloat16* __restrict__ vb,
                                                            const __nv_bfloat16* __restrict__ q_gamma,
@@ -54,13 +57,22 @@ __global__ void __launch_bounds__(128) qk_norm_rope_kernel(deer_kv_desc kv, cons
     pdl_trigger();
     pdl_wait();
     const long long nq = (long long)B * k * Hq, nk = (long long)B * k * Hkv;
-    if (item >= nq + nk + (qkv ? nk : 0)) return;
+    const bool packed = qkv != nullptr || part != nullptr;
+    if (item >= nq + nk + (packed ? nk : 0)) return;
+    const long long part_stride = (long long)B * k * (Hq + 2 * Hkv) * D;
+    // element `off` of the packed projection output, as a bf16-rounded float
+    auto packed_at = [&](long long off) -> float {
+        if (!part) return __bfloat162float(qkv[off]);
+        float sum = 0.f;
+        for (int s = 0; s < ksplit; ++s) sum += part[(long long)s * part_stride + off];
+        return __bfloat162float(__float2bfloat16(sum));
+    };
     if (item >= nq + nk) {                                        // a V head: copy out of the packed rows
         const long long r = item - nq - nk;
         const long long bi = r / Hkv;
         const int hh = (int)(r % Hkv);
-        const __nv_bfloat16* src = qkv + (bi * (Hq + 2 * Hkv) + Hq + Hkv + hh) * D;
-        for (int d = lane; d < D; d += 32) vb[r * D + d] = src[d];
+        const long long src = (bi * (Hq + 2 * Hkv) + Hq + Hkv + hh) * D;
+        for (int d = lane; d < D; d += 32) vb[r * D + d] = __float2bfloat16(packed_at(src + d));
         return;
     }
     const bool is_q = item < nq;
@@ -69,7 +81,7 @@ __global__ void __launch_bounds__(128) qk_norm_rope_kernel(deer_kv_desc kv, cons
     const long long bi = r / H;                                   // b * k + i
     const int b = (int)(bi / k), i = (int)(bi % k);
     __nv_bfloat16* v = (is_q ? q : kb) + r * D;
-    const __nv_bfloat16* in = qkv ? qkv + (bi * (Hq + 2 * Hkv) + (is_q ? 0 : Hq) + (r % H)) * D : v;
+    const long long in_off = (bi * (Hq + 2 * Hkv) + (is_q ? 0 : Hq) + (r % H)) * D;
     const __nv_bfloat16* gamma = is_q ? q_gamma : k_gamma;
     const int s = seq_ids[b];
     const int n = (s >= 0 && s < kv.max_seqs) ? kv.seq_len[s] : 0;
@@ -83,8 +95,8 @@ __global__ void __launch_bounds__(128) qk_norm_rope_kernel(deer_kv_desc kv, cons
         const int d = lane + 32 * t;
         a[t] = c[t] = 0.f;
         if (d < half) {
-            a[t] = __bfloat162float(in[d]);
-            c[t] = __bfloat162float(in[d + half]);
+            a[t] = packed ? packed_at(in_off + d) : __bfloat162float(v[d]);
+            c[t] = packed ? packed_at(in_off + d + half) : __bfloat162float(v[d + half]);
             ss += a[t] * a[t] + c[t] * c[t];
         }
     }
@@ -134,8 +146,9 @@ extern "C" int deer_rmsnorm(const void* x, const void* gamma, void* y, int M, in
     return DEER_OK;
 }
 
-static int qk_norm_rope(deer_kv* kv, const int32_t* seq_ids, const void* qkv, void* q, void* k_blk, void* v_blk, const void* q_gamma,
-                        const void* k_gamma, int B, int k, int Hq, float eps, float theta, void* stream) {
+static int qk_norm_rope(deer_kv* kv, const int32_t* seq_ids, const void* qkv, const float* part, int ksplit, void* q, void* k_blk,
+                        void* v_blk, const void* q_gamma, const void* k_gamma, int B, int k, int Hq, float eps, float theta,
+                        void* stream) {
     DEER_CHECK_ARG(kv && seq_ids && q && k_blk, DEER_ERR_INVALID_ARG, "deer_qk_norm_rope: null argument");
     DEER_CHECK_ARG((q_gamma == nullptr) == (k_gamma == nullptr), DEER_ERR_INVALID_ARG,
                    "deer_qk_norm_rope: q_gamma and k_gamma come together");
@@ -143,9 +156,9 @@ static int qk_norm_rope(deer_kv* kv, const int32_t* seq_ids, const void* qkv, vo
                    "deer_qk_norm_rope: bad sizes");
     if (B == 0) return DEER_OK;
     const int Hkv = kv->d.n_kv_heads, D = kv->d.head_dim;
-    const long long items = (long long)B * k * (Hq + Hkv + (qkv ? Hkv : 0));
+    const long long items = (long long)B * k * (Hq + Hkv + ((qkv || part) ? Hkv : 0));
     DEER_CUDA(launch_pdl(qk_norm_rope_kernel, dim3((unsigned)((items + 3) / 4)), dim3(128), 0, static_cast<cudaStream_t>(stream), kv->d,
-                         seq_ids, static_cast<const __nv_bfloat16*>(qkv), static_cast<__nv_bfloat16*>(q),
+                         seq_ids, static_cast<const __nv_bfloat16*>(qkv), part, ksplit, static_cast<__nv_bfloat16*>(q),
                          static_cast<__nv_bfloat16*>(k_blk), static_cast<__nv_bfloat16*>(v_blk),
                          static_cast<const __nv_bfloat16*>(q_gamma), static_cast<const __nv_bfloat16*>(k_gamma), B, k, Hq, Hkv, D, eps,
                          log2((double)theta)));
@@ -154,14 +167,119 @@ static int qk_norm_rope(deer_kv* kv, const int32_t* seq_ids, const void* qkv, vo
 
 extern "C" int deer_qk_norm_rope(deer_kv* kv, const int32_t* seq_ids, void* q, void* k_blk, const void* q_gamma,
                                  const void* k_gamma, int B, int k, int Hq, float eps, float theta, void* stream) {
-    return qk_norm_rope(kv, seq_ids, nullptr, q, k_blk, nullptr, q_gamma, k_gamma, B, k, Hq, eps, theta, stream);
+    return qk_norm_rope(kv, seq_ids, nullptr, nullptr, 1, q, k_blk, nullptr, q_gamma, k_gamma, B, k, Hq, eps, theta, stream);
 }
 
 extern "C" int deer_qkv_split_norm_rope(deer_kv* kv, const int32_t* seq_ids, const void* qkv, void* q, void* k_blk, void* v_blk,
                                         const void* q_gamma, const void* k_gamma, int B, int k, int Hq, float eps, float theta,
                                         void* stream) {
     DEER_CHECK_ARG(qkv && v_blk, DEER_ERR_INVALID_ARG, "deer_qkv_split_norm_rope: null argument");
-    return qk_norm_rope(kv, seq_ids, qkv, q, k_blk, v_blk, q_gamma, k_gamma, B, k, Hq, eps, theta, stream);
+    return qk_norm_rope(kv, seq_ids, qkv, nullptr, 1, q, k_blk, v_blk, q_gamma, k_gamma, B, k, Hq, eps, theta, stream);
+}
+
+// ---- a projection and the row-wise step behind it as one call ------------------------------------------------
+int deer_linear_for_tail(const void* x, const void* w, const void* residual, void* y_bf16, int M, int K, int N, void* workspace,
+                         size_t workspace_bytes, int* ksplit_out, cudaStream_t st);
+
+namespace {
+
+// One block per row: y = sum of the partial products (or the projection's bf16 output) + residual, rounded to bf16;
+// then, if gamma is given, y_norm = RMSNorm(y) * gamma over the rounded values (what a separate pass would read).
+__global__ void __launch_bounds__(256) residual_norm_tail_kernel(const float* __restrict__ part, int ksplit, const __nv_bfloat16* __restrict__ y_in,
+                                                                 const __nv_bfloat16* __restrict__ residual,
+                                                                 const __nv_bfloat16* __restrict__ gamma, __nv_bfloat16* __restrict__ y,
+                                                                 __nv_bfloat16* __restrict__ y_norm, int M, int N, float eps) {
+    __shared__ float red[8];
+    pdl_trigger();
+    pdl_wait();
+    const size_t row = blockIdx.x;
+    const size_t stride = (size_t)M * N;
+    float ss = 0.f;
+    for (int c = threadIdx.x; c < N; c += 256) {
+        const size_t o = row * N + c;
+        float v;
+        if (part) {
+            v = 0.f;
+            for (int s = 0; s < ksplit; ++s) v += part[(size_t)s * stride + o];
+            if (residual) v += __bfloat162float(residual[o]);
+        } else {
+            v = __bfloat162float(y_in[o]);                 // the projection added the residual itself
+        }
+        const __nv_bfloat16 vb = __float2bfloat16(v);
+        if (part) y[o] = vb;
+        const float vr = __bfloat162float(vb);
+        ss += vr * vr;
+    }
+    if (!gamma) return;
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += red[w];
+    const float inv = rsqrtf(tot / (float)N + eps);
+    for (int c = threadIdx.x; c < N; c += 256) {
+        const size_t o = row * N + c;
+        // this thread wrote y[o] itself a moment ago
+        y_norm[o] = __float2bfloat16(__bfloat162float(part ? y[o] : y_in[o]) * inv * __bfloat162float(gamma[c]));
+    }
+}
+
+}  // namespace
+
+extern "C" size_t deer_layer_workspace_bytes(int M, int K, int N) {
+    const size_t a = deer_linear_workspace_bytes(M, K, N), b = (size_t)(M > 0 ? M : 0) * (N > 0 ? N : 0) * 2;
+    return a > b ? a : b;
+}
+
+extern "C" int deer_linear_qkv_rope(deer_kv* kv, const int32_t* seq_ids, const void* x, const void* w_qkv, void* q, void* k_blk,
+                                    void* v_blk, const void* q_gamma, const void* k_gamma, int B, int k, int Hq, int hid, float eps,
+                                    float theta, void* workspace, size_t workspace_bytes, void* stream) {
+    DEER_CHECK_ARG(kv && seq_ids && x && w_qkv && q && k_blk && v_blk && workspace, DEER_ERR_INVALID_ARG,
+                   "deer_linear_qkv_rope: null argument");
+    DEER_CHECK_ARG(deer_aligned16(x) && deer_aligned16(w_qkv) && deer_aligned16(workspace), DEER_ERR_INVALID_ARG,
+                   "deer_linear_qkv_rope: pointers must be 16-byte aligned");
+    DEER_CHECK_ARG(B >= 0 && k >= 1 && k <= DEER_MAX_BLOCK && Hq > 0 && hid > 0 && hid % 64 == 0, DEER_ERR_INVALID_ARG,
+                   "deer_linear_qkv_rope: bad sizes");
+    if (B == 0) return DEER_OK;
+    const int M = B * k, N = (Hq + 2 * kv->d.n_kv_heads) * kv->d.head_dim;
+    DEER_CHECK_ARG(workspace_bytes >= deer_layer_workspace_bytes(M, hid, N), DEER_ERR_WORKSPACE,
+                   "deer_linear_qkv_rope: workspace of %zu bytes needed, %zu given", deer_layer_workspace_bytes(M, hid, N), workspace_bytes);
+    int ksplit = 1;
+    // if the contraction is not cut, the packed bf16 output takes the room the partial products would have had
+    const size_t lin_bytes = deer_linear_workspace_bytes(M, hid, N);
+    int rc = deer_linear_for_tail(x, w_qkv, nullptr, workspace, M, hid, N, lin_bytes ? workspace : nullptr, lin_bytes ? workspace_bytes : 0,
+                                  &ksplit, static_cast<cudaStream_t>(stream));
+    if (rc != DEER_OK) return rc;
+    // either the packed bf16 output or the partial products sit in the workspace now
+    return qk_norm_rope(kv, seq_ids, ksplit > 1 ? nullptr : workspace, ksplit > 1 ? static_cast<const float*>(workspace) : nullptr,
+                        ksplit, q, k_blk, v_blk, q_gamma, k_gamma, B, k, Hq, eps, theta, stream);
+}
+
+extern "C" int deer_linear_residual_norm(const void* x, const void* w, const void* residual, const void* gamma, void* y, void* y_norm,
+                                         int M, int K, int N, float eps, void* workspace, size_t workspace_bytes, void* stream) {
+    DEER_CHECK_ARG(x && w && y && (!gamma || y_norm), DEER_ERR_INVALID_ARG, "deer_linear_residual_norm: null argument");
+    DEER_CHECK_ARG(deer_aligned16(x) && deer_aligned16(w) && deer_aligned16(y) && deer_aligned16(residual) && deer_aligned16(workspace),
+                   DEER_ERR_INVALID_ARG, "deer_linear_residual_norm: pointers must be 16-byte aligned");
+    DEER_CHECK_ARG(M >= 0 && N >= 16 && K > 0 && K % 64 == 0 && eps >= 0.f, DEER_ERR_INVALID_ARG, "deer_linear_residual_norm: bad sizes");
+    if (M == 0) return DEER_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int ksplit = 1;
+    int rc = deer_linear_for_tail(x, w, residual, y, M, K, N, workspace, workspace_bytes, &ksplit, st);
+    if (rc != DEER_OK) return rc;
+    if (ksplit > 1) {
+        DEER_CUDA(launch_pdl(residual_norm_tail_kernel, dim3(M), dim3(256), 0, st, (const float*)workspace, ksplit,
+                             (const __nv_bfloat16*)nullptr, static_cast<const __nv_bfloat16*>(residual),
+                             static_cast<const __nv_bfloat16*>(gamma), static_cast<__nv_bfloat16*>(y), static_cast<__nv_bfloat16*>(y_norm),
+                             M, N, eps));
+        return DEER_OK;
+    }
+    // the contraction was not cut: the projection has written y + residual itself, the tail only normalises
+    if (!gamma) return DEER_OK;
+    DEER_CUDA(launch_pdl(residual_norm_tail_kernel, dim3(M), dim3(256), 0, st, (const float*)nullptr, 1, (const __nv_bfloat16*)y,
+                         (const __nv_bfloat16*)nullptr, static_cast<const __nv_bfloat16*>(gamma), static_cast<__nv_bfloat16*>(y),
+                         static_cast<__nv_bfloat16*>(y_norm), M, N, eps));
+    return DEER_OK;
 }
 
 extern "C" int deer_swiglu(const void* gate_up, void* y, int M, int I, void* stream) {

@@ -97,6 +97,7 @@ extern "C" int deer_lmhead_select(const void* h, const void* w, int M, int hid, 
     p.out_logits = out_logits;
     p.out_bf16 = nullptr;
     p.residual = nullptr;
+    p.swiglu = 0;
     p.lin_part = nullptr;
     p.max_ksplit = 1;
     p.part = static_cast<Partial*>(workspace);
@@ -160,6 +161,48 @@ __global__ void __launch_bounds__(256) linear_reduce_kernel(const float* __restr
 
 }  // namespace
 
+// y = x w^T on the tensor-core kernels, in one of three forms:
+//   ksplit_out == nullptr / *ksplit_out == 1   y (+ residual) written in bf16 by the kernel itself;
+//   *ksplit_out > 1                             fp32 partial products [ksplit][M][N] left in `workspace` for the caller's
+//                                               tail kernel to sum (residual is then the tail's business);
+//   swiglu                                      columns are (gate, up) pairs: y [M][N / 2] = silu(gate) * up.
+static int linear_launch(const void* x, const void* w, const void* residual, void* y, int M, int K, int N, int swiglu,
+                         void* workspace, size_t workspace_bytes, bool leave_partials, int* ksplit_out, cudaStream_t st) {
+    using namespace lmhead;
+    Params p;
+    p.h = static_cast<const __nv_bfloat16*>(x);
+    p.w = static_cast<const __nv_bfloat16*>(w);
+    p.M = M;
+    p.hid = K;
+    p.V = N;
+    p.inv_t_log2 = LOG2E;
+    p.draft_ids = nullptr;
+    p.out_draft_logit = nullptr;
+    p.out_logits = nullptr;
+    p.out_bf16 = static_cast<__nv_bfloat16*>(y);
+    p.residual = static_cast<const __nv_bfloat16*>(residual);
+    p.swiglu = swiglu;
+    // the contraction is cut only as far as the caller's workspace holds the partial products (none: never)
+    p.lin_part = swiglu ? nullptr : static_cast<float*>(workspace);
+    p.max_ksplit = (workspace && !swiglu) ? (int)(workspace_bytes / ((size_t)M * N * sizeof(float))) : 1;
+    if (p.max_ksplit > LIN_MAX_KSPLIT) p.max_ksplit = LIN_MAX_KSPLIT;
+    if (p.max_ksplit < 2) {
+        p.lin_part = nullptr;
+        p.max_ksplit = 1;
+    }
+    p.part = nullptr;
+    int nparts = 0, ksplit = 1;
+    const int rc = launch_umma(p, 0, &nparts, st, &ksplit);
+    if (rc != DEER_OK) return rc;
+    if (ksplit_out) *ksplit_out = ksplit;
+    if (ksplit > 1 && !leave_partials) {
+        const long long total = (long long)M * N;
+        DEER_CUDA(launch_pdl(linear_reduce_kernel, dim3((unsigned)((total / 2 + 256) / 256)), dim3(256), 0, st,
+                             (const float*)p.lin_part, ksplit, total, p.residual, p.out_bf16));
+    }
+    return DEER_OK;
+}
+
 extern "C" size_t deer_linear_workspace_bytes(int M, int K, int N) {
     (void)K;
     if (M <= 0 || N <= 0 || M > 128) return 0;            // larger M never cuts the contraction
@@ -177,35 +220,23 @@ extern "C" int deer_linear(const void* x, const void* w, const void* residual, v
     DEER_CHECK_ARG(umma_supported(M > 0 ? M : 1, K, N), DEER_ERR_UNSUPPORTED,
                    "deer_linear: K must be a multiple of 64 and N at least 16");
     if (M == 0) return DEER_OK;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    Params p;
-    p.h = static_cast<const __nv_bfloat16*>(x);
-    p.w = static_cast<const __nv_bfloat16*>(w);
-    p.M = M;
-    p.hid = K;
-    p.V = N;
-    p.inv_t_log2 = LOG2E;
-    p.draft_ids = nullptr;
-    p.out_draft_logit = nullptr;
-    p.out_logits = nullptr;
-    p.out_bf16 = static_cast<__nv_bfloat16*>(y);
-    p.residual = static_cast<const __nv_bfloat16*>(residual);
-    // the contraction is cut only as far as the caller's workspace holds the partial products (none: never)
-    p.lin_part = static_cast<float*>(workspace);
-    p.max_ksplit = workspace ? (int)(workspace_bytes / ((size_t)M * N * sizeof(float))) : 1;
-    if (p.max_ksplit > LIN_MAX_KSPLIT) p.max_ksplit = LIN_MAX_KSPLIT;
-    if (p.max_ksplit < 2) {
-        p.lin_part = nullptr;
-        p.max_ksplit = 1;
-    }
-    p.part = nullptr;
-    int nparts = 0, ksplit = 1;
-    const int rc = launch_umma(p, 0, &nparts, st, &ksplit);
-    if (rc != DEER_OK) return rc;
-    if (ksplit > 1) {
-        const long long total = (long long)M * N;
-        DEER_CUDA(launch_pdl(linear_reduce_kernel, dim3((unsigned)((total / 2 + 256) / 256)), dim3(256), 0, st,
-                             (const float*)p.lin_part, ksplit, total, p.residual, p.out_bf16));
-    }
-    return DEER_OK;
+    return linear_launch(x, w, residual, y, M, K, N, 0, workspace, workspace_bytes, false, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int deer_linear_swiglu(const void* x, const void* w_pairs, void* y, int M, int K, int I, void* stream) {
+    using namespace lmhead;
+    DEER_CHECK_ARG(x && w_pairs && y, DEER_ERR_INVALID_ARG, "deer_linear_swiglu: null argument");
+    DEER_CHECK_ARG(deer_aligned16(x) && deer_aligned16(w_pairs) && deer_aligned16(y), DEER_ERR_INVALID_ARG,
+                   "deer_linear_swiglu: pointers must be 16-byte aligned");
+    DEER_CHECK_ARG(M >= 0 && I > 0 && K > 0, DEER_ERR_INVALID_ARG, "deer_linear_swiglu: bad sizes");
+    DEER_CHECK_ARG(K % 64 == 0 && I % 8 == 0, DEER_ERR_UNSUPPORTED, "deer_linear_swiglu: K must be a multiple of 64, I of 8");
+    if (M == 0) return DEER_OK;
+    return linear_launch(x, w_pairs, nullptr, y, M, K, 2 * I, 1, nullptr, 0, false, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+// The projection whose tail another kernel takes over: leaves either bf16 y (+ residual) or fp32 partial products
+// without the residual (see linear_launch); *ksplit_out tells which.  Used by the fused layer calls in layer.cu.
+int deer_linear_for_tail(const void* x, const void* w, const void* residual, void* y_bf16, int M, int K, int N, void* workspace,
+                         size_t workspace_bytes, int* ksplit_out, cudaStream_t st) {
+    return linear_launch(x, w, residual, y_bf16, M, K, N, 0, workspace, workspace_bytes, true, ksplit_out, st);
 }

@@ -28,6 +28,7 @@ struct Params {
     float* out_logits;           // [M][V] or null
     __nv_bfloat16* out_bf16;     // [M][V] or null: plain linear layer, y = h w^T (+ residual), nothing selected
     const __nv_bfloat16* residual;   // [M][V] or null, added before the bf16 rounding
+    int swiglu;                  // linear layer: (gate, up) column pairs -> silu(gate) * up, out_bf16 [M][V / 2]
     float* lin_part;             // linear layer: room for max_ksplit partial products [M][V] fp32, or null
     int max_ksplit;
     Partial* part;               // [nparts][M]

@@ -60,6 +60,7 @@ struct Args {
     float* out_logits;
     __nv_bfloat16* out_bf16; // linear-layer mode: the product (+ residual) in bf16 is all that is written
     const __nv_bfloat16* residual;
+    int swiglu;              // linear-layer mode: columns come in (gate, up) pairs; out_bf16 [M][V / 2] gets silu(gate) * up
     int ksplit;              // linear-layer mode, few output columns: the contraction is cut into ksplit ranges, one per
     float* lin_part;         // blockIdx.y / nparts; the partial sums go to lin_part[ksplit][M][V] (fp32) and are added up after
     Partial* part;           // [nparts][M]
@@ -83,6 +84,31 @@ __device__ __forceinline__ void consume16(const uint32_t (&r)[16], int vbase, in
 #pragma unroll
             for (int j = 0; j < 16; ++j)
                 if (j < nv) dst[j] = __uint_as_float(r[j]);
+        }
+        return;
+    }
+    if (a.out_bf16 && a.swiglu) {
+        // gate / up interleaved: 16 columns = 8 (gate, up) pairs -> 8 activations = 16 contiguous bytes of the row;
+        // gate and up are rounded to bf16 first, as a layer that stores them would
+        __nv_bfloat16* dst = a.out_bf16 + (zrow + vbase) / 2;
+        float o[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float g = __bfloat162float(__float2bfloat16(__uint_as_float(r[2 * j])));
+            const float u = __bfloat162float(__float2bfloat16(__uint_as_float(r[2 * j + 1])));
+            o[j] = g / (1.f + __expf(-g)) * u;
+        }
+        if (nv == 16 && (((zrow + vbase) / 2) & 7) == 0) {
+            uint4 ov;
+            ov.x = pack_bf16(o[0], o[1]);
+            ov.y = pack_bf16(o[2], o[3]);
+            ov.z = pack_bf16(o[4], o[5]);
+            ov.w = pack_bf16(o[6], o[7]);
+            *reinterpret_cast<uint4*>(dst) = ov;
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (2 * j + 1 < nv) dst[j] = __float2bfloat16(o[j]);
         }
         return;
     }
@@ -300,10 +326,24 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
         *abort_flag = 0;
         mbar_init_fence();
     }
-    if (warp == 0 && lane == 0) {
+    // The weights are the model's: nothing that runs before this kernel writes them, so the first ring of weight
+    // tiles is requested right away -- before the tensor memory is there, and before the kernel ahead of this one
+    // in the stream has finished.  The h tiles of those stages follow once it has.
+    int pre = 0;                                  // stages whose weight tile was requested ahead (producer thread only)
+    if (tid == 0 && n_tiles > 0) {
         prefetch_tensormap(&tm_h);
-        prefetch_tensormap(&tm_w_hi);
-        prefetch_tensormap(&tm_w_lo);
+        int it = 0;
+        for (int t = 0; t < n_tiles && it < a.stages; ++t) {
+            int row0, g;
+            tile_span(tl, t, row0, g);
+            const CUtensorMap* tm_w = (g == a.gmax) ? &tm_w_hi : &tm_w_lo;
+            const uint32_t stage_tx = (uint32_t)(a.h_box_rows * 128 + g * 16 * 128);
+            for (int kb = 0; kb < KB && it < a.stages; ++kb, ++it) {
+                mbar_expect_tx(full_bar(it), stage_tx);
+                tma_load_2d(smem_base + it * stage_bytes + a.a_bytes, tm_w, (kb0 + kb) * BK, row0, full_bar(it));
+            }
+        }
+        pre = it;
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(tmem_slot), 512);
@@ -313,7 +353,7 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
     __syncthreads();
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    pdl_wait();                                   // everything above needed no input; h (and what follows) does
+    pdl_wait();                                   // h, the draft ids and every output depend on what ran before
 
     // Accumulator rows at or beyond h_box_rows are never read back, and row i of an MMA depends on row i
     // of its 128-row operand only, so the h atom holds just h_box_rows rows: the rest of the 16 KB the
@@ -330,11 +370,13 @@ lmhead_umma_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
                 const uint32_t stage_tx = (uint32_t)(a.h_box_rows * 128 + g * 16 * 128);
                 for (int kb = 0; kb < KB; ++kb, ++it) {
                     const int s = it % a.stages;
-                    const uint32_t ph = (uint32_t)(it / a.stages) & 1u;
-                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
-                    mbar_expect_tx(full_bar(s), stage_tx);
                     const uint32_t sa = smem_base + s * stage_bytes;
-                    tma_load_2d(sa + a.a_bytes, tm_w, (kb0 + kb) * BK, row0, full_bar(s));     // the whole N-row tile in one box
+                    if (it >= pre) {                       // the first `pre` weight tiles are on their way already
+                        const uint32_t ph = (uint32_t)(it / a.stages) & 1u;
+                        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+                        mbar_expect_tx(full_bar(s), stage_tx);
+                        tma_load_2d(sa + a.a_bytes, tm_w, (kb0 + kb) * BK, row0, full_bar(s));     // the whole N-row tile in one box
+                    }
                     tma_load_2d(sa, &tm_h, (kb0 + kb) * BK, m0, full_bar(s));
                 }
             }
@@ -591,6 +633,7 @@ int launch_umma(const Params& p, int need_sum, int* nparts_out, cudaStream_t st,
     a.out_bf16 = p.out_bf16;
     a.residual = p.residual;
     a.ksplit = ksplit;
+    a.swiglu = p.swiglu;
     a.lin_part = p.lin_part;
     a.part = p.part;
     CUtensorMap tm_h, tm_w_hi, tm_w_lo;

@@ -117,22 +117,30 @@ __global__ void __launch_bounds__(256) moe_route_kernel(const __nv_bfloat16* __r
                 be = oe;
             }
         }
-        if ((be & 31) == lane) v[be >> 5] = -1.f;                // taken
-        if (lane == t) {
-            chosen_w = bv / sum;
-            chosen_e = be;
+        const bool none = be >= E;                               // nothing left to choose from (fewer live experts than top_k, or
+                                                                 // probabilities that are not numbers): the choice stays empty
+        if (!none) {
+#pragma unroll
+            for (int j = 0; j < PER; ++j)
+                if (lane + 32 * j == be) v[j] = -1.f;            // taken
         }
-        tot += bv / sum;
+        if (lane == t) {
+            chosen_w = none ? 0.f : bv / sum;
+            chosen_e = none ? -1 : be;
+        }
+        if (!none) tot += bv / sum;
     }
     if (lane < top_k) {
         experts[(size_t)(m0 + r) * top_k + lane] = chosen_e;
-        weights[(size_t)(m0 + r) * top_k + lane] = renorm ? chosen_w / tot : chosen_w;
+        weights[(size_t)(m0 + r) * top_k + lane] = (renorm && tot > 0.f) ? chosen_w / tot : chosen_w;
     }
 }
 
 // ---------------------------------------------------------------- regrouping by expert
 // One block: counts per expert, exclusive offsets, a slot for every (row, choice) pair.  Which pair of an expert
 // gets which of its slots is left to the atomics: no result depends on it.
+// A pair whose expert is not one (an empty choice of the router) gets no slot: slot_of = -1, and the slots at the
+// end that nobody took are marked with source -1.
 __global__ void __launch_bounds__(1024) moe_sort_kernel(const int32_t* __restrict__ experts, int pairs, int top_k, int E,
                                                         int32_t* __restrict__ expert_off, int32_t* __restrict__ slot_src,
                                                         int32_t* __restrict__ slot_of) {
@@ -157,6 +165,7 @@ __global__ void __launch_bounds__(1024) moe_sort_kernel(const int32_t* __restric
     }
     __syncthreads();
     for (int e = tid; e <= E; e += 1024) expert_off[e] = off[e];
+    for (int i = off[E] + tid; i < pairs; i += 1024) slot_src[i] = -1;
     for (int i = tid; i < pairs; i += 1024) {
         const int e = experts[i];
         int slot = -1;
@@ -170,19 +179,21 @@ __global__ void __launch_bounds__(1024) moe_sort_kernel(const int32_t* __restric
 
 // Rows into expert order: xs[slot][:] = x[slot_src[slot]][:].  One block per slot.
 __global__ void __launch_bounds__(256) moe_gather_kernel(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ slot_src,
-                                                         int hid, __nv_bfloat16* __restrict__ xs) {
+                                                         int M, int hid, __nv_bfloat16* __restrict__ xs) {
     pdl_trigger();
     pdl_wait();
     const int slot = blockIdx.x;
     const int src = slot_src[slot];
+    const bool ok = src >= 0 && src < M;                          // a slot nobody took reads as zeros
     for (int pc = threadIdx.x; pc < hid / 8; pc += 256)
-        *reinterpret_cast<uint4*>(xs + (size_t)slot * hid + pc * 8) = *reinterpret_cast<const uint4*>(x + (size_t)src * hid + pc * 8);
+        *reinterpret_cast<uint4*>(xs + (size_t)slot * hid + pc * 8) =
+            ok ? *reinterpret_cast<const uint4*>(x + (size_t)src * hid + pc * 8) : make_uint4(0, 0, 0, 0);
 }
 
 // y[m][:] = residual[m][:] + sum_j weights[m][j] * ys[slot_of[m][j]][:].  One block per row.
 __global__ void __launch_bounds__(256) moe_combine_kernel(const __nv_bfloat16* __restrict__ ys, const int32_t* __restrict__ slot_of,
                                                           const float* __restrict__ weights, const __nv_bfloat16* __restrict__ residual,
-                                                          int hid, int top_k, __nv_bfloat16* __restrict__ y) {
+                                                          int hid, int top_k, int pairs, __nv_bfloat16* __restrict__ y) {
     __shared__ int s_slot[MAX_TOPK];
     __shared__ float s_w[MAX_TOPK];
     pdl_trigger();
@@ -208,7 +219,7 @@ __global__ void __launch_bounds__(256) moe_combine_kernel(const __nv_bfloat16* _
             for (int j = 0; j < 8; ++j) acc[j] = 0.f;
         }
         for (int t = 0; t < top_k; ++t) {
-            if (s_slot[t] < 0) continue;
+            if (s_slot[t] < 0 || s_slot[t] >= pairs) continue;
             const uint4 v = *reinterpret_cast<const uint4*>(ys + (size_t)s_slot[t] * hid + pc * 8);
             const uint32_t vw[4] = {v.x, v.y, v.z, v.w};
             const float w = s_w[t];
@@ -248,6 +259,7 @@ struct GroupArgs {
     int w_rows_per_expert;         // rows of w per expert (2 I for gate/up, hid for down)
     int up_offset;                 // SWIGLU: distance from a gate row to its up row (I)
     int n_out;                     // output columns (I for SWIGLU, hid for plain)
+    int n_slots;                   // rows of xs / out
     int x_box_rows;                // rows of xs one TMA box brings
     int a_bytes, stage_bytes, stages;
     __nv_bfloat16* out;            // [slots][n_out]
@@ -284,8 +296,8 @@ moe_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_c
     pdl_wait();                                    // the offsets and the gathered rows come from the kernels before
     const int e = blockIdx.z;
     const int m_lo = a.expert_off[e] + (int)blockIdx.x * 128;
-    const int rows = min(128, a.expert_off[e + 1] - m_lo);
-    if (rows <= 0) return;                         // block-uniform: this expert has no (more) rows
+    const int rows = min(128, min(a.expert_off[e + 1], a.n_slots) - m_lo);
+    if (rows <= 0 || m_lo < 0) return;             // block-uniform: this expert has no (more) rows
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 256);
     tcgen05_fence_before();
     __syncthreads();
@@ -449,6 +461,7 @@ int launch_grouped(const void* xs, size_t slots, const void* w, int E, int K, in
     a.w_rows_per_expert = w_rows_per_expert;
     a.up_offset = up_offset;
     a.n_out = n_out;
+    a.n_slots = (int)slots;
     a.x_box_rows = M >= 128 ? 128 : (M + 7) / 8 * 8;        // an expert never meets more rows than there are
     a.a_bytes = a.x_box_rows * 128;
     a.stage_bytes = a.a_bytes + G_W_BYTES;
@@ -525,12 +538,13 @@ extern "C" int deer_moe_mlp(const void* x, const void* w_router, const void* w_g
     DEER_CUDA(launch_pdl(moe_sort_kernel, dim3(1), dim3(1024), 0, st, (const int32_t*)w.experts, pairs, top_k, E, w.expert_off, w.slot_src,
                          w.slot_of));
     DEER_CUDA(launch_pdl(moe_gather_kernel, dim3(pairs), dim3(256), 0, st, static_cast<const __nv_bfloat16*>(x), (const int32_t*)w.slot_src,
-                         hid, w.xs));
+                         M, hid, w.xs));
     rc = launch_grouped<true>(w.xs, (size_t)pairs, w_gate_up, E, hid, 2 * I, I, I, M, w.expert_off, w.act, nullptr, st);
     if (rc != DEER_OK) return rc;
     rc = launch_grouped<false>(w.act, (size_t)pairs, w_down, E, I, hid, 0, hid, M, w.expert_off, w.ys, nullptr, st);
     if (rc != DEER_OK) return rc;
     DEER_CUDA(launch_pdl(moe_combine_kernel, dim3(M), dim3(256), 0, st, (const __nv_bfloat16*)w.ys, (const int32_t*)w.slot_of,
-                         (const float*)w.weights, static_cast<const __nv_bfloat16*>(residual), hid, top_k, static_cast<__nv_bfloat16*>(y)));
+                         (const float*)w.weights, static_cast<const __nv_bfloat16*>(residual), hid, top_k, pairs,
+                         static_cast<__nv_bfloat16*>(y)));
     return DEER_OK;
 }

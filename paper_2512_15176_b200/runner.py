@@ -254,15 +254,24 @@ class VerifierLayer:
     draft block, on the library's calls: RMSNorm -> Q/K/V projections -> per-head
     RMSNorm of q, k + rotary embedding -> block attention against the paged cache
     (the block's K/V rows are appended) -> output projection + residual -> RMSNorm
-    -> gate/up projection -> SiLU(gate) * up -> down projection + residual.
-    Weights are [out][in] bf16 tensors on the device ("wqkv" = the query, key and
-    value projections stacked in that order); every intermediate stays there
-    (attributes, so that a test can look at each stage)."""
+    -> MLP + residual.  The MLP is the dense SiLU-gated one (gate/up projection,
+    SiLU(gate) * up, down projection) or, with ``moe=(experts, top_k)``, the routed
+    mixture of experts.
+    Weights are [out][in] bf16 tensors on the device: "wqkv" = the query, key and
+    value projections stacked in that order, "wo", "ln1", "ln2", optional "q_norm" /
+    "k_norm"; dense: "wgu" (gate rows then up rows), "wd"; routed: "w_router" [E][hid],
+    "w_gate_up" [E][2 I][hid], "w_down" [E][hid][I].
+    ``fused=False`` issues every step as a call of its own (15 kernels; every
+    intermediate is an attribute, so that a test can look at each stage);
+    ``fused=True`` uses the calls that take a projection together with the row-wise
+    step behind it (9 kernels; the dense gate/up weights are re-laid once as
+    (gate, up) row pairs)."""
 
     def __init__(self, cfg: StepConfig, kv: L.KVCache, weights: dict, max_seq_len: int, inter: int, eps=1e-6,
-                 theta=1.0e6, device="cuda"):
+                 theta=1.0e6, device="cuda", fused=False, moe=None, reserve=True):
         self.cfg, self.kv, self.w, self.max_seq_len = cfg, kv, weights, int(max_seq_len)
         self.inter, self.eps, self.theta = int(inter), float(eps), float(theta)
+        self.fused, self.moe, self.reserve = bool(fused), moe, bool(reserve)
         B, k, Hq, Hkv, D, M, hid = cfg.B, cfg.k, cfg.Hq, cfg.Hkv, cfg.D, cfg.M, cfg.hid
         bf = torch.bfloat16
         e = lambda *shape: torch.empty(*shape, dtype=bf, device=device)
@@ -270,24 +279,81 @@ class VerifierLayer:
         self.xn, self.q, self.k_blk, self.v_blk = e(M, hid), e(B, k, Hq, D), e(B, k, Hkv, D), e(B, k, Hkv, D)
         self.qkv = e(M, (Hq + 2 * Hkv) * D)
         self.attn_out, self.x1, self.xn2 = e(B, k, Hq, D), e(M, hid), e(M, hid)
-        self.gu, self.act, self.x2 = e(M, 2 * self.inter), e(M, self.inter), e(M, hid)
+        self.act, self.x2, self.xn_next = e(M, self.inter), e(M, hid), e(M, hid)
+        self.gu = e(M, 2 * self.inter) if not (fused or moe) else None
         self.attn_ws = _ws(L.deer_block_attn_workspace_bytes(B, k, Hq, Hkv, D, self.max_seq_len), device)
-        self.lin_ws = _ws(max(L.deer_linear_workspace_bytes(M, hid, n) for n in ((Hq + 2 * Hkv) * D, 2 * self.inter, hid)) or 16, device)
+        n_qkv = (Hq + 2 * Hkv) * D
+        self.lin_ws = _ws(max(L.deer_layer_workspace_bytes(M, hid, n) for n in (n_qkv, 2 * self.inter, hid)) or 16, device)
         self.scale = 1.0 / math.sqrt(D)
+        if moe:
+            E, self.top_k = int(moe[0]), int(moe[1])
+            self.moe_ws = _ws(L.deer_moe_workspace_bytes(M, hid, E, self.inter, self.top_k), device)
+        elif fused:
+            wgu = weights["wgu"]
+            self.wgu_pairs = torch.stack([wgu[:self.inter], wgu[self.inter:]], dim=1).reshape(2 * self.inter, hid).contiguous()
 
-    def forward(self, x: torch.Tensor) -> torch.Tensor:
+    def forward(self, x: torch.Tensor, xn: Optional[torch.Tensor] = None, next_ln: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """x [M, hid]: the layer's input.  xn: RMSNorm(x) * ln1 if the caller already has it (the previous layer's
+        fused tail).  next_ln: the next layer's first RMSNorm weights; with them (fused, dense MLP) the layer also
+        leaves RMSNorm(output) in ``xn_next``."""
         c, w = self.cfg, self.w
         M = c.M
-        L.deer_rmsnorm(x, w["ln1"], self.xn, self.eps)
-        L.deer_linear(self.xn, w["wqkv"], self.qkv, workspace=self.lin_ws)
-        L.deer_qkv_split_norm_rope(self.kv, self.seq_ids, self.qkv, self.q, self.k_blk, self.v_blk, w.get("q_norm"),
-                                   w.get("k_norm"), self.eps, self.theta)
-        L.deer_kv_reserve(self.kv, self.seq_ids, c.k)
+        if xn is None:
+            L.deer_rmsnorm(x, w["ln1"], self.xn, self.eps)
+            xn = self.xn
+        if self.fused:
+            L.deer_linear_qkv_rope(self.kv, self.seq_ids, xn, w["wqkv"], self.q, self.k_blk, self.v_blk, w.get("q_norm"),
+                                   w.get("k_norm"), self.eps, self.theta, self.lin_ws)
+        else:
+            L.deer_linear(xn, w["wqkv"], self.qkv, workspace=self.lin_ws)
+            L.deer_qkv_split_norm_rope(self.kv, self.seq_ids, self.qkv, self.q, self.k_blk, self.v_blk, w.get("q_norm"),
+                                       w.get("k_norm"), self.eps, self.theta)
+        if self.reserve:
+            L.deer_kv_reserve(self.kv, self.seq_ids, c.k)
         L.deer_block_attn(self.kv, self.seq_ids, self.q, self.k_blk, self.v_blk, self.attn_out, L.DEER_MASK_CAUSAL, True,
                           self.scale, self.max_seq_len, self.attn_ws)
-        L.deer_linear(self.attn_out.view(M, -1), w["wo"], self.x1, residual=x, workspace=self.lin_ws)
-        L.deer_rmsnorm(self.x1, w["ln2"], self.xn2, self.eps)
-        L.deer_linear(self.xn2, w["wgu"], self.gu, workspace=self.lin_ws)
-        L.deer_swiglu(self.gu, self.act)
-        L.deer_linear(self.act, w["wd"], self.x2, residual=self.x1, workspace=self.lin_ws)
+        if self.fused:
+            L.deer_linear_residual_norm(self.attn_out.view(M, -1), w["wo"], self.x1, residual=x, gamma=w["ln2"], y_norm=self.xn2,
+                                        eps=self.eps, workspace=self.lin_ws)
+        else:
+            L.deer_linear(self.attn_out.view(M, -1), w["wo"], self.x1, residual=x, workspace=self.lin_ws)
+            L.deer_rmsnorm(self.x1, w["ln2"], self.xn2, self.eps)
+        if self.moe:
+            L.deer_moe_mlp(self.xn2, w["w_router"], w["w_gate_up"], w["w_down"], self.x2, self.top_k, self.moe_ws, residual=self.x1)
+            if next_ln is not None:
+                L.deer_rmsnorm(self.x2, next_ln, self.xn_next, self.eps)
+        elif self.fused:
+            L.deer_linear_swiglu(self.xn2, self.wgu_pairs, self.act)
+            L.deer_linear_residual_norm(self.act, w["wd"], self.x2, residual=self.x1, gamma=next_ln,
+                                        y_norm=self.xn_next if next_ln is not None else None, eps=self.eps, workspace=self.lin_ws)
+        else:
+            L.deer_linear(self.xn2, w["wgu"], self.gu, workspace=self.lin_ws)
+            L.deer_swiglu(self.gu, self.act)
+            L.deer_linear(self.act, w["wd"], self.x2, residual=self.x1, workspace=self.lin_ws)
+            if next_ln is not None:
+                L.deer_rmsnorm(self.x2, next_ln, self.xn_next, self.eps)
         return self.x2
+
+
+class VerifierStack:
+    """``layers`` decoder layers in a row over one paged cache layout: every layer has key / value pools of its own,
+    all of them indexed by the same page table, lengths and free stack (``kvs[l]`` = a ``binding.KVCache`` built
+    on layer l's pools and the shared integer state).  One ``deer_kv_reserve`` per step serves all layers; the
+    caller commits once after the acceptance (through any of the handles)."""
+
+    def __init__(self, cfg: StepConfig, kvs, weights, max_seq_len: int, inter: int, eps=1e-6, theta=1.0e6, device="cuda",
+                 fused=True, moe=None):
+        assert len(kvs) == len(weights)
+        self.cfg, self.kvs, self.eps = cfg, kvs, eps
+        self.layers = [VerifierLayer(cfg, kv, w, max_seq_len, inter, eps, theta, device, fused=fused, moe=moe, reserve=False)
+                       for kv, w in zip(kvs, weights)]
+        self.seq_ids = self.layers[0].seq_ids
+
+    def forward(self, x: torch.Tensor) -> torch.Tensor:
+        L.deer_kv_reserve(self.kvs[0], self.seq_ids, self.cfg.k)
+        xn = None
+        for i, layer in enumerate(self.layers):
+            nxt = self.layers[i + 1].w["ln1"] if i + 1 < len(self.layers) else None
+            x = layer.forward(x, xn=xn, next_ln=nxt)
+            xn = layer.xn_next if nxt is not None else None
+        return x

@@ -30,6 +30,9 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("what", choices=["lmhead", "attn", "qstats", "layer"])
     ap.add_argument("--inter", type=int, default=12288)
+    ap.add_argument("--separate", action="store_true", help="layer: every step as a call of its own instead of the fused calls")
+    ap.add_argument("--experts", type=int, default=0, help="layer: routed MLP with this many experts (0 = dense)")
+    ap.add_argument("--top-k", type=int, default=8)
     ap.add_argument("--M", type=int, default=32)
     ap.add_argument("--hid", type=int, default=4096)
     ap.add_argument("--V", type=int, default=32768)
@@ -90,11 +93,18 @@ def main():
         mk = lambda n, shape, sig: W.normal(34, n, shape, sig, device=dev)
         w = {"ln1": mk("ln1", (hid,), 1.0), "ln2": mk("ln2", (hid,), 1.0), "q_norm": mk("qn", (a.D,), 1.0),
              "k_norm": mk("kn", (a.D,), 1.0), "wqkv": mk("wqkv", (QD + 2 * KD, hid), hid ** -0.5),
-             "wo": mk("wo", (hid, QD), QD ** -0.5),
-             "wgu": mk("wgu", (2 * a.inter, hid), hid ** -0.5), "wd": mk("wd", (hid, a.inter), a.inter ** -0.5)}
+             "wo": mk("wo", (hid, QD), QD ** -0.5)}
+        if a.experts:
+            w.update({"w_router": mk("wr", (a.experts, hid), hid ** -0.5 * 3.0),
+                      "w_gate_up": mk("wgue", (a.experts, 2 * a.inter, hid), hid ** -0.5),
+                      "w_down": mk("wde", (a.experts, hid, a.inter), a.inter ** -0.5)})
+        else:
+            w.update({"wgu": mk("wgu", (2 * a.inter, hid), hid ** -0.5), "wd": mk("wd", (hid, a.inter), a.inter ** -0.5)})
         x = mk("x", (cfg.M, hid), 1.0)
-        layer = VerifierLayer(cfg, kv, w, a.ctx + a.k, a.inter)
+        layer = VerifierLayer(cfg, kv, w, a.ctx + a.k, a.inter, fused=not a.separate,
+                              moe=(a.experts, a.top_k) if a.experts else None)
         side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())       # the weights and pools were drawn on the current stream
         with torch.cuda.stream(side):
             for _ in range(3):
                 layer.forward(x)
@@ -104,8 +114,16 @@ def main():
                 layer.forward(x)
         torch.cuda.synchronize()
         call = g.replay
-        nbytes = sum(t.numel() * 2 for n, t in w.items()) + W.algorithmic_bytes(cfg, lengths)["attn"]
-        flops = 2.0 * cfg.M * sum(t.numel() for n, t in w.items() if n.startswith("w"))
+        dense = sum(t.numel() * 2 for n, t in w.items() if n not in ("w_gate_up", "w_down"))
+        if a.experts:
+            e_ids = torch.empty(cfg.M, a.top_k, dtype=torch.int32, device=dev)
+            e_w = torch.empty(cfg.M, a.top_k, dtype=torch.float32, device=dev)
+            L.deer_moe_route(layer.xn2, w["w_router"], a.top_k, e_ids, e_w)
+            torch.cuda.synchronize()
+            dense += int(torch.unique(e_ids).numel()) * 3 * a.inter * hid * 2      # the experts the rows really chose
+        nbytes = dense + W.algorithmic_bytes(cfg, lengths)["attn"]
+        flops = 2.0 * cfg.M * (dense / 2 if not a.experts else sum(t.numel() for n, t in w.items() if n in ("wqkv", "wo"))
+                               + a.top_k * 3 * a.inter * hid)
     else:
         M = a.B * a.k
         ql = W.normal(33, "ql", (a.B, a.k, a.V), 1.0, dtype=torch.float32, device=dev)

@@ -214,3 +214,31 @@ def nucleus_margin_ok(z32, T, top_k, top_p, margin=1e-4):
         if top_p - before < margin or (incl - top_p < margin and lo[-1] < len(vals) - 1):
             return False
     return True
+
+
+def sampled_oracle_kv(kv, seqs, extra_tokens, page_size=16):
+    """An oracle cache holding only the sequences ``seqs`` of the device cache ``kv`` (their pages copied from the
+    device pools into a compact pool, page ids renumbered, room for ``extra_tokens`` more tokens each): what the
+    oracle needs to follow a few sequences of a batch whose pools are too large to draw or hold on the host.
+    Sequence j of the result is sequence seqs[j] of the device cache."""
+    pt = kv.page_table.cpu().numpy()
+    sl = kv.seq_len.cpu().numpy()
+    npg = kv.n_pages.cpu().numpy()
+    Hkv, D = kv.k_pool.shape[1], kv.k_pool.shape[3]
+    per_seq = [int(npg[s]) + -(-extra_tokens // page_size) + 1 for s in seqs]
+    total = sum(per_seq)
+    max_pages = max(per_seq)
+    k_pool = np.zeros((total, Hkv, page_size, D), dtype=np.float32)
+    v_pool = np.zeros((total, Hkv, page_size, D), dtype=np.float32)
+    table = np.full((len(seqs), max_pages), -1, dtype=np.int32)
+    nxt = 0
+    for j, s in enumerate(seqs):
+        ids = torch.from_numpy(pt[s, :npg[s]].astype(np.int64)).to(kv.k_pool.device)
+        k_pool[nxt:nxt + npg[s]] = kv.k_pool[ids].float().cpu().numpy()
+        v_pool[nxt:nxt + npg[s]] = kv.v_pool[ids].float().cpu().numpy()
+        table[j, :npg[s]] = np.arange(nxt, nxt + npg[s])
+        nxt += int(npg[s])
+    free = np.arange(total - 1, nxt - 1, -1, dtype=np.int32)          # the unused pages, popped in ascending order
+    stack = np.zeros(total, dtype=np.int32)
+    stack[:free.size] = free
+    return O.PagedKV(k_pool, v_pool, table, sl[list(seqs)], npg[list(seqs)], stack, free.size)

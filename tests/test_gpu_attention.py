@@ -113,3 +113,36 @@ def test_sequence_longer_than_bound_is_reported():
     L.deer_block_attn(kv, seq_ids, q.cuda(), kb.cuda(), vb.cuda(), out, 0, 0, 0.125, 50, ws)
     assert L.deer_kv_status(kv) == L.DEER_ERR_INVALID_ARG
     assert L.deer_kv_status(kv) == 0          # reading clears it
+
+
+@pytest.mark.parametrize("gain", [8.0, 40.0])
+def test_dominant_keys_far_above_the_first_tile(gain):
+    """Keys planted late in the context whose scores lie hundreds of octaves above everything seen before them: the
+    exponentials of a segment are taken against its first tile's maximum, so such a tile must raise the reference
+    point (at gain 8 the exponentials are huge but finite, at gain 40 they overflow) and the output must still be
+    the softmax by definition -- essentially the planted key's value row."""
+    from paper_2512_15176_b200 import binding as L
+    cfg = W.StepConfig("dominant", 2, 8, 2, 128, 8, 64, 64, (0, 0), seed=83)
+    lens = [900, 3000]
+    st = Hn.draw_state(cfg, lens, True)
+    q, kb, vb = Hn.draw_block(cfg, 0, True)
+    G = cfg.Hq // cfg.Hkv
+    planted = [(0, 700, 3, 5), (1, 150, 0, 0), (1, 2999, 7, 6), (1, 1600, 2, 3)]     # (sequence, token, block row, query head)
+    for b, t, i, h in planted:
+        pg = int(st.layout.page_table[b, t // 16])
+        st.k_pool[pg, h // G, t % 16] = (q[b, i, h].float() * gain).to(torch.bfloat16)
+    okv = Hn.oracle_kv(st)
+    want = Hn.oracle_attention(cfg, okv, q, kb, vb)
+    kv = Hn.gpu_kv(st)
+    seq_ids = torch.arange(cfg.B, dtype=torch.int32, device="cuda")
+    msl = max(lens)
+    ws = torch.empty(L.deer_block_attn_workspace_bytes(cfg.B, cfg.k, cfg.Hq, cfg.Hkv, cfg.D, msl), dtype=torch.uint8, device="cuda")
+    out = torch.full((cfg.B, cfg.k, cfg.Hq, cfg.D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    L.deer_block_attn(kv, seq_ids, q.cuda(), kb.cuda(), vb.cuda(), out, cfg.mask, 0, 1.0 / math.sqrt(cfg.D), msl, ws)
+    torch.cuda.synchronize()
+    assert L.deer_kv_status(kv) == 0
+    Hn.check_attention(out.cpu(), want, f"dominant keys, gain {gain}")
+    for b, t, i, h in planted:
+        pg = int(st.layout.page_table[b, t // 16])
+        v_row = st.v_pool[pg, h // G, t % 16].float()
+        assert (out[b, i, h].cpu().float() - v_row).abs().max() < 2e-2          # that row's output is the planted key's value

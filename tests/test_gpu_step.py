@@ -285,3 +285,74 @@ def test_host_buffer_step_notices_a_swapped_device_buffer():
     np.testing.assert_array_equal(a, want_a)
     np.testing.assert_array_equal(out, want_out)
     assert torch.equal(other_h.cpu(), h1)
+
+
+@pytest.mark.parametrize("B,ctx,k,V,steps", [
+    (4, 32768, 32, 8192, 64),          # the longest context, every sequence followed by the oracle
+    (64, 16384, 16, 8192, 64),         # the largest batch with a long context: four sampled sequences
+    (64, 32768, 8, 151936, 1),         # the largest batch and context at the full vocabulary, one step
+])
+def test_c5_sweep_corners(B, ctx, k, V, steps):
+    """Sweep corners at their real sizes.  The pools are drawn on the device (gigabytes); the oracle follows a seeded
+    sample of four sequences (their pages copied out) for the attention values and the cache contents, and every
+    sequence for the integer cache state, over all consecutive steps, each with freshly planted drafts and a commit.
+    Attention is compared at the first, a middle and the last step."""
+    from paper_2512_15176_b200 import binding as L
+    from paper_2512_15176_b200.runner import VerifyStep
+    cfg = W.sweep_config(B, ctx, k, W.MASK_CAUSAL, steps=steps).with_(V=V)
+    lengths = W.seq_lengths(cfg)
+    lay = W.kv_layout(cfg, lengths)
+    kp, vp = W.kv_pools(cfg, lay.num_pages, device="cuda", sigma=1.0)
+    kv = L.KVCache.from_layout(lay, kp, vp, "cuda")
+    del kp, vp
+    sample = sorted(W.rng(cfg.seed, "sample").choice(B, size=min(4, B), replace=False).tolist())
+    okv_s = Hn.sampled_oracle_kv(kv, sample, steps * k)
+    okv_all = O.PagedKV(np.zeros((1, 1, 16, 1), np.float32), np.zeros((1, 1, 16, 1), np.float32), lay.page_table, lay.seq_len,
+                        lay.n_pages, lay.free_stack, lay.free_top)
+    w = W.lm_head(cfg)
+    w64 = Hn.f64(w)
+    msl = int(lengths.max()) + steps * k
+    vs = VerifyStep(cfg, kv, w.cuda(), msl, store_logits=False)
+    ids_all, ids_s = np.arange(B), np.arange(len(sample))
+    check_at = {0, steps // 2, steps - 1}
+    # the hidden states (and so the targets) stay; every step plants a new prefix and draws new block rows
+    h, z, _ = Hn.draw_hidden_with_margin(cfg, w64, 0)
+    target = O.select_argmax(z).reshape(B, k)
+    vs.load(h=h)
+    for step in range(steps):
+        q, kb, vb = Hn.draw_block(cfg, step, True)
+        Lp = W.planted_prefix_lengths(cfg, step)
+        drafts = W.plant_drafts(cfg, target, Lp, step)
+        a, out, n = O.accept_greedy(drafts, target)
+        np.testing.assert_array_equal(a, Lp)
+        assert okv_all.reserve(ids_all, k) and okv_s.reserve(ids_s, k)
+        qs, kbs, vbs = (Hn.f64(t[sample]) for t in (q, kb, vb))
+        if step in check_at:
+            want = O.block_attention(qs, kbs, vbs, okv_s.k_pool, okv_s.v_pool, okv_s.page_table, okv_s.seq_len, ids_s,
+                                     cfg.mask, 1.0 / math.sqrt(cfg.D))
+        okv_s.append(ids_s, kbs.astype(np.float32), vbs.astype(np.float32))
+        okv_all.commit(ids_all, a)
+        okv_s.commit(ids_s, a[sample])
+        vs.load(q, kb, vb, None, drafts)
+        vs.run()
+        if step in check_at:
+            torch.cuda.synchronize()
+            assert L.deer_kv_status(kv) == 0
+            Hn.check_attention(vs.attn_out.cpu()[sample], want, f"{cfg.name} step {step}")
+            if step == 0:
+                Hn.check_ids(vs.target_ids.cpu().numpy(), target, z, cfg.name)
+            np.testing.assert_array_equal(vs.accept_len.cpu().numpy(), a)
+            np.testing.assert_array_equal(vs.out_ids.cpu().numpy(), out)
+            Hn.kv_state_equal(kv, okv_all, f"{cfg.name} step {step}")
+    torch.cuda.synchronize()
+    assert L.deer_kv_status(kv) == 0
+    Hn.kv_state_equal(kv, okv_all, cfg.name)
+    # contents of the sampled sequences: each side gathers through its own page table
+    pt, sl = kv.page_table.cpu().numpy(), kv.seq_len.cpu().numpy()
+    for j, s in enumerate(sample):
+        npg = -(-int(sl[s]) // 16)
+        pages = torch.from_numpy(pt[s, :npg].astype(np.int64)).cuda()
+        for pool, opool in ((kv.k_pool, okv_s.k_pool), (kv.v_pool, okv_s.v_pool)):
+            got = pool[pages].float().cpu().numpy().transpose(0, 2, 1, 3).reshape(npg * 16, cfg.Hkv, cfg.D)[:int(sl[s])]
+            want_c = O.gather_prefix(opool, okv_s.page_table[j], int(okv_s.seq_len[j]), 16)
+            np.testing.assert_array_equal(got, want_c, err_msg=f"{cfg.name} contents of sequence {s}")
