@@ -423,11 +423,11 @@ int deer_linear_swiglu(const void* x, const void* w_pairs, void* y, int M, int K
  * weights once; gate, up (each rounded to bf16, as a dense layer would store them), the activations and the expert
  * outputs are bf16, sums fp32.
  * deer_moe_route is the first stage alone: experts i32 [M][top_k] in order of falling probability, weights f32
- * [M][top_k] (renormalise = 0: the softmax probabilities themselves).
- *   workspace  >= deer_moe_workspace_bytes(...) bytes, 16-byte aligned, contents arbitrary. */
+ * [M][top_k] (renormalise = 0: the softmax probabilities themselves); its workspace holds the M x E fp32 logits.
+ *   workspace  >= deer_moe_workspace_bytes(...) bytes (deer_moe_route: M * E * 4), 16-byte aligned, contents arbitrary. */
 size_t deer_moe_workspace_bytes(int M, int hid, int E, int I, int top_k);
 int deer_moe_route(const void* x, const void* w_router, int M, int hid, int E, int top_k, int renormalise,
-                   int32_t* experts, float* weights, void* stream);
+                   int32_t* experts, float* weights, void* workspace, size_t workspace_bytes, void* stream);
 int deer_moe_mlp(const void* x, const void* w_router, const void* w_gate_up, const void* w_down, const void* residual,
                  void* y, int M, int hid, int E, int I, int top_k, void* workspace, size_t workspace_bytes, void* stream);
 

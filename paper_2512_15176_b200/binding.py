@@ -120,7 +120,8 @@ def lib() -> ctypes.CDLL:
     L.deer_linear_swiglu.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p]
     L.deer_moe_workspace_bytes.restype = c_size_t
     L.deer_moe_workspace_bytes.argtypes = [c_int] * 5
-    L.deer_moe_route.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p]
+    L.deer_moe_route.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_size_t,
+                                 c_void_p]
     L.deer_moe_mlp.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_int,
                                c_void_p, c_size_t, c_void_p]
     L.deer_verify_step_host.argtypes = [c_void_p, POINTER(deer_step_dev), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
@@ -342,10 +343,14 @@ def deer_moe_workspace_bytes(M, hid, E, I, top_k) -> int:
     return lib().deer_moe_workspace_bytes(M, hid, E, I, top_k)
 
 
-def deer_moe_route(x, w_router, top_k, experts, weights, renormalise=True, stream=None):
+def deer_moe_route(x, w_router, top_k, experts, weights, renormalise=True, workspace=None, stream=None):
     M, hid = x.shape
-    _check(lib().deer_moe_route(_ptr(x), _ptr(w_router), M, hid, w_router.shape[0], int(top_k), 1 if renormalise else 0,
-                                _ptr(experts), _ptr(weights), _stream(stream)))
+    E = w_router.shape[0]
+    if workspace is None:                      # plumbing: room for the M x E fp32 logits
+        workspace = torch.empty(max(16, M * E * 4), dtype=torch.uint8, device=x.device)
+    _check(lib().deer_moe_route(_ptr(x), _ptr(w_router), M, hid, E, int(top_k), 1 if renormalise else 0,
+                                _ptr(experts), _ptr(weights), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                _stream(stream)))
 
 
 def deer_moe_mlp(x, w_router, w_gate_up, w_down, y, top_k, workspace, residual=None, stream=None):

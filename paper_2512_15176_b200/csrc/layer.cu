@@ -90,14 +90,38 @@ __global__ void __launch_bounds__(128) qk_norm_rope_kernel(deer_kv_desc kv, cons
     // lane l holds the pairs d = l, l + 32, ... (D <= 128: at most two pairs)
     float a[2], c[2];
     float ss = 0.f;
+    if (part) {
+        // all of this lane's values at once: up to four columns per partial product, four partial products in flight
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        const bool two = lane + 32 < half;
+#pragma unroll 4
+        for (int s = 0; s < ksplit; ++s) {
+            const float* ps = part + (long long)s * part_stride + in_off;
+            if (lane < half) {
+                acc[0] += ps[lane];
+                acc[1] += ps[lane + half];
+            }
+            if (two) {
+                acc[2] += ps[lane + 32];
+                acc[3] += ps[lane + 32 + half];
+            }
+        }
 #pragma unroll
-    for (int t = 0; t < 2; ++t) {
-        const int d = lane + 32 * t;
-        a[t] = c[t] = 0.f;
-        if (d < half) {
-            a[t] = packed ? packed_at(in_off + d) : __bfloat162float(v[d]);
-            c[t] = packed ? packed_at(in_off + d + half) : __bfloat162float(v[d + half]);
-            ss += a[t] * a[t] + c[t] * c[t];
+        for (int t = 0; t < 2; ++t) {
+            a[t] = __bfloat162float(__float2bfloat16(acc[2 * t]));          // what the projection would have stored
+            c[t] = __bfloat162float(__float2bfloat16(acc[2 * t + 1]));
+            if (lane + 32 * t < half) ss += a[t] * a[t] + c[t] * c[t];
+        }
+    } else {
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+            const int d = lane + 32 * t;
+            a[t] = c[t] = 0.f;
+            if (d < half) {
+                a[t] = packed ? packed_at(in_off + d) : __bfloat162float(v[d]);
+                c[t] = packed ? packed_at(in_off + d + half) : __bfloat162float(v[d + half]);
+                ss += a[t] * a[t] + c[t] * c[t];
+            }
         }
     }
     float inv = 1.f;
@@ -185,47 +209,103 @@ namespace {
 
 // One block per row: y = sum of the partial products (or the projection's bf16 output) + residual, rounded to bf16;
 // then, if gamma is given, y_norm = RMSNorm(y) * gamma over the rounded values (what a separate pass would read).
-__global__ void __launch_bounds__(256) residual_norm_tail_kernel(const float* __restrict__ part, int ksplit, const __nv_bfloat16* __restrict__ y_in,
-                                                                 const __nv_bfloat16* __restrict__ residual,
-                                                                 const __nv_bfloat16* __restrict__ gamma, __nv_bfloat16* __restrict__ y,
-                                                                 __nv_bfloat16* __restrict__ y_norm, int M, int N, float eps) {
-    __shared__ float red[8];
+// A thread takes four neighbouring columns at a time and has the loads of four partial products in flight.
+__global__ void __launch_bounds__(1024) residual_norm_tail_kernel(const float* __restrict__ part, int ksplit, const __nv_bfloat16* __restrict__ y_in,
+                                                                  const __nv_bfloat16* __restrict__ residual,
+                                                                  const __nv_bfloat16* __restrict__ gamma, __nv_bfloat16* __restrict__ y,
+                                                                  __nv_bfloat16* __restrict__ y_norm, int M, int N, float eps) {
+    __shared__ float red[32];
     pdl_trigger();
     pdl_wait();
+    const int T = blockDim.x;
     const size_t row = blockIdx.x;
     const size_t stride = (size_t)M * N;
+    const bool vec = (N & 3) == 0;
     float ss = 0.f;
-    for (int c = threadIdx.x; c < N; c += 256) {
-        const size_t o = row * N + c;
-        float v;
-        if (part) {
-            v = 0.f;
-            for (int s = 0; s < ksplit; ++s) v += part[(size_t)s * stride + o];
-            if (residual) v += __bfloat162float(residual[o]);
-        } else {
-            v = __bfloat162float(y_in[o]);                 // the projection added the residual itself
+    if (vec) {
+        for (int c = threadIdx.x * 4; c < N; c += T * 4) {
+            const size_t o = row * N + c;
+            float v[4];
+            if (part) {
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+                for (int s = 0; s < ksplit; ++s) {
+                    const float4 t = __ldg(reinterpret_cast<const float4*>(part + (size_t)s * stride + o));
+                    acc.x += t.x;
+                    acc.y += t.y;
+                    acc.z += t.z;
+                    acc.w += t.w;
+                }
+                v[0] = acc.x; v[1] = acc.y; v[2] = acc.z; v[3] = acc.w;
+                if (residual) {
+                    const uint2 r = *reinterpret_cast<const uint2*>(residual + o);
+                    v[0] += __uint_as_float(r.x << 16);
+                    v[1] += __uint_as_float(r.x & 0xffff0000u);
+                    v[2] += __uint_as_float(r.y << 16);
+                    v[3] += __uint_as_float(r.y & 0xffff0000u);
+                }
+                uint2 ov;
+                ov.x = pack_bf16(v[0], v[1]);
+                ov.y = pack_bf16(v[2], v[3]);
+                *reinterpret_cast<uint2*>(y + o) = ov;
+                v[0] = __uint_as_float(ov.x << 16); v[1] = __uint_as_float(ov.x & 0xffff0000u);
+                v[2] = __uint_as_float(ov.y << 16); v[3] = __uint_as_float(ov.y & 0xffff0000u);
+            } else {
+                const uint2 r = *reinterpret_cast<const uint2*>(y_in + o);      // the projection added the residual itself
+                v[0] = __uint_as_float(r.x << 16); v[1] = __uint_as_float(r.x & 0xffff0000u);
+                v[2] = __uint_as_float(r.y << 16); v[3] = __uint_as_float(r.y & 0xffff0000u);
+            }
+            ss += (v[0] * v[0] + v[1] * v[1]) + (v[2] * v[2] + v[3] * v[3]);
         }
-        const __nv_bfloat16 vb = __float2bfloat16(v);
-        if (part) y[o] = vb;
-        const float vr = __bfloat162float(vb);
-        ss += vr * vr;
+    } else {
+        for (int c = threadIdx.x; c < N; c += T) {
+            const size_t o = row * N + c;
+            float v;
+            if (part) {
+                v = 0.f;
+                for (int s = 0; s < ksplit; ++s) v += part[(size_t)s * stride + o];
+                if (residual) v += __bfloat162float(residual[o]);
+                y[o] = __float2bfloat16(v);
+                v = __bfloat162float(y[o]);
+            } else {
+                v = __bfloat162float(y_in[o]);
+            }
+            ss += v * v;
+        }
     }
     if (!gamma) return;
     ss = warp_sum(ss);
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
     __syncthreads();
     float tot = 0.f;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) tot += red[w];
+    for (int w = 0; w < (T >> 5); ++w) tot += red[w];
     const float inv = rsqrtf(tot / (float)N + eps);
-    for (int c = threadIdx.x; c < N; c += 256) {
-        const size_t o = row * N + c;
-        // this thread wrote y[o] itself a moment ago
-        y_norm[o] = __float2bfloat16(__bfloat162float(part ? y[o] : y_in[o]) * inv * __bfloat162float(gamma[c]));
+    const __nv_bfloat16* src = part ? y : y_in;            // this thread wrote its part of y itself a moment ago
+    if (vec) {
+        for (int c = threadIdx.x * 4; c < N; c += T * 4) {
+            const size_t o = row * N + c;
+            const uint2 r = *reinterpret_cast<const uint2*>(src + o);
+            const uint2 g = *reinterpret_cast<const uint2*>(gamma + c);
+            uint2 ov;
+            ov.x = pack_bf16(__uint_as_float(r.x << 16) * inv * __uint_as_float(g.x << 16),
+                             __uint_as_float(r.x & 0xffff0000u) * inv * __uint_as_float(g.x & 0xffff0000u));
+            ov.y = pack_bf16(__uint_as_float(r.y << 16) * inv * __uint_as_float(g.y << 16),
+                             __uint_as_float(r.y & 0xffff0000u) * inv * __uint_as_float(g.y & 0xffff0000u));
+            *reinterpret_cast<uint2*>(y_norm + o) = ov;
+        }
+    } else {
+        for (int c = threadIdx.x; c < N; c += T)
+            y_norm[row * N + c] = __float2bfloat16(__bfloat162float(src[row * N + c]) * inv * __bfloat162float(gamma[c]));
     }
 }
 
 }  // namespace
+
+// Threads of a tail block: one per four columns, a whole number of warps, 1024 at most.
+static int tail_threads(int N) {
+    int t = ((N + 3) / 4 + 31) / 32 * 32;
+    return t < 32 ? 32 : (t > 1024 ? 1024 : t);
+}
 
 extern "C" size_t deer_layer_workspace_bytes(int M, int K, int N) {
     const size_t a = deer_linear_workspace_bytes(M, K, N), b = (size_t)(M > 0 ? M : 0) * (N > 0 ? N : 0) * 2;
@@ -268,7 +348,7 @@ extern "C" int deer_linear_residual_norm(const void* x, const void* w, const voi
     int rc = deer_linear_for_tail(x, w, residual, y, M, K, N, workspace, workspace_bytes, &ksplit, st);
     if (rc != DEER_OK) return rc;
     if (ksplit > 1) {
-        DEER_CUDA(launch_pdl(residual_norm_tail_kernel, dim3(M), dim3(256), 0, st, (const float*)workspace, ksplit,
+        DEER_CUDA(launch_pdl(residual_norm_tail_kernel, dim3(M), dim3(tail_threads(N)), 0, st, (const float*)workspace, ksplit,
                              (const __nv_bfloat16*)nullptr, static_cast<const __nv_bfloat16*>(residual),
                              static_cast<const __nv_bfloat16*>(gamma), static_cast<__nv_bfloat16*>(y), static_cast<__nv_bfloat16*>(y_norm),
                              M, N, eps));
@@ -276,7 +356,7 @@ extern "C" int deer_linear_residual_norm(const void* x, const void* w, const voi
     }
     // the contraction was not cut: the projection has written y + residual itself, the tail only normalises
     if (!gamma) return DEER_OK;
-    DEER_CUDA(launch_pdl(residual_norm_tail_kernel, dim3(M), dim3(256), 0, st, (const float*)nullptr, 1, (const __nv_bfloat16*)y,
+    DEER_CUDA(launch_pdl(residual_norm_tail_kernel, dim3(M), dim3(tail_threads(N)), 0, st, (const float*)nullptr, 1, (const __nv_bfloat16*)y,
                          (const __nv_bfloat16*)nullptr, static_cast<const __nv_bfloat16*>(gamma), static_cast<__nv_bfloat16*>(y),
                          static_cast<__nv_bfloat16*>(y_norm), M, N, eps));
     return DEER_OK;

@@ -9,7 +9,7 @@
 // gate/up projection pairs 128 gate rows with the 128 up rows of the same channels in one accumulator, so
 // SiLU(gate) * up is taken in the epilogue and only the activations are written.
 //
-// Kernels: route (logits in fp32, softmax, top-k, renormalise) -> sort (counts, offsets, slots) -> gather ->
+// Kernels: router logits (fp32) -> choice (softmax, top-k, renormalise) -> sort (counts, offsets, slots) -> gather ->
 // grouped gate/up + SwiGLU -> grouped down -> combine.  All waits are bounded as in the other tensor-core kernels.
 
 #include "sm100.cuh"
@@ -28,19 +28,20 @@ __device__ __forceinline__ float warp_sum(float v) {
 }
 
 // ---------------------------------------------------------------- router
-// A block takes 8 rows: their hidden states sit in shared memory, warp w walks the experts w, w + 8, ... and
-// forms the 8 dot products of each at once (the router matrix crosses L2 once per 8 rows); then warp r finishes
-// row r: softmax over the experts, the top_k largest (lowest index among equals), weights renormalised to sum 1.
+// Logits: block (row group of 8, expert group of 8); the rows' hidden states sit in shared memory, warp w takes
+// expert 8 * group + w and forms its 8 dot products at once, all of its loads of the expert's row in flight
+// together.  Choice: one warp per row -- softmax over the experts, the top_k largest (lowest index among equals),
+// weights renormalised to sum 1.
 constexpr int RT_ROWS = 8;
+constexpr int RT_EXPERTS = 8;
 
-__global__ void __launch_bounds__(256) moe_route_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ wr,
-                                                        int M, int hid, int E, int top_k, int renorm,
-                                                        int32_t* __restrict__ experts, float* __restrict__ weights) {
+__global__ void __launch_bounds__(256) moe_logits_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ wr,
+                                                         int M, int hid, int E, float* __restrict__ logits) {
     extern __shared__ unsigned char smem_raw[];
     __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(smem_raw);                 // [8][hid]
-    float* logit = reinterpret_cast<float*>(smem_raw + (size_t)RT_ROWS * hid * 2);   // [8][E]
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int m0 = blockIdx.x * RT_ROWS;
+    const int e = blockIdx.y * RT_EXPERTS + warp;
     pdl_trigger();
     pdl_wait();
     const int pieces = hid / 8;
@@ -51,13 +52,22 @@ __global__ void __launch_bounds__(256) moe_route_kernel(const __nv_bfloat16* __r
         *reinterpret_cast<uint4*>(xs + (size_t)r * hid + pc * 8) = v;
     }
     __syncthreads();
-    for (int e = warp; e < E; e += 8) {
-        float acc[RT_ROWS];
+    if (e >= E) return;
+    float acc[RT_ROWS];
 #pragma unroll
-        for (int r = 0; r < RT_ROWS; ++r) acc[r] = 0.f;
-        for (int pc = lane; pc < pieces; pc += 32) {
-            const uint4 wv = __ldg(reinterpret_cast<const uint4*>(wr + (size_t)e * hid + pc * 8));
-            const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
+    for (int r = 0; r < RT_ROWS; ++r) acc[r] = 0.f;
+    for (int pc0 = lane; pc0 < pieces; pc0 += 32 * 4) {
+        uint4 wv[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int pc = pc0 + 32 * u;
+            wv[u] = pc < pieces ? __ldg(reinterpret_cast<const uint4*>(wr + (size_t)e * hid + pc * 8)) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int pc = pc0 + 32 * u;
+            if (pc >= pieces) break;
+            const uint32_t ww[4] = {wv[u].x, wv[u].y, wv[u].z, wv[u].w};
 #pragma unroll
             for (int r = 0; r < RT_ROWS; ++r) {
                 const uint4 xv = *reinterpret_cast<const uint4*>(xs + (size_t)r * hid + pc * 8);
@@ -69,15 +79,21 @@ __global__ void __launch_bounds__(256) moe_route_kernel(const __nv_bfloat16* __r
                 }
             }
         }
-#pragma unroll
-        for (int r = 0; r < RT_ROWS; ++r) {
-            const float s = warp_sum(acc[r]);
-            if (lane == 0) logit[r * E + e] = s;
-        }
     }
-    __syncthreads();
-    const int r = warp;
-    if (m0 + r >= M) return;
+#pragma unroll
+    for (int r = 0; r < RT_ROWS; ++r) {
+        const float sum = warp_sum(acc[r]);
+        if (lane == 0 && m0 + r < M) logits[(size_t)(m0 + r) * E + e] = sum;
+    }
+}
+
+__global__ void __launch_bounds__(256) moe_choose_kernel(const float* __restrict__ logits, int M, int E, int top_k, int renorm,
+                                                         int32_t* __restrict__ experts, float* __restrict__ weights) {
+    const int lane = threadIdx.x & 31;
+    const int m = blockIdx.x * 8 + (threadIdx.x >> 5);
+    pdl_trigger();
+    pdl_wait();
+    if (m >= M) return;
     // lane l holds the experts l, l + 32, ...
     constexpr int PER = MAX_E / 32;
     float v[PER];
@@ -85,7 +101,7 @@ __global__ void __launch_bounds__(256) moe_route_kernel(const __nv_bfloat16* __r
 #pragma unroll
     for (int j = 0; j < PER; ++j) {
         const int e = lane + 32 * j;
-        v[j] = e < E ? logit[r * E + e] : -INFINITY;
+        v[j] = e < E ? logits[(size_t)m * E + e] : -INFINITY;
         mx = fmaxf(mx, v[j]);
     }
 #pragma unroll
@@ -131,8 +147,8 @@ __global__ void __launch_bounds__(256) moe_route_kernel(const __nv_bfloat16* __r
         if (!none) tot += bv / sum;
     }
     if (lane < top_k) {
-        experts[(size_t)(m0 + r) * top_k + lane] = chosen_e;
-        weights[(size_t)(m0 + r) * top_k + lane] = (renorm && tot > 0.f) ? chosen_w / tot : chosen_w;
+        experts[(size_t)m * top_k + lane] = chosen_e;
+        weights[(size_t)m * top_k + lane] = (renorm && tot > 0.f) ? chosen_w / tot : chosen_w;
     }
 }
 
@@ -417,6 +433,7 @@ struct MoeWs {
     int32_t* slot_src;     // [M top_k]
     int32_t* slot_of;      // [M][top_k]
     int32_t* status;       // [1]
+    float* logits;         // [M][E]           router logits
     __nv_bfloat16* xs;     // [M top_k][hid]   rows in expert order
     __nv_bfloat16* act;    // [M top_k][I]
     __nv_bfloat16* ys;     // [M top_k][hid]
@@ -438,6 +455,7 @@ MoeWs carve(void* base, int M, int hid, int E, int I, int top_k) {
     w.slot_src = static_cast<int32_t*>(take(pairs * 4));
     w.slot_of = static_cast<int32_t*>(take(pairs * 4));
     w.status = static_cast<int32_t*>(take(4));
+    w.logits = static_cast<float*>(take((size_t)M * E * 4));
     w.xs = static_cast<__nv_bfloat16*>(take(pairs * hid * 2));
     w.act = static_cast<__nv_bfloat16*>(take(pairs * I * 2));
     w.ys = static_cast<__nv_bfloat16*>(take(pairs * hid * 2));
@@ -488,16 +506,18 @@ int check_shape(int M, int hid, int E, int I, int top_k, const char* who) {
     DEER_CHECK_ARG(E <= MAX_E && top_k <= MAX_TOPK && top_k <= E, DEER_ERR_UNSUPPORTED, "%s: at most %d experts, top_k <= min(%d, E)",
                    who, MAX_E, MAX_TOPK);
     DEER_CHECK_ARG(hid % 64 == 0 && I % 64 == 0, DEER_ERR_UNSUPPORTED, "%s: hid and I must be multiples of 64", who);
-    DEER_CHECK_ARG((size_t)RT_ROWS * hid * 2 + (size_t)RT_ROWS * E * 4 <= 200 * 1024, DEER_ERR_UNSUPPORTED, "%s: hid too large", who);
+    DEER_CHECK_ARG((size_t)RT_ROWS * hid * 2 <= 200 * 1024, DEER_ERR_UNSUPPORTED, "%s: hid too large", who);
     return DEER_OK;
 }
 
-int route(const void* x, const void* w_router, int M, int hid, int E, int top_k, int renorm, int32_t* experts, float* weights,
-          cudaStream_t st) {
-    const size_t smem = (size_t)RT_ROWS * hid * 2 + (size_t)RT_ROWS * E * 4;
-    DEER_CUDA(cudaFuncSetAttribute(moe_route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    DEER_CUDA(launch_pdl(moe_route_kernel, dim3((M + RT_ROWS - 1) / RT_ROWS), dim3(256), smem, st, static_cast<const __nv_bfloat16*>(x),
-                         static_cast<const __nv_bfloat16*>(w_router), M, hid, E, top_k, renorm, experts, weights));
+int route(const void* x, const void* w_router, int M, int hid, int E, int top_k, int renorm, float* logits, int32_t* experts,
+          float* weights, cudaStream_t st) {
+    const size_t smem = (size_t)RT_ROWS * hid * 2;
+    DEER_CUDA(cudaFuncSetAttribute(moe_logits_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    DEER_CUDA(launch_pdl(moe_logits_kernel, dim3((M + RT_ROWS - 1) / RT_ROWS, (E + RT_EXPERTS - 1) / RT_EXPERTS), dim3(256), smem, st,
+                         static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w_router), M, hid, E, logits));
+    DEER_CUDA(launch_pdl(moe_choose_kernel, dim3((M + 7) / 8), dim3(256), 0, st, (const float*)logits, M, E, top_k, renorm, experts,
+                         weights));
     return DEER_OK;
 }
 
@@ -509,13 +529,16 @@ extern "C" size_t deer_moe_workspace_bytes(int M, int hid, int E, int I, int top
 }
 
 extern "C" int deer_moe_route(const void* x, const void* w_router, int M, int hid, int E, int top_k, int renormalise,
-                              int32_t* experts, float* weights, void* stream) {
+                              int32_t* experts, float* weights, void* workspace, size_t workspace_bytes, void* stream) {
     DEER_CHECK_ARG(x && w_router && experts && weights, DEER_ERR_INVALID_ARG, "deer_moe_route: null argument");
+    DEER_CHECK_ARG(workspace && workspace_bytes >= (size_t)(M > 0 ? M : 0) * (E > 0 ? E : 0) * sizeof(float), DEER_ERR_WORKSPACE,
+                   "deer_moe_route: the workspace holds the M x E router logits (fp32)");
     DEER_CHECK_ARG(deer_aligned16(x) && deer_aligned16(w_router), DEER_ERR_INVALID_ARG, "deer_moe_route: pointers must be 16-byte aligned");
     const int rc = check_shape(M, hid, E, 64, top_k, "deer_moe_route");
     if (rc != DEER_OK) return rc;
     if (M == 0) return DEER_OK;
-    return route(x, w_router, M, hid, E, top_k, renormalise ? 1 : 0, experts, weights, static_cast<cudaStream_t>(stream));
+    return route(x, w_router, M, hid, E, top_k, renormalise ? 1 : 0, static_cast<float*>(workspace), experts, weights,
+                 static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int deer_moe_mlp(const void* x, const void* w_router, const void* w_gate_up, const void* w_down, const void* residual,
@@ -533,7 +556,7 @@ extern "C" int deer_moe_mlp(const void* x, const void* w_router, const void* w_g
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const MoeWs w = carve(workspace, M, hid, E, I, top_k);
     const int pairs = M * top_k;
-    rc = route(x, w_router, M, hid, E, top_k, 1, w.experts, w.weights, st);
+    rc = route(x, w_router, M, hid, E, top_k, 1, w.logits, w.experts, w.weights, st);
     if (rc != DEER_OK) return rc;
     DEER_CUDA(launch_pdl(moe_sort_kernel, dim3(1), dim3(1024), 0, st, (const int32_t*)w.experts, pairs, top_k, E, w.expert_off, w.slot_src,
                          w.slot_of));
