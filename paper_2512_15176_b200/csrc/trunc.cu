@@ -2,7 +2,7 @@
 //
 // Both truncations keep an upper level set {v : z[v] >= tau} of the row, so the work is a selection problem:
 // find the logit value at which the number of tokens at or above it reaches top_k, or at which their probability
-// mass reaches top_p of the mass under consideration.  One thread block per row (a block per SM walking rows,
+// mass reaches top_p of the mass under consideration.  One thread block per row (two blocks per SM walking rows,
 // so that the rows in flight stay in L2 between passes):
 //   1. a histogram pass over the row: tokens are binned by logit value, 2048 bins below the row's largest
 //      possible logit T * lse, a count and a probability mass per bin;
@@ -11,6 +11,9 @@
 //      where the threshold is found exactly: tie groups whole, counts exact, masses in fp64.
 // If the bin holds more tokens than shared memory takes (heavy ties), it is binned again by bit pattern until it
 // does.  Top-k runs first; the nucleus then looks only at the tokens top-k kept, as samplers do.
+// A small top_k on a long row (the usual sampler setting) takes one pass instead: a strided sample of the row
+// places a cut that leaves a few hundred tokens, the pass gathers everything above the cut, and top-k and the
+// nucleus inside it are both resolved in that list; a list that came out short or long falls back to the above.
 // Probabilities are 2^(z c - lse c), c = log2(e) / T, by the hardware's exp2 (2 ulp): the masses only decide in
 // which bin and at which tie group a target is crossed, and enter the result as log(kept mass).
 
@@ -20,7 +23,8 @@ namespace {
 
 constexpr int NB = 2048;           // bins per level (+ 1 for what lies below the binned range)
 constexpr int CAP = 1024;          // candidates resolved exactly in shared memory
-constexpr int THREADS = 1024;
+constexpr int THREADS = 512;        // two blocks per SM: one streams its row while the other scans, sorts or waits
+constexpr int LIST = THREADS;      // candidates of the one-pass path: one per thread in the sort
 constexpr int NW = THREADS / 32;
 constexpr float LOG2E = 1.4426950408889634f;
 
@@ -73,19 +77,29 @@ struct Shared {
     double tot_mass;
 };
 
-// Applies f(z) to every token of the row that is under consideration (z >= floor_z), -0 folded into +0.
+// Applies f(z) to every token of the row that is under consideration (z >= floor_z), -0 folded into +0.  Four
+// 16-byte loads per thread are in flight at a time: a pass is a stream over 600 KB, bound by load latency otherwise.
 template <typename F>
 __device__ __forceinline__ void for_each_token(const Row& r, F f) {
     const int tid = threadIdx.x;
     if ((r.V & 3) == 0) {
         const float4* z4 = reinterpret_cast<const float4*>(r.z);
         const int n4 = r.V >> 2;
-        for (int i = tid; i < n4; i += THREADS) {
-            const float4 x = __ldg(z4 + i);
-            const float e[4] = {x.x + 0.f, x.y + 0.f, x.z + 0.f, x.w + 0.f};
+        for (int i0 = tid; i0 < n4; i0 += 4 * THREADS) {
+            float4 x[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (e[j] >= r.floor_z) f(e[j]);
+            for (int u = 0; u < 4; ++u) {
+                const int i = i0 + u * THREADS;
+                x[u] = i < n4 ? __ldg(z4 + i) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (i0 + u * THREADS >= n4) break;
+                const float e[4] = {x[u].x + 0.f, x[u].y + 0.f, x[u].z + 0.f, x[u].w + 0.f};
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (e[j] >= r.floor_z) f(e[j]);
+            }
         }
     } else {
         for (int i = tid; i < r.V; i += THREADS) {
@@ -364,7 +378,198 @@ __device__ void select_level_set(const Row& r, int kind, int k_target, float fra
     __syncthreads();
 }
 
-__global__ void __launch_bounds__(THREADS, 1) truncate_kernel(int M, int V, const float* __restrict__ logits,
+// Top-k and the nucleus inside it (top_k = 0: the nucleus of the whole row, whose mass is 1 by the definition of
+// lse), resolved in a candidate list that is complete above some cut and holds at least top_k tokens: the list is sorted (descending, one element per thread: a bitonic network, in registers by
+// shuffles within a warp and through shared memory across warps), the probabilities are summed along it in fp64, and
+// both thresholds are read off at the ends of tie groups.  Result in sh.tau / res_cnt / res_mass; false, and no
+// result, when the nucleus reaches below the list.
+static_assert(LIST <= CAP, "the list lives in the exact stage's arrays");
+__device__ bool resolve_sorted(const Row& r, Shared& sh, int n, int top_k, float top_p) {
+    const int tid = threadIdx.x;
+    int P = 32;
+    while (P < n) P <<= 1;
+    float x = tid < n ? sh.cz[tid] : -INFINITY;
+    __syncthreads();
+    for (int size = 2; size <= P; size <<= 1) {
+        const bool desc = (tid & size) == 0;
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            float y;
+            if (stride >= 32) {
+                sh.cz[tid] = x;
+                __syncthreads();
+                y = sh.cz[tid ^ stride];
+                __syncthreads();
+            } else {
+                y = __shfl_xor_sync(0xffffffffu, x, stride);
+            }
+            const bool lower = (tid & stride) == 0;
+            x = (lower == desc) ? fmaxf(x, y) : fminf(x, y);
+        }
+    }
+    sh.cz[tid] = x;
+    __syncthreads();
+    const double p = tid < n ? (double)ex2_approx(fmaf(x, r.c, -r.lc)) : 0.0;
+    int ec, tc;
+    double em, tm;
+    block_scan(tid < n ? 1 : 0, p, ec, em, &tc, &tm, sh);
+    const double upto = em + p;                                   // mass of the list down to and including this element
+    const bool group_end = tid < n && (tid == n - 1 || sh.cz[tid + 1] != x);
+    if (top_k > 0) {
+        const float tau_k = sh.cz[top_k - 1];
+        if (group_end && x == tau_k) {
+            sh.tau = x;
+            sh.res_cnt = tid + 1;
+            sh.res_mass = upto;
+        }
+    } else if (tid == n - 1) {
+        sh.res_cnt = n;                                           // nothing cut by count: the set under consideration
+        sh.res_mass = 1.0;                                        // is the row, and the list must reach its nucleus
+        sh.tot_mass = upto;
+    }
+    __syncthreads();
+    if (top_p >= 1.f) return true;
+    const int cnt_k = sh.res_cnt;
+    const double target = (double)top_p * sh.res_mass;
+    const bool reaches = top_k > 0 || sh.tot_mass >= target;
+    __syncthreads();
+    if (!reaches) return false;
+    if (tid == 0) sh.cross_bin = cnt_k - 1;                       // rounding may leave the whole set just short of the target
+    __syncthreads();
+    if (group_end && tid < cnt_k && upto >= target) atomicMin(&sh.cross_bin, tid);
+    __syncthreads();
+    if (tid == sh.cross_bin) {
+        sh.tau = x;
+        sh.res_cnt = tid + 1;
+        sh.res_mass = upto;
+    }
+    __syncthreads();
+    return true;
+}
+
+// The usual case of a long row and a small top_k, or a nucleus of a few hundred tokens at most (any peaked
+// distribution), in one pass over the row.  A strided sample of 32 tokens per thread is binned first; the bin at which the sample's running count reaches a chosen number gives a cut theta
+// that, for the whole row, is expected to leave a few hundred tokens: at least top_k and no more than the exact
+// stage holds.  The pass over the row then appends every token >= theta to the candidate list in shared memory
+// (no histogram: a compare per token), and both the top-k threshold and the nucleus inside the top-k set are
+// resolved in the sorted list.  The sample only places the cut: the list is complete above theta whatever it was.
+// A list that came out too short or too long is taken again with the cut moved; if that does not settle it, or the
+// nucleus is longer than a list can be, nothing is decided (returns false: the general selection takes over).
+__device__ bool one_pass(const Row& r, int top_k, float top_p, Shared& sh) {
+    const int tid = threadIdx.x;
+    constexpr int SAMPLE4 = 8;                                    // float4 loads per thread in the sample
+    const int n4 = r.V >> 2;
+    if ((r.V & 3) != 0 || n4 < 8 * SAMPLE4 * THREADS) return false;
+    Level lv;
+    lv.by_key = 0;
+    lv.ztop = r.lc / r.c;
+    lv.scale = (float)NB / ((logf((float)r.V) + 20.f) / (r.c / LOG2E));
+    lv.klo = 0;
+    lv.khi = 0xffffffffu;
+    constexpr int PER = (NB + 1 + THREADS - 1) / THREADS;
+    for (int i = tid; i <= NB; i += THREADS) sh.cnt[i] = 0;
+    if (tid == 0) {
+        sh.cross_bin = NB + 1;
+        sh.n_cand = 0;
+    }
+    __syncthreads();
+    {
+        const float4* z4 = reinterpret_cast<const float4*>(r.z);
+        const int stride = n4 / (SAMPLE4 * THREADS);
+        float4 x[SAMPLE4];
+#pragma unroll
+        for (int u = 0; u < SAMPLE4; ++u) x[u] = __ldg(z4 + (size_t)(u * THREADS + tid) * stride);
+#pragma unroll
+        for (int u = 0; u < SAMPLE4; ++u) {
+            atomicAdd(&sh.cnt[bin_of(lv, x[u].x + 0.f)], 1);
+            atomicAdd(&sh.cnt[bin_of(lv, x[u].y + 0.f)], 1);
+            atomicAdd(&sh.cnt[bin_of(lv, x[u].z + 0.f)], 1);
+            atomicAdd(&sh.cnt[bin_of(lv, x[u].w + 0.f)], 1);
+        }
+    }
+    __syncthreads();
+    // the list should hold about max(2 top_k, top_k + 256) tokens, and at most 3/4 of its capacity (which is what a
+    // nucleus alone gets, its size being unknown)
+    const int want = top_k > 0 ? min(max(2 * top_k, top_k + 256), 3 * LIST / 4) : 3 * LIST / 4;
+    const float ratio = (float)r.V / (float)(4 * SAMPLE4 * THREADS);
+    int s_target = max((int)ceilf((float)want / ratio), 4);
+    int c = 0;
+    for (int j = 0; j < PER; ++j) {
+        const int b = tid * PER + j;
+        if (b <= NB) c += sh.cnt[b];
+    }
+    int ec, tc;
+    double em, tm;
+    block_scan(c, 0.0, ec, em, &tc, &tm, sh);
+    // A list that came out too long or too short moves the cut by what it counted and takes the pass again (the row
+    // is in L2 by then): three attempts at most.
+    for (int attempt = 0; attempt < 3; ++attempt) {
+        if (tid == 0) {
+            sh.cross_bin = NB + 1;
+            sh.n_cand = 0;
+        }
+        __syncthreads();
+        {
+            int rc = ec;
+            for (int j = 0; j < PER; ++j) {
+                const int b = tid * PER + j;
+                if (b > NB) break;
+                rc += sh.cnt[b];
+                if (rc >= s_target) {
+                    atomicMin(&sh.cross_bin, b);
+                    break;
+                }
+            }
+        }
+        __syncthreads();
+        const int bs = sh.cross_bin;
+        __syncthreads();
+        if (bs >= NB) return false;                               // the cut would fall below the binned range
+        const float theta = lv.ztop - (float)(bs + 1) / lv.scale;
+        {
+            const float4* z4 = reinterpret_cast<const float4*>(r.z);
+            auto keep = [&](float z) {
+                if (z >= theta) {
+                    const int slot = atomicAdd(&sh.n_cand, 1);
+                    if (slot < LIST) sh.cz[slot] = z + 0.f;
+                }
+            };
+            for (int i0 = tid; i0 < n4; i0 += 4 * THREADS) {
+                float4 x[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int i = i0 + u * THREADS;
+                    x[u] = i < n4 ? __ldg(z4 + i) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (fmaxf(fmaxf(x[u].x, x[u].y), fmaxf(x[u].z, x[u].w)) >= theta) {   // one test per 16 bytes; few pass
+                        keep(x[u].x);
+                        keep(x[u].y);
+                        keep(x[u].z);
+                        keep(x[u].w);
+                    }
+            }
+        }
+        __syncthreads();
+        const int n = sh.n_cand;
+        __syncthreads();
+        int s_next;
+        if (n > LIST) {
+            s_next = (int)((float)s_target * (0.6f * (float)LIST / (float)n));
+        } else if (n < max(top_k, 1)) {
+            s_next = (int)ceilf((float)s_target * 1.5f * (float)want / (float)max(n, 1));
+        } else {
+            if (resolve_sorted(r, sh, n, top_k, top_p)) return true;
+            if (2 * n > LIST) return false;                       // the nucleus is longer than a list can be
+            s_next = 2 * s_target;
+        }
+        if (s_next < 1 || s_next == s_target) return false;
+        s_target = s_next;
+    }
+    return false;
+}
+
+__global__ void __launch_bounds__(THREADS, 2) truncate_kernel(int M, int V, const float* __restrict__ logits,
                                                               const float* __restrict__ lse, float inv_t, int top_k, float top_p,
                                                               float* __restrict__ tau_out, float* __restrict__ lse_out) {
     extern __shared__ unsigned char smem_raw[];
@@ -381,14 +586,26 @@ __global__ void __launch_bounds__(THREADS, 1) truncate_kernel(int M, int V, cons
         float tau = -INFINITY;
         double mass = 1.0;
         bool any = false;
-        if (top_k > 0 && top_k < V) {
+        bool done = false;
+        const bool cut_by_count = top_k > 0 && top_k < V;
+        if (cut_by_count ? top_k <= LIST / 4 : top_p < 1.f) {
+            done = one_pass(r, cut_by_count ? top_k : 0, top_p, sh);
+            __syncthreads();
+            if (done) {
+                tau = sh.tau;
+                mass = sh.res_mass;
+                any = true;
+            }
+            __syncthreads();
+        }
+        if (!done && top_k > 0 && top_k < V) {
             select_level_set(r, BY_COUNT, top_k, 0.f, sh);
             tau = sh.tau;
             mass = sh.res_mass;
             any = true;
             __syncthreads();
         }
-        if (top_p < 1.f) {
+        if (!done && top_p < 1.f) {
             r.floor_z = tau;
             select_level_set(r, BY_MASS, 0, top_p, sh);
             tau = sh.tau;
@@ -415,7 +632,7 @@ extern "C" int deer_truncate(int M, int V, const float* target_logits, const flo
     if (M == 0) return DEER_OK;
     const int sms = deer_sm_count();
     DEER_CUDA(cudaFuncSetAttribute(truncate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(Shared)));
-    DEER_CUDA(launch_pdl(truncate_kernel, dim3(M < sms ? M : sms), dim3(THREADS), sizeof(Shared), static_cast<cudaStream_t>(stream), M, V,
+    DEER_CUDA(launch_pdl(truncate_kernel, dim3(M < 2 * sms ? M : 2 * sms), dim3(THREADS), sizeof(Shared), static_cast<cudaStream_t>(stream), M, V,
                          target_logits, target_lse, 1.f / temperature, top_k, top_p, tau, lse_trunc));
     return DEER_OK;
 }

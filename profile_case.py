@@ -5,6 +5,8 @@ program that profiler captures are taken from.
     python profile_case.py attn --B 8 --Hq 32 --Hkv 8 --k 32 --ctx 8192 --iters 3
     python profile_case.py qstats --B 4 --k 32 --V 151936 --iters 3
     python profile_case.py layer --B 1 --k 32 --ctx 4096 --hid 4096 --inter 12288 --iters 20
+    python profile_case.py trunc --M 512 --V 151936 --top-k-trunc 50 --top-p 0.9 --iters 3
+    python profile_case.py moe --M 32 --hid 2048 --experts 128 --inter 768 --top-k 8 --iters 3
 
 Prints the average CUDA-event time per call and the achieved GB/s over the
 call's algorithmic bytes.
@@ -28,7 +30,10 @@ from paper_2512_15176_b200 import workload as W  # noqa: E402
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["lmhead", "attn", "qstats", "layer"])
+    ap.add_argument("what", choices=["lmhead", "attn", "qstats", "layer", "trunc", "moe"])
+    ap.add_argument("--top-p", type=float, default=0.9)
+    ap.add_argument("--top-k-trunc", type=int, default=50)
+    ap.add_argument("--peaked", action="store_true", help="trunc: rows with a language model's rank-frequency shape")
     ap.add_argument("--inter", type=int, default=12288)
     ap.add_argument("--separate", action="store_true", help="layer: every step as a call of its own instead of the fused calls")
     ap.add_argument("--experts", type=int, default=0, help="layer: routed MLP with this many experts (0 = dense)")
@@ -124,6 +129,34 @@ def main():
         nbytes = dense + W.algorithmic_bytes(cfg, lengths)["attn"]
         flops = 2.0 * cfg.M * (dense / 2 if not a.experts else sum(t.numel() for n, t in w.items() if n in ("wqkv", "wo"))
                                + a.top_k * 3 * a.inter * hid)
+    elif a.what == "trunc":
+        # top-k / nucleus threshold per row of fp32 logits (the sampling setting's truncation ahead of the acceptance)
+        z = W.normal(35, "z", (a.M, a.V), 1.3, dtype=torch.float32, device=dev)
+        if a.peaked:        # a language model's shape: -1.1 log(rank) under a permutation per row, plus noise
+            base = -1.1 * torch.log(torch.arange(1, a.V + 1, device=dev, dtype=torch.float32))
+            perm = torch.argsort(torch.rand(a.M, a.V, device=dev, generator=torch.Generator(dev).manual_seed(35)), dim=1)
+            z = z * 0.25 + base[perm]
+        lse = torch.logsumexp(z / 0.6, dim=1).contiguous()
+        tau = torch.empty(a.M, dtype=torch.float32, device=dev)
+        lse_t = torch.empty(a.M, dtype=torch.float32, device=dev)
+        call = lambda: L.deer_truncate(z, lse, 0.6, a.top_k_trunc, a.top_p, tau, lse_t)
+        nbytes = a.M * a.V * 4
+        flops = 0.0
+    elif a.what == "moe":
+        # the routed MLP alone at M rows
+        E, I, hid = a.experts or 128, a.inter, a.hid
+        mk = lambda n, shape, sig: W.normal(36, n, shape, sig, device=dev)
+        x = mk("x", (a.M, hid), 1.0)
+        wr, wgu, wd = mk("wr", (E, hid), hid ** -0.5 * 3.0), mk("wgu", (E, 2 * I, hid), hid ** -0.5), mk("wd", (E, hid, I), I ** -0.5)
+        y = torch.empty(a.M, hid, dtype=torch.bfloat16, device=dev)
+        ws = torch.empty(L.deer_moe_workspace_bytes(a.M, hid, E, I, a.top_k), dtype=torch.uint8, device=dev)
+        e_ids = torch.empty(a.M, a.top_k, dtype=torch.int32, device=dev)
+        e_w = torch.empty(a.M, a.top_k, dtype=torch.float32, device=dev)
+        L.deer_moe_route(x, wr, a.top_k, e_ids, e_w)
+        torch.cuda.synchronize()
+        call = lambda: L.deer_moe_mlp(x, wr, wgu, wd, y, a.top_k, ws)
+        nbytes = int(torch.unique(e_ids).numel()) * 3 * I * hid * 2 + E * hid * 2       # the chosen experts' matrices + the router
+        flops = 2.0 * a.M * a.top_k * 3 * I * hid
     else:
         M = a.B * a.k
         ql = W.normal(33, "ql", (a.B, a.k, a.V), 1.0, dtype=torch.float32, device=dev)

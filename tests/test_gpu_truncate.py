@@ -105,6 +105,72 @@ def test_truncate_with_heavy_ties():
         np.testing.assert_allclose(got_lse, want_lse, atol=3e-4, rtol=0)
 
 
+def _peaked_rows(seed, M, V, slope):
+    """Rows shaped like a language model's: logit = -slope * log(rank) under a random permutation, plus noise."""
+    g = np.random.default_rng(seed)
+    z = np.empty((M, V), dtype=np.float32)
+    base = (-slope * np.log(np.arange(1, V + 1))).astype(np.float32)
+    for m in range(M):
+        z[m, g.permutation(V)] = base
+    return z + W.normal(seed, "noise", (M, V), 0.3, dtype=torch.float32).numpy()
+
+
+def test_truncate_peaked_rows():
+    """Peaked rows of full vocabulary length: the nucleus is a few tokens to a few hundred (and, at 0.9999, far more
+    than any short candidate list holds)."""
+    T = float(np.float32(0.8))
+    z32 = _peaked_rows(1360, 6, 151936, 1.1)
+    for top_k, top_p in [(0, 0.9), (0, 0.5), (40, 0.95), (0, 0.9999), (100, 1.0)]:
+        clear = True
+        if top_p < 1.0:
+            top_p, clear = _pick_top_p(z32, T, top_k, top_p)
+        want_tau, want_lse = _expected(z32, T, top_k, top_p)
+        got_tau, got_lse = _run_truncate(z32, T, top_k, top_p)
+        for m in range(z32.shape[0]):
+            _check_level_set(z32[m], T, top_k, top_p, got_tau[m], f"row {m} top_k {top_k} top_p {top_p}")
+        if clear:
+            np.testing.assert_array_equal(got_tau, want_tau)
+            np.testing.assert_allclose(got_lse, want_lse, atol=3e-4, rtol=0)
+
+
+def test_truncate_on_rows_that_mislead_a_sample():
+    """Long rows whose largest logits sit exactly on, or exactly off, a regular stride of positions, or fill a tie
+    group larger than any candidate list: a cut placed from a strided sample of the row is then far too high or
+    far too low, and the result must still be the oracle's (the kernel may use a sample only to place a cut)."""
+    T = float(np.float32(0.8))
+    V = 151936
+    base = W.normal(1350, "z", (6, V), 1.0, dtype=torch.float32).numpy() - np.float32(6.0)
+    pos = np.arange(V)
+    rows = []
+    for stride4 in (9, 8, 37):                                  # float4 strides a sampler might use
+        on = (pos // 4) % stride4 == 0
+        z = base[len(rows)].copy()                              # high values exactly on the stride
+        z[on] += np.float32(9.0)
+        rows.append(z)
+    z = base[3].copy()                                          # 40 high values on the stride 9, nothing else near
+    z[(np.arange(40) * 9 * 4 * 50)] = np.float32(8.0) + np.arange(40, dtype=np.float32) / 64
+    rows.append(z)
+    z = base[4].copy()                                          # 3000 high values, all off the stride 9
+    off = pos[(pos // 4) % 9 == 4][:3000]
+    z[off] = np.float32(7.0) + (np.arange(3000) % 17).astype(np.float32) / 32
+    rows.append(z)
+    z = base[5].copy()                                          # a tie group of 5000 at the top
+    z[:5000] = np.float32(6.5)
+    rows.append(z)
+    z32 = np.stack(rows).astype(np.float32)
+    for top_k, top_p in [(50, 1.0), (20, 0.9), (300, 0.5), (1, 1.0)]:
+        clear = True
+        if top_p < 1.0:
+            top_p, clear = _pick_top_p(z32, T, top_k, top_p)
+        want_tau, want_lse = _expected(z32, T, top_k, top_p)
+        got_tau, got_lse = _run_truncate(z32, T, top_k, top_p)
+        for m in range(len(rows)):
+            _check_level_set(z32[m], T, top_k, top_p, got_tau[m], f"row {m} top_k {top_k} top_p {top_p}")
+        if clear:
+            np.testing.assert_array_equal(got_tau, want_tau)
+            np.testing.assert_allclose(got_lse, want_lse, atol=3e-4, rtol=0)
+
+
 def _sample_truncated(cfg, zt32, ql, drafts, u, r, top_k, top_p, from_oracle, eos=-1, bonus=False, tau_out=None):
     """deer_accept_truncated on given fp32 logits.  from_oracle: the thresholds and truncated log-sum-exps come from the
     oracle (the acceptance in isolation); otherwise from deer_truncate (the two calls chained; tau_out receives its
