@@ -447,7 +447,8 @@ __device__ bool resolve_sorted(const Row& r, Shared& sh, int n, int top_k, float
 }
 
 // The usual case of a long row and a small top_k, or a nucleus of a few hundred tokens at most (any peaked
-// distribution), in one pass over the row.  A strided sample of 32 tokens per thread is binned first; the bin at which the sample's running count reaches a chosen number gives a cut theta
+// distribution), in one pass over the row.  A sample of 32 tokens per thread, in evenly spaced 128-byte runs, is
+// binned first; the bin at which the sample's running count reaches a chosen number gives a cut theta
 // that, for the whole row, is expected to leave a few hundred tokens: at least top_k and no more than the exact
 // stage holds.  The pass over the row then appends every token >= theta to the candidate list in shared memory
 // (no histogram: a compare per token), and both the top-k threshold and the nucleus inside the top-k set are
@@ -474,10 +475,14 @@ __device__ bool one_pass(const Row& r, int top_k, float top_p, Shared& sh) {
     __syncthreads();
     {
         const float4* z4 = reinterpret_cast<const float4*>(r.z);
-        const int stride = n4 / (SAMPLE4 * THREADS);
+        // runs of 128 bytes (a DRAM burst is used whole), evenly spaced over the row
+        const int run_stride = n4 / (SAMPLE4 * THREADS / 8);
         float4 x[SAMPLE4];
 #pragma unroll
-        for (int u = 0; u < SAMPLE4; ++u) x[u] = __ldg(z4 + (size_t)(u * THREADS + tid) * stride);
+        for (int u = 0; u < SAMPLE4; ++u) {
+            const int j = u * THREADS + tid;
+            x[u] = __ldg(z4 + (size_t)(j >> 3) * run_stride + (j & 7));
+        }
 #pragma unroll
         for (int u = 0; u < SAMPLE4; ++u) {
             atomicAdd(&sh.cnt[bin_of(lv, x[u].x + 0.f)], 1);

@@ -139,7 +139,7 @@ def test_truncate_on_rows_that_mislead_a_sample():
     far too low, and the result must still be the oracle's (the kernel may use a sample only to place a cut)."""
     T = float(np.float32(0.8))
     V = 151936
-    base = W.normal(1350, "z", (6, V), 1.0, dtype=torch.float32).numpy() - np.float32(6.0)
+    base = W.normal(1350, "z", (7, V), 1.0, dtype=torch.float32).numpy() - np.float32(6.0)
     pos = np.arange(V)
     rows = []
     for stride4 in (9, 8, 37):                                  # float4 strides a sampler might use
@@ -156,6 +156,9 @@ def test_truncate_on_rows_that_mislead_a_sample():
     rows.append(z)
     z = base[5].copy()                                          # a tie group of 5000 at the top
     z[:5000] = np.float32(6.5)
+    rows.append(z)
+    z = base[6].copy()                                          # high values in 128-byte runs, 512 runs per row
+    z[(pos // 4) % (V // 4 // 512) < 8] += np.float32(9.0)
     rows.append(z)
     z32 = np.stack(rows).astype(np.float32)
     for top_k, top_p in [(50, 1.0), (20, 0.9), (300, 0.5), (1, 1.0)]:
