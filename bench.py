@@ -331,8 +331,7 @@ def measure(cfg, steps, warmup, dev, peaks, flush, world=1, rank=0, with_e2e=Fal
 
     def phase_accept():
         if not bidir:              # the drafter's block fill proposes; nothing is accepted or committed
-            vs.accept()
-            vs.commit()
+            vs.accept_commit()
 
     phases = [phase_attn, vs.lmhead, phase_accept]
 

@@ -116,6 +116,14 @@ int deer_kv_reserve(deer_kv* kv, const int32_t* seq_ids, int B, int k, void* str
  * (e.g. deer_accept's accept_len), so no host round-trip is needed. */
 int deer_kv_commit(deer_kv* kv, const int32_t* seq_ids, const int32_t* keep, int B, int k, void* stream);
 
+/* (3) + (4) in one launch for greedy verification: deer_accept(DEER_ACC_GREEDY [| DEER_ACC_BONUS]) followed by
+ * deer_kv_commit(keep = accept_len), same arguments, same results in accept_len / out_ids / n_out and in the cache
+ * (Section 3.2's exact-match rule, Algorithm 1's update of j).  All arrays are device pointers; B <= 1024.
+ * Errors: DEER_ERR_UNSUPPORTED for any other mode or size; the cache's status word as deer_kv_commit. */
+int deer_accept_commit(deer_kv* kv, const int32_t* seq_ids, int mode, int B, int k, const int32_t* draft_ids,
+                       const int32_t* target_ids, int32_t eos_id, int32_t* accept_len, int32_t* out_ids, int32_t* n_out,
+                       void* stream);
+
 /* Copy the status word to *code (host pointer) after synchronising `stream`,
  * and reset it to 0 on the device. */
 int deer_kv_status(deer_kv* kv, int32_t* code, void* stream);

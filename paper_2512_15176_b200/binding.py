@@ -24,7 +24,7 @@ DEER_ACC_GREEDY, DEER_ACC_SAMPLE, DEER_ACC_SAMPLE_PRESTATS, DEER_ACC_BONUS = 0, 
 DEER_EMIT_PENDING = 1
 
 EXPORTS = [
-    "deer_last_error", "deer_kv_create", "deer_kv_destroy", "deer_kv_reserve", "deer_kv_commit", "deer_kv_status",
+    "deer_last_error", "deer_kv_create", "deer_kv_destroy", "deer_kv_reserve", "deer_kv_commit", "deer_accept_commit", "deer_kv_status",
     "deer_block_attn_workspace_bytes", "deer_block_attn", "deer_lmhead_workspace_bytes", "deer_lmhead_select",
     "deer_accept_workspace_bytes", "deer_accept", "deer_verify_step_host",
     "deer_lmhead_static_max_rows", "deer_lmhead_select_static", "deer_emit", "deer_draft_stats",
@@ -73,6 +73,8 @@ def lib() -> ctypes.CDLL:
     L.deer_kv_destroy.argtypes = [c_void_p]
     L.deer_kv_reserve.argtypes = [c_void_p, c_void_p, c_int, c_int, c_void_p]
     L.deer_kv_commit.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int, c_void_p]
+    L.deer_accept_commit.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_void_p, c_int32, c_void_p, c_void_p,
+                                     c_void_p, c_void_p]
     L.deer_kv_status.argtypes = [c_void_p, POINTER(c_int32), c_void_p]
     L.deer_block_attn_workspace_bytes.restype = c_size_t
     L.deer_block_attn_workspace_bytes.argtypes = [c_int] * 6
@@ -263,6 +265,11 @@ def deer_accept(mode, B, k, V, draft_ids, target_ids, target_logits, target_lse,
                              _ptr(accept_len), _ptr(out_ids), _ptr(n_out), _ptr(workspace),
                              workspace.numel() * workspace.element_size() if workspace is not None else 0,
                              _stream(stream)))
+
+
+def deer_accept_commit(kv: KVCache, seq_ids, mode, k, draft_ids, target_ids, eos_id, accept_len, out_ids, n_out, stream=None):
+    _check(lib().deer_accept_commit(kv.handle, _ptr(seq_ids), int(mode), seq_ids.numel(), k, _ptr(draft_ids), _ptr(target_ids),
+                                    int(eos_id), _ptr(accept_len), _ptr(out_ids), _ptr(n_out), _stream(stream)))
 
 
 def deer_truncate(target_logits, target_lse, temperature, top_k, top_p, tau, lse_trunc, stream=None):

@@ -10,6 +10,7 @@
 // (b) and (c) are one kernel.  Only (a) touches more than a few rows.
 
 #include "common.cuh"
+#include "greedy.cuh"
 
 namespace {
 
@@ -24,22 +25,8 @@ __global__ void accept_greedy_kernel(int B, int k, int kd, const int32_t* __rest
     pdl_trigger();
     pdl_wait();
     if (b >= B) return;
-    const int32_t* d = draft + (size_t)b * k;
-    const int32_t* t = target + (size_t)b * k;
-    int32_t* o = out_ids + (size_t)b * k;
-    int a = 0;
-    while (a < kd && d[a] == t[a]) ++a;          // kd = k - 1 with the extra row: then a < k and t[a] is always emitted
-    int n = a < k ? a + 1 : a;
-    for (int i = 0; i < k; ++i) o[i] = i < a ? d[i] : (i == a ? t[i] : -1);
-    if (eos_id >= 0) {
-        for (int i = 0; i < n; ++i)
-            if (o[i] == eos_id) {
-                for (int j = i + 1; j < n; ++j) o[j] = -1;
-                n = i + 1;
-                a = min(a, n);
-                break;
-            }
-    }
+    int n;
+    const int a = greedy_accept_row(draft + (size_t)b * k, target + (size_t)b * k, out_ids + (size_t)b * k, k, kd, eos_id, &n);
     accept_len[b] = a;
     n_out[b] = n;
 }

@@ -13,6 +13,7 @@
 #include <new>
 
 #include "common.cuh"
+#include "greedy.cuh"
 
 // ---- error text ------------------------------------------------------------
 static thread_local char g_err[512] = "";
@@ -129,13 +130,11 @@ kv_reserve_kernel(deer_kv_desc d, const int32_t* __restrict__ seq_ids, int B, in
     if (b == 0) *d.free_top = top - total;
 }
 
-__global__ void __launch_bounds__(KV_THREADS)
-kv_commit_kernel(deer_kv_desc d, const int32_t* __restrict__ seq_ids, const int32_t* __restrict__ keep, int B, int k) {
-    __shared__ int warp_sums[32];
-    __shared__ int total;
+// The body of the commit for thread b of the block: seq_len[s] += keep (clamped), pages wholly beyond the new length
+// go back to the free stack.  `keep` is this thread's sequence's value; every thread of the block calls it.
+__device__ __forceinline__ void commit_rows(const deer_kv_desc& d, const int32_t* __restrict__ seq_ids, int keep, int B, int k,
+                                            int* warp_sums, int* total) {
     const int b = threadIdx.x;
-    pdl_trigger();
-    pdl_wait();
     int s = -1, have = 0, need_pages = 0;
     if (b < B) {
         s = seq_ids[b];
@@ -143,7 +142,7 @@ kv_commit_kernel(deer_kv_desc d, const int32_t* __restrict__ seq_ids, const int3
             deer_report(d.status, DEER_ERR_INVALID_ARG);
             s = -1;
         } else {
-            int kp = keep[b];
+            int kp = keep;
             kp = kp < 0 ? 0 : (kp > k ? k : kp);
             have = d.n_pages[s];
             int n = d.seq_len[s] + kp;
@@ -157,9 +156,9 @@ kv_commit_kernel(deer_kv_desc d, const int32_t* __restrict__ seq_ids, const int3
         }
     }
     const int surplus = (s >= 0 && have > need_pages) ? have - need_pages : 0;
-    const int offset = block_exclusive_scan(surplus, &total, warp_sums);
+    const int offset = block_exclusive_scan(surplus, total, warp_sums);
     const int top = *d.free_top;
-    if (top + total > d.num_pages) {          // inconsistent state: more pages returned than exist
+    if (top + *total > d.num_pages) {         // inconsistent state: more pages returned than exist
         if (b == 0) deer_report(d.status, DEER_ERR_BAD_PAGE);
         return;
     }
@@ -172,7 +171,37 @@ kv_commit_kernel(deer_kv_desc d, const int32_t* __restrict__ seq_ids, const int3
         d.n_pages[s] = need_pages;
     }
     __syncthreads();
-    if (b == 0) *d.free_top = top + total;
+    if (b == 0) *d.free_top = top + *total;
+}
+
+__global__ void __launch_bounds__(KV_THREADS)
+kv_commit_kernel(deer_kv_desc d, const int32_t* __restrict__ seq_ids, const int32_t* __restrict__ keep, int B, int k) {
+    __shared__ int warp_sums[32];
+    __shared__ int total;
+    pdl_trigger();
+    pdl_wait();
+    commit_rows(d, seq_ids, threadIdx.x < B ? keep[threadIdx.x] : 0, B, k, warp_sums, &total);
+}
+
+// Greedy acceptance and the commit of what it accepted, one thread per sequence: the end of a greedy verify step in
+// one launch.
+__global__ void __launch_bounds__(KV_THREADS)
+kv_accept_commit_kernel(deer_kv_desc d, const int32_t* __restrict__ seq_ids, int B, int k, int kd, const int32_t* __restrict__ draft,
+                        const int32_t* __restrict__ target, int32_t eos_id, int32_t* __restrict__ accept_len,
+                        int32_t* __restrict__ out_ids, int32_t* __restrict__ n_out) {
+    __shared__ int warp_sums[32];
+    __shared__ int total;
+    const int b = threadIdx.x;
+    pdl_trigger();
+    pdl_wait();
+    int a = 0;
+    if (b < B) {
+        int n;
+        a = greedy_accept_row(draft + (size_t)b * k, target + (size_t)b * k, out_ids + (size_t)b * k, k, kd, eos_id, &n);
+        accept_len[b] = a;
+        n_out[b] = n;
+    }
+    commit_rows(d, seq_ids, a, B, k, warp_sums, &total);
 }
 
 // ---- entry points ----------------------------------------------------------
@@ -191,5 +220,21 @@ extern "C" int deer_kv_commit(deer_kv* kv, const int32_t* seq_ids, const int32_t
     DEER_CHECK_ARG(k >= 0 && k <= DEER_MAX_BLOCK, DEER_ERR_UNSUPPORTED, "deer_kv_commit: k must be in [0, 32]");
     if (B == 0) return DEER_OK;
     DEER_CUDA(launch_pdl(kv_commit_kernel, dim3(1), dim3(KV_THREADS), 0, static_cast<cudaStream_t>(stream), kv->d, seq_ids, keep, B, k));
+    return DEER_OK;
+}
+
+extern "C" int deer_accept_commit(deer_kv* kv, const int32_t* seq_ids, int mode, int B, int k, const int32_t* draft_ids,
+                                  const int32_t* target_ids, int32_t eos_id, int32_t* accept_len, int32_t* out_ids, int32_t* n_out,
+                                  void* stream) {
+    DEER_CHECK_ARG(kv && seq_ids && draft_ids && target_ids && accept_len && out_ids && n_out, DEER_ERR_INVALID_ARG,
+                   "deer_accept_commit: null argument");
+    DEER_CHECK_ARG((mode & ~DEER_ACC_BONUS) == DEER_ACC_GREEDY, DEER_ERR_UNSUPPORTED,
+                   "deer_accept_commit: greedy acceptance only (sampling takes deer_accept, then deer_kv_commit)");
+    DEER_CHECK_ARG(B >= 0 && B <= KV_THREADS, DEER_ERR_UNSUPPORTED, "deer_accept_commit: B must be in [0, %d]", KV_THREADS);
+    DEER_CHECK_ARG(k >= 1 && k <= DEER_MAX_BLOCK, DEER_ERR_UNSUPPORTED, "deer_accept_commit: k must be in [1, 32]");
+    if (B == 0) return DEER_OK;
+    const int kd = (mode & DEER_ACC_BONUS) ? k - 1 : k;
+    DEER_CUDA(launch_pdl(kv_accept_commit_kernel, dim3(1), dim3(KV_THREADS), 0, static_cast<cudaStream_t>(stream), kv->d, seq_ids, B, k,
+                         kd, draft_ids, target_ids, eos_id, accept_len, out_ids, n_out));
     return DEER_OK;
 }

@@ -95,10 +95,8 @@ int enqueue(deer_kv* kv, const deer_step_dev* dev, const void* w, const void* q_
     rc = deer_lmhead_select(dev->h, w, (int)M, hid, V, DEER_SEL_ARGMAX, 1.f, nullptr, dev->target_ids, nullptr, nullptr, nullptr,
                             nullptr, dev->lm_ws, dev->lm_ws_bytes, stream);
     if (rc != DEER_OK) return rc;
-    rc = deer_accept(DEER_ACC_GREEDY, B, k, V, dev->draft_ids, dev->target_ids, nullptr, nullptr, nullptr, 1.f, nullptr, nullptr,
-                     nullptr, -1, dev->accept_len, dev->out_ids, dev->n_out, nullptr, 0, stream);
-    if (rc != DEER_OK) return rc;
-    rc = deer_kv_commit(kv, dev->seq_ids, dev->accept_len, B, k, stream);
+    rc = deer_accept_commit(kv, dev->seq_ids, DEER_ACC_GREEDY, B, k, dev->draft_ids, dev->target_ids, -1, dev->accept_len,
+                            dev->out_ids, dev->n_out, stream);
     if (rc != DEER_OK) return rc;
     DEER_CUDA(cudaMemcpyAsync(accept_len_host, dev->accept_len, (size_t)B * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     DEER_CUDA(cudaMemcpyAsync(out_ids_host, dev->out_ids, M * sizeof(int32_t), cudaMemcpyDeviceToHost, st));

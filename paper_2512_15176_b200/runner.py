@@ -132,6 +132,16 @@ class VerifyStep:
     def commit(self):
         L.deer_kv_commit(self.kv, self.seq_ids, self.accept_len, self.cfg.k)
 
+    def accept_commit(self):
+        """The end of the step: one launch when the acceptance is greedy, acceptance then commit otherwise."""
+        if self.cfg.mode == "sample":
+            self.accept()
+            self.commit()
+            return
+        extra = L.DEER_ACC_BONUS if self.bonus else 0
+        L.deer_accept_commit(self.kv, self.seq_ids, L.DEER_ACC_GREEDY | extra, self.cfg.k, self.draft_ids, self.target_ids,
+                             self.eos_id, self.accept_len, self.out_ids, self.n_out)
+
     def run(self):
         """One whole step.  The drafter block fill (bidirectional mask) has no
         acceptance and commits nothing."""
@@ -144,14 +154,13 @@ class VerifyStep:
         self.reserve()
         self.attn(append=True)
         self.lmhead()
-        self.accept()
-        self.commit()
+        self.accept_commit()
 
-    #: kernels launched by one run(), by mode (attention + merge, LM head, reserve + commit, acceptance)
+    #: kernels launched by one run(), by mode (attention + merge, LM head, reserve, acceptance and commit)
     def launches_per_step(self) -> int:
         if self.cfg.mask == MASK_BIDIR:
             return 4
-        return 2 + 2 + 2 + (2 if self.cfg.mode == "sample" else 1)
+        return 2 + 2 + 1 + (3 if self.cfg.mode == "sample" else 1)
 
 
 class DecodeLoop:

@@ -205,6 +205,40 @@ def test_kv_soak_64_steps(B, k, Hkv, D):
     Hn.check_attention(out.cpu(), want, "after soak")
 
 
+@pytest.mark.parametrize("B,k,bonus,with_eos", [(1, 32, False, False), (64, 32, False, True), (300, 5, True, False), (7, 1, False, True)])
+def test_accept_commit_in_one_launch(B, k, bonus, with_eos):
+    """deer_accept_commit against the oracle's greedy acceptance followed by its commit: the acceptance outputs and
+    the whole cache state (lengths, page counts, page table, free stack), bit for bit."""
+    from paper_2512_15176_b200 import binding as L
+    cfg = W.StepConfig("ac", B, 4, 2, 64, k, 64, 5000, (0, 200), seed=960 + B)
+    st = Hn.draw_state(cfg, stress=True)
+    okv = Hn.oracle_kv(st)
+    kv = Hn.gpu_kv(st)
+    ids = np.arange(B)
+    seq_ids = torch.arange(B, dtype=torch.int32, device="cuda")
+    target = W.rng(cfg.seed, "t").integers(0, cfg.V, size=(B, k)).astype(np.int32)
+    draft = W.plant_drafts(cfg, target, W.planted_prefix_lengths(cfg))
+    eos = int(target[0, min(1, k - 1)]) if with_eos else -1
+    a = torch.full((B,), -9, dtype=torch.int32, device="cuda")
+    o = torch.full((B, k), -9, dtype=torch.int32, device="cuda")
+    n = torch.full((B,), -9, dtype=torch.int32, device="cuda")
+    L.deer_kv_reserve(kv, seq_ids, k)
+    L.deer_accept_commit(kv, seq_ids, L.DEER_ACC_GREEDY | (L.DEER_ACC_BONUS if bonus else 0), k, torch.as_tensor(draft, device="cuda"),
+                         torch.as_tensor(target, device="cuda"), eos, a, o, n)
+    torch.cuda.synchronize()
+    want = O.accept_greedy(draft, target, eos, bonus=bonus)
+    for g, w_ in zip((a.cpu().numpy(), o.cpu().numpy(), n.cpu().numpy()), want):
+        np.testing.assert_array_equal(g, w_)
+    assert okv.reserve(ids, k)
+    okv.commit(ids, want[0])
+    Hn.kv_state_equal(kv, okv, "after accept + commit")
+    assert L.deer_kv_status(kv) == 0
+    # sampling is not this call's business
+    with pytest.raises(L.DeerError):
+        L.deer_accept_commit(kv, seq_ids, L.DEER_ACC_SAMPLE, k, torch.as_tensor(draft, device="cuda"),
+                             torch.as_tensor(target, device="cuda"), eos, a, o, n)
+
+
 def test_reserve_without_pages_reports_and_changes_nothing():
     from paper_2512_15176_b200 import binding as L
     cfg = W.StepConfig("np", 3, 4, 2, 64, 32, 64, 64, (16, 16), seed=950)

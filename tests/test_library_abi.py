@@ -58,6 +58,11 @@ def test_host_side_argument_validation(lib):
         assert lib.deer_block_attn(kv, fake, fake, fake, fake, fake, 0, 8, 4, 0, 0, 1.0, 64, None, 0, None) == L.DEER_OK
         assert lib.deer_kv_reserve(kv, fake, 0, 8, None) == L.DEER_OK
         assert lib.deer_kv_commit(kv, fake, fake, 0, 8, None) == L.DEER_OK
+        # acceptance + commit in one launch: greedy only, empty batch is a no-op
+        assert lib.deer_accept_commit(kv, fake, L.DEER_ACC_GREEDY, 0, 8, fake, fake, -1, fake, fake, fake, None) == L.DEER_OK
+        assert lib.deer_accept_commit(kv, fake, L.DEER_ACC_SAMPLE, 4, 8, fake, fake, -1, fake, fake, fake, None) == L.DEER_ERR_UNSUPPORTED
+        assert lib.deer_accept_commit(kv, fake, L.DEER_ACC_GREEDY, 4, 40, fake, fake, -1, fake, fake, fake, None) == L.DEER_ERR_UNSUPPORTED
+        assert lib.deer_accept_commit(kv, None, L.DEER_ACC_GREEDY, 4, 8, fake, fake, -1, fake, fake, fake, None) == L.DEER_ERR_INVALID_ARG
         assert lib.deer_kv_reserve(kv, fake, 4, 40, None) == L.DEER_ERR_UNSUPPORTED
     finally:
         lib.deer_kv_destroy(kv)
