@@ -403,14 +403,21 @@ def measure(cfg, steps, warmup, dev, peaks, flush, world=1, rank=0, with_e2e=Fal
     e2e_s, h2d, d2h = 0.0, 0, 0
     if greedy and with_e2e:
         pin = lambda t: t.contiguous().pin_memory()
-        hq, hkb, hvb, hh = pin(q), pin(kb), pin(vb), pin(h)
+        # q, k_blk, v_blk side by side in one pinned buffer and one device buffer, the three results likewise: the call
+        # then moves each group with one copy
+        nq, nk = q.numel(), kb.numel()
+        hin = torch.empty(nq + 2 * nk, dtype=torch.bfloat16).pin_memory()
+        hq, hkb, hvb = hin[:nq].view_as(q), hin[nq:nq + nk].view_as(kb), hin[nq + nk:].view_as(vb)
+        hq.copy_(q), hkb.copy_(kb), hvb.copy_(vb)
+        hh = pin(h)
         hd = pin(torch.from_numpy(drafts))
-        ha = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
-        ho = torch.empty(cfg.B, cfg.k, dtype=torch.int32).pin_memory()
-        hn = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
-        sd = L.deer_step_dev(vs.q.data_ptr(), vs.k_blk.data_ptr(), vs.v_blk.data_ptr(), vs.attn_out.data_ptr(), vs.h.data_ptr(),
-                             vs.seq_ids.data_ptr(), vs.draft_ids.data_ptr(), vs.target_ids.data_ptr(), vs.accept_len.data_ptr(),
-                             vs.out_ids.data_ptr(), vs.n_out.data_ptr(), vs.attn_ws.data_ptr(), vs.attn_ws.numel(),
+        hout = torch.empty(2 * cfg.B + cfg.M, dtype=torch.int32).pin_memory()
+        ha, ho, hn = hout[:cfg.B], hout[cfg.B:cfg.B + cfg.M].view(cfg.B, cfg.k), hout[cfg.B + cfg.M:]
+        din = torch.empty(nq + 2 * nk, dtype=torch.bfloat16, device=dev)
+        dout = torch.empty(2 * cfg.B + cfg.M, dtype=torch.int32, device=dev)
+        sd = L.deer_step_dev(din.data_ptr(), din[nq:].data_ptr(), din[nq + nk:].data_ptr(), vs.attn_out.data_ptr(), vs.h.data_ptr(),
+                             vs.seq_ids.data_ptr(), vs.draft_ids.data_ptr(), vs.target_ids.data_ptr(), dout.data_ptr(),
+                             dout[cfg.B:].data_ptr(), dout[cfg.B + cfg.M:].data_ptr(), vs.attn_ws.data_ptr(), vs.attn_ws.numel(),
                              vs.lm_ws.data_ptr(), vs.lm_ws.numel())
         h2d = sum(t.numel() * t.element_size() for t in (hq, hkb, hvb, hh, hd))
         d2h = sum(t.numel() * t.element_size() for t in (ha, ho, hn))

@@ -455,6 +455,9 @@ int deer_moe_mlp(const void* x, const void* w_router, const void* w_gate_up, con
  * pointer and size of `kv`'s descriptor, of `dev` and of the argument list is
  * part of that key, so swapping any buffer records a new graph.  Not to be
  * called on a stream that is being captured.
+ * Buffers that follow one another in memory on both the host and the device
+ * side -- q, k_blk, v_blk in that order; accept_len, out_ids, n_out in that
+ * order -- are moved by one copy instead of three.
  * ---------------------------------------------------------------------- */
 typedef struct deer_step_dev {
     void* q; void* k_blk; void* v_blk; void* attn_out;     /* bf16 staging, shapes as in deer_block_attn */

@@ -16,6 +16,8 @@
 
 #include <mutex>
 
+#include <cuda.h>
+
 #include "common.cuh"
 
 namespace {
@@ -63,6 +65,26 @@ int side_stream() {
     return DEER_OK;
 }
 
+// True when [p, p + bytes) lies inside one allocation (host or device): a single copy must not cross from one
+// allocation into a neighbour that merely happens to follow it in the address space.
+bool one_allocation(const void* p, size_t bytes) {
+    typedef CUresult (*range_fn)(CUdeviceptr*, size_t*, CUdeviceptr);
+    static range_fn fn = [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuMemGetAddressRange", &f, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess)
+            f = nullptr;
+        cudaGetLastError();
+        return reinterpret_cast<range_fn>(f);
+    }();
+    if (!fn) return false;
+    CUdeviceptr base = 0;
+    size_t size = 0;
+    if (fn(&base, &size, reinterpret_cast<CUdeviceptr>(p)) != CUDA_SUCCESS) return false;
+    const CUdeviceptr a = reinterpret_cast<CUdeviceptr>(p);
+    return a >= base && a + bytes <= base + size;
+}
+
 int enqueue(deer_kv* kv, const deer_step_dev* dev, const void* w, const void* q_host, const void* k_blk_host,
             const void* v_blk_host, const void* h_host, const int32_t* draft_ids_host, int B, int k, int Hq, int hid, int V,
             float scale, int max_seq_len, int32_t* accept_len_host, int32_t* out_ids_host, int32_t* n_out_host, void* stream,
@@ -83,9 +105,18 @@ int enqueue(deer_kv* kv, const deer_step_dev* dev, const void* w, const void* q_
     DEER_CUDA(cudaMemcpyAsync(dev->h, h_host, M * hid * 2, cudaMemcpyHostToDevice, sh));
     DEER_CUDA(cudaMemcpyAsync(dev->draft_ids, draft_ids_host, M * sizeof(int32_t), cudaMemcpyHostToDevice, sh));
     if (fork) DEER_CUDA(cudaEventRecord(g_join, g_side));
-    DEER_CUDA(cudaMemcpyAsync(dev->q, q_host, M * Hq * D * 2, cudaMemcpyHostToDevice, st));
-    DEER_CUDA(cudaMemcpyAsync(dev->k_blk, k_blk_host, M * Hkv * D * 2, cudaMemcpyHostToDevice, st));
-    DEER_CUDA(cudaMemcpyAsync(dev->v_blk, v_blk_host, M * Hkv * D * 2, cudaMemcpyHostToDevice, st));
+    // q, k_blk and v_blk go in one copy where they follow one another in memory on both sides
+    const size_t q_bytes = M * Hq * D * 2, kv_bytes = M * Hkv * D * 2;
+    auto at = [](const void* p, size_t off) { return static_cast<const char*>(p) + off; };
+    if (at(q_host, q_bytes) == k_blk_host && at(k_blk_host, kv_bytes) == v_blk_host && at(dev->q, q_bytes) == dev->k_blk &&
+        at(dev->k_blk, kv_bytes) == dev->v_blk && one_allocation(q_host, q_bytes + 2 * kv_bytes) &&
+        one_allocation(dev->q, q_bytes + 2 * kv_bytes)) {
+        DEER_CUDA(cudaMemcpyAsync(dev->q, q_host, q_bytes + 2 * kv_bytes, cudaMemcpyHostToDevice, st));
+    } else {
+        DEER_CUDA(cudaMemcpyAsync(dev->q, q_host, q_bytes, cudaMemcpyHostToDevice, st));
+        DEER_CUDA(cudaMemcpyAsync(dev->k_blk, k_blk_host, kv_bytes, cudaMemcpyHostToDevice, st));
+        DEER_CUDA(cudaMemcpyAsync(dev->v_blk, v_blk_host, kv_bytes, cudaMemcpyHostToDevice, st));
+    }
     rc = deer_kv_reserve(kv, dev->seq_ids, B, k, stream);
     if (rc != DEER_OK) return rc;
     rc = deer_block_attn(kv, dev->seq_ids, dev->q, dev->k_blk, dev->v_blk, dev->attn_out, B, k, Hq, DEER_MASK_CAUSAL, 1, scale,
@@ -98,9 +129,16 @@ int enqueue(deer_kv* kv, const deer_step_dev* dev, const void* w, const void* q_
     rc = deer_accept_commit(kv, dev->seq_ids, DEER_ACC_GREEDY, B, k, dev->draft_ids, dev->target_ids, -1, dev->accept_len,
                             dev->out_ids, dev->n_out, stream);
     if (rc != DEER_OK) return rc;
-    DEER_CUDA(cudaMemcpyAsync(accept_len_host, dev->accept_len, (size_t)B * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-    DEER_CUDA(cudaMemcpyAsync(out_ids_host, dev->out_ids, M * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-    DEER_CUDA(cudaMemcpyAsync(n_out_host, dev->n_out, (size_t)B * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    // and so do the three results on the way back
+    if (accept_len_host + B == out_ids_host && out_ids_host + M == n_out_host && dev->accept_len + B == dev->out_ids &&
+        dev->out_ids + M == dev->n_out && one_allocation(accept_len_host, (2 * (size_t)B + M) * sizeof(int32_t)) &&
+        one_allocation(dev->accept_len, (2 * (size_t)B + M) * sizeof(int32_t))) {
+        DEER_CUDA(cudaMemcpyAsync(accept_len_host, dev->accept_len, (2 * (size_t)B + M) * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    } else {
+        DEER_CUDA(cudaMemcpyAsync(accept_len_host, dev->accept_len, (size_t)B * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+        DEER_CUDA(cudaMemcpyAsync(out_ids_host, dev->out_ids, M * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+        DEER_CUDA(cudaMemcpyAsync(n_out_host, dev->n_out, (size_t)B * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    }
     return DEER_OK;
 }
 

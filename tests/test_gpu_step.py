@@ -174,11 +174,13 @@ def test_c5_sweep_points(B, ctx, k, mask):
         _greedy_step(cfg, stress=True, steps=3)
 
 
-@pytest.mark.parametrize("own_stream", [False, True])
-def test_host_buffer_step_matches_oracle(own_stream):
+@pytest.mark.parametrize("own_stream,adjacent", [(False, False), (True, False), (True, True), (False, True)])
+def test_host_buffer_step_matches_oracle(own_stream, adjacent):
     """deer_verify_step_host, four consecutive steps from pinned host buffers that are refilled in place: on the legacy
     default stream every call enqueues its copies and kernels one by one; on a stream of its own the first call
-    captures them into a graph and the later ones replay it.  Verdicts and cache state against the oracle."""
+    captures them into a graph and the later ones replay it.  With `adjacent`, q / k_blk / v_blk and the three results
+    are slices of one buffer on each side (the call then moves each group with one copy).  Verdicts and cache state
+    against the oracle."""
     from paper_2512_15176_b200 import binding as L
     from paper_2512_15176_b200.runner import VerifyStep
     steps = 4
@@ -192,15 +194,27 @@ def test_host_buffer_step_matches_oracle(own_stream):
     ids = np.arange(cfg.B)
     pin = lambda t: t.contiguous().pin_memory()
     q0, kb0, vb0 = Hn.draw_block(cfg, 0, True)
-    hq, hkb, hvb = pin(q0), pin(kb0), pin(vb0)
     hh = pin(torch.empty(cfg.M, cfg.hid, dtype=torch.bfloat16))
     hd = pin(torch.empty(cfg.B, cfg.k, dtype=torch.int32))
-    ha = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
-    ho = torch.empty(cfg.B, cfg.k, dtype=torch.int32).pin_memory()
-    hn = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
-    sd = L.deer_step_dev(vs.q.data_ptr(), vs.k_blk.data_ptr(), vs.v_blk.data_ptr(), vs.attn_out.data_ptr(), vs.h.data_ptr(),
-                         vs.seq_ids.data_ptr(), vs.draft_ids.data_ptr(), vs.target_ids.data_ptr(), vs.accept_len.data_ptr(),
-                         vs.out_ids.data_ptr(), vs.n_out.data_ptr(), vs.attn_ws.data_ptr(), vs.attn_ws.numel(),
+    if adjacent:
+        nq, nk = q0.numel(), kb0.numel()
+        hin = torch.empty(nq + 2 * nk, dtype=torch.bfloat16).pin_memory()
+        hq, hkb, hvb = hin[:nq].view_as(q0), hin[nq:nq + nk].view_as(kb0), hin[nq + nk:].view_as(vb0)
+        hout = torch.full((2 * cfg.B + cfg.M,), -7, dtype=torch.int32).pin_memory()
+        ha, ho, hn = hout[:cfg.B], hout[cfg.B:cfg.B + cfg.M].view(cfg.B, cfg.k), hout[cfg.B + cfg.M:]
+        din = torch.empty(nq + 2 * nk, dtype=torch.bfloat16, device="cuda")
+        dout = torch.empty(2 * cfg.B + cfg.M, dtype=torch.int32, device="cuda")
+        dq, dk, dv = din, din[nq:], din[nq + nk:]
+        da, do, dn = dout, dout[cfg.B:], dout[cfg.B + cfg.M:]
+    else:
+        hq, hkb, hvb = pin(q0), pin(kb0), pin(vb0)
+        ha = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
+        ho = torch.empty(cfg.B, cfg.k, dtype=torch.int32).pin_memory()
+        hn = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
+        dq, dk, dv, da, do, dn = vs.q, vs.k_blk, vs.v_blk, vs.accept_len, vs.out_ids, vs.n_out
+    sd = L.deer_step_dev(dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), vs.attn_out.data_ptr(), vs.h.data_ptr(),
+                         vs.seq_ids.data_ptr(), vs.draft_ids.data_ptr(), vs.target_ids.data_ptr(), da.data_ptr(),
+                         do.data_ptr(), dn.data_ptr(), vs.attn_ws.data_ptr(), vs.attn_ws.numel(),
                          vs.lm_ws.data_ptr(), vs.lm_ws.numel())
     stream = torch.cuda.Stream() if own_stream else None
     torch.cuda.synchronize()
