@@ -484,7 +484,7 @@ int launch_grouped(const void* xs, size_t slots, const void* w, int E, int K, in
     a.a_bytes = a.x_box_rows * 128;
     a.stage_bytes = a.a_bytes + G_W_BYTES;
     if (a.stage_bytes < G_A_SPAN) a.stage_bytes = G_A_SPAN;
-    a.stages = (200 * 1024) / a.stage_bytes;
+    a.stages = (108 * 1024) / a.stage_bytes;            // two blocks per SM: one streams while the other starts or drains
     if (a.stages > G_MAX_STAGES) a.stages = G_MAX_STAGES;
     a.out = out;
     a.status = status;
