@@ -128,6 +128,12 @@ int deer_accept_commit(deer_kv* kv, const int32_t* seq_ids, int mode, int B, int
  * and reset it to 0 on the device. */
 int deer_kv_status(deer_kv* kv, int32_t* code, void* stream);
 
+/* Self-test of the bounded waits (no counterpart in the paper): one thread block waits on a barrier that nothing
+ * arrives on, with the same wait the tensor-core kernels use; the wait gives up after its limit (about a second of
+ * SM clocks), the block raises DEER_ERR_TIMEOUT in the cache's status word and returns, and the context stays
+ * usable.  Asynchronous on `stream`; read the outcome with deer_kv_status(). */
+int deer_selftest_bounded_wait(deer_kv* kv, void* stream);
+
 /* ------------------------------------------------------------------------
  * (1) Block attention (Section 3.2: the verifier scores all k block
  * positions in one pass, p_AR(. | x_{1:j+i-1}); the drafter fills the k masked

@@ -24,7 +24,7 @@ DEER_ACC_GREEDY, DEER_ACC_SAMPLE, DEER_ACC_SAMPLE_PRESTATS, DEER_ACC_BONUS = 0, 
 DEER_EMIT_PENDING = 1
 
 EXPORTS = [
-    "deer_last_error", "deer_kv_create", "deer_kv_destroy", "deer_kv_reserve", "deer_kv_commit", "deer_accept_commit", "deer_kv_status",
+    "deer_last_error", "deer_kv_create", "deer_kv_destroy", "deer_kv_reserve", "deer_kv_commit", "deer_accept_commit", "deer_kv_status", "deer_selftest_bounded_wait",
     "deer_block_attn_workspace_bytes", "deer_block_attn", "deer_lmhead_workspace_bytes", "deer_lmhead_select",
     "deer_accept_workspace_bytes", "deer_accept", "deer_verify_step_host",
     "deer_lmhead_static_max_rows", "deer_lmhead_select_static", "deer_emit", "deer_draft_stats",
@@ -76,6 +76,7 @@ def lib() -> ctypes.CDLL:
     L.deer_accept_commit.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_void_p, c_int32, c_void_p, c_void_p,
                                      c_void_p, c_void_p]
     L.deer_kv_status.argtypes = [c_void_p, POINTER(c_int32), c_void_p]
+    L.deer_selftest_bounded_wait.argtypes = [c_void_p, c_void_p]
     L.deer_block_attn_workspace_bytes.restype = c_size_t
     L.deer_block_attn_workspace_bytes.argtypes = [c_int] * 6
     L.deer_block_attn.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_int,
@@ -199,6 +200,10 @@ class KVCache:
 
 def deer_kv_reserve(kv: KVCache, seq_ids: torch.Tensor, k: int, stream=None) -> None:
     _check(lib().deer_kv_reserve(kv.handle, _ptr(seq_ids), seq_ids.numel(), k, _stream(stream)))
+
+
+def deer_selftest_bounded_wait(kv: KVCache, stream=None) -> None:
+    _check(lib().deer_selftest_bounded_wait(kv.handle, _stream(stream)))
 
 
 def deer_kv_commit(kv: KVCache, seq_ids: torch.Tensor, keep: torch.Tensor, k: int, stream=None) -> None:

@@ -823,3 +823,28 @@ int launch_umma(AttnParams p, cudaStream_t st) {
 }
 
 }  // namespace attn
+
+// ---- self-test of the bounded waits ------------------------------------------------------------
+namespace {
+__global__ void bounded_wait_selftest_kernel(int32_t* status) {
+    __shared__ uint64_t bar_word;
+    __shared__ int abort_flag;
+    const uint32_t bar = smem_u32(&bar_word);
+    if (threadIdx.x == 0) {
+        sm100::mbar_init(bar, 1);                 // one arrival expected; none will come
+        abort_flag = 0;
+        sm100::mbar_init_fence();
+    }
+    __syncthreads();
+    const bool got = sm100::mbar_wait(bar, 0u, &abort_flag);    // every thread waits, as a kernel's warps do
+    __syncthreads();
+    if (threadIdx.x == 0 && !got && abort_flag) deer_report(status, DEER_ERR_TIMEOUT);
+}
+}  // namespace
+
+extern "C" int deer_selftest_bounded_wait(deer_kv* kv, void* stream) {
+    DEER_CHECK_ARG(kv, DEER_ERR_INVALID_ARG, "deer_selftest_bounded_wait: null argument");
+    bounded_wait_selftest_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(kv->d.status);
+    DEER_CUDA(cudaGetLastError());
+    return DEER_OK;
+}

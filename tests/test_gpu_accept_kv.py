@@ -249,3 +249,24 @@ def test_reserve_without_pages_reports_and_changes_nothing():
     L.deer_kv_reserve(kv, torch.arange(3, dtype=torch.int32, device="cuda"), 32)
     assert L.deer_kv_status(kv) == L.DEER_ERR_NO_PAGES
     assert torch.equal(kv.page_table, before[0]) and torch.equal(kv.n_pages, before[1]) and torch.equal(kv.free_top, before[2])
+
+
+def test_bounded_wait_gives_up_and_reports():
+    """The wait every tensor-core kernel uses, on a barrier nothing arrives on: it gives up after its limit (about a
+    second), the status word says so, and the context goes on working."""
+    import time
+    from paper_2512_15176_b200 import binding as L
+    cfg = W.StepConfig("bw", 2, 4, 2, 64, 4, 64, 64, (8, 8), seed=990)
+    st = Hn.draw_state(cfg)
+    kv = Hn.gpu_kv(st)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    L.deer_selftest_bounded_wait(kv)
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    assert 0.2 < dt < 10.0, dt
+    assert L.deer_kv_status(kv) == L.DEER_ERR_TIMEOUT
+    assert L.deer_kv_status(kv) == 0
+    L.deer_kv_reserve(kv, torch.arange(2, dtype=torch.int32, device="cuda"), 4)
+    torch.cuda.synchronize()
+    assert L.deer_kv_status(kv) == 0
