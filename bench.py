@@ -399,7 +399,7 @@ def measure(cfg, steps, warmup, dev, peaks, flush, world=1, rank=0, with_e2e=Fal
     status = L.deer_kv_status(kv)
     accepted = int(vs.accept_len.sum().item()) if not bidir else None
 
-    # ---- end to end: host buffers in, verdict out, every step (the greedy verify step has such a call) ----
+    # ---- end to end: host buffers in, results out, every step (the greedy verify step has such a call) ----
     e2e_s, h2d, d2h = 0.0, 0, 0
     if greedy and with_e2e:
         pin = lambda t: t.contiguous().pin_memory()

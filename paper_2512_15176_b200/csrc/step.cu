@@ -1,6 +1,6 @@
 // One greedy verify step driven from host buffers: the end-to-end form of
 // Algorithm 1's loop body on the verifier side (copy the block in, score it,
-// accept, commit, copy the verdict out).
+// accept, commit, copy the results out).
 //
 // The five copies in, eight kernels and three copies out are sixteen
 // enqueue calls; issued one by one they cost more host time than the copies

@@ -179,7 +179,7 @@ def test_host_buffer_step_matches_oracle(own_stream, adjacent):
     """deer_verify_step_host, four consecutive steps from pinned host buffers that are refilled in place: on the legacy
     default stream every call enqueues its copies and kernels one by one; on a stream of its own the first call
     captures them into a graph and the later ones replay it.  With `adjacent`, q / k_blk / v_blk and the three results
-    are slices of one buffer on each side (the call then moves each group with one copy).  Verdicts and cache state
+    are slices of one buffer on each side (the call then moves each group with one copy).  Results and cache state
     against the oracle."""
     from paper_2512_15176_b200 import binding as L
     from paper_2512_15176_b200.runner import VerifyStep
