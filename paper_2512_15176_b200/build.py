@@ -42,17 +42,26 @@ def _headers_mtime() -> float:
     return max(os.path.getmtime(h) for h in hs)
 
 
-def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False) -> str:
-    os.makedirs(BUILD, exist_ok=True)
+PROBES_LIB = os.path.join(HERE, "libdeer_probes.so")
+
+
+def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False, probes: bool = False) -> str:
+    """Build the library; with ``probes`` a second one, ``libdeer_probes.so``, compiled with DEER_TIMING_PROBES (the
+    kernels then record clock values at the hand-overs of their pipelines; see ``profile_case.py --probes``)."""
+    build_dir = BUILD + ("_probes" if probes else "")
+    lib = PROBES_LIB if probes else LIB
+    os.makedirs(build_dir, exist_ok=True)
     nvcc = _nvcc()
     hm = _headers_mtime()
     flags = list(NVCC_FLAGS)
+    if probes:
+        flags += ["-DDEER_TIMING_PROBES"]
     if ptxas_info:
         flags += ["-Xptxas", "-v"]
     jobs = []
     objs = []
     for src in sources():
-        obj = os.path.join(BUILD, os.path.basename(src)[:-3] + ".o")
+        obj = os.path.join(build_dir, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
         if force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), hm):
             jobs.append([nvcc, *flags, "-c", src, "-o", obj])
@@ -66,10 +75,10 @@ def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False) 
 
     with ThreadPoolExecutor(max_workers=min(8, max(1, len(jobs)))) as ex:
         list(ex.map(run, jobs))
-    if jobs or not os.path.exists(LIB):
-        run([nvcc, "-shared", "-o", LIB, *objs])
-    return LIB
+    if jobs or not os.path.exists(lib):
+        run([nvcc, "-shared", "-o", lib, *objs])
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, ptxas_info="--ptxas" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, ptxas_info="--ptxas" in sys.argv, probes="--probes" in sys.argv))

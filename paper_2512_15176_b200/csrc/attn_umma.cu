@@ -38,8 +38,18 @@
 #include "attn.cuh"
 #include "sm100.cuh"
 
+#ifdef DEER_TIMING_PROBES
+// Probe table of the attention kernel: row = tile index of block PROBE_BLOCK minus PROBE_TILE0, columns:
+// 0 slot free seen by the producer, 1 K landed seen by the S issuer, 2 S committed, 3 S complete seen by the softmax,
+// 4 P handed over, 5 P and V seen by the O issuer, 6 O committed.
+__device__ long long g_attn_probe[DEER_PROBE_ROWS][DEER_PROBE_COLS];
+extern "C" int deer_attn_probe_read(long long* host) {
+    return (int)cudaMemcpyFromSymbol(host, g_attn_probe, sizeof(g_attn_probe));
+}
+#endif
 namespace attn {
 namespace umma {
+constexpr int PROBE_BLOCK = 20, PROBE_TILE0 = 40;      // which block and which of its tiles the probes record
 
 using namespace sm100;
 
@@ -304,6 +314,7 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     int oks = 1;
                     if (lane == 0) oks = mbar_wait(bar(BAR_SLOT_EMPTY + sl), ((uint32_t)(it / NSLOT) & 1u) ^ 1u, abort_flag) ? 1 : 0;
                     if (!__shfl_sync(0xffffffffu, oks, 0)) { ok = false; break; }
+                    DEER_PROBE(g_attn_probe, lane == 0 && blockIdx.x == PROBE_BLOCK, it - PROBE_TILE0, 0);
                     const uint32_t kdst = ring_addr + sl * SLOT_BYTES;
                     const uint32_t dst = is_v ? kdst + K_BYTES : kdst;
                     const uint32_t fb = bar((is_v ? BAR_V_FULL : BAR_K_FULL) + sl);
@@ -352,6 +363,7 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         // S buffer free (the softmax warps have read its previous tile), K tile landed
                         if (!mbar_wait(bar(BAR_S_FREE + sb), ((uint32_t)(it / NS) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
                         if (!mbar_wait(bar(BAR_K_FULL + sl), (uint32_t)(it / NSLOT) & 1u, abort_flag)) { ok = false; break; }
+                        DEER_PROBE(g_attn_probe, blockIdx.x == PROBE_BLOCK, it - PROBE_TILE0, 1);
                         tcgen05_fence_after();
                         const uint32_t d_tmem = tmem_base + (uint32_t)(sb * ATT_TILE);
                         const bool blk = (t == last_tile);
@@ -364,6 +376,7 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                             umma_bf16_ss(d_tmem, ad, bd, idesc_qk, kk != 0 ? 1u : 0u);
                         }
                         umma_commit(bar(BAR_S_FULL + sb));
+                        DEER_PROBE(g_attn_probe, blockIdx.x == PROBE_BLOCK, it - PROBE_TILE0, 2);
                     }
                     // Q buffer reusable once this warp's MMAs of the segment are done (the other S issuer says the same)
                     if (ok) umma_commit(bar(BAR_Q_EMPTY + qb));
@@ -383,6 +396,7 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         const int sl = it % NSLOT;
                         if (!mbar_wait(bar(BAR_P_READY + (it & 1)), (uint32_t)(it >> 1) & 1u, abort_flag)) { ok = false; break; }
                         if (!mbar_wait(bar(BAR_V_FULL + sl), (uint32_t)(it / NSLOT) & 1u, abort_flag)) { ok = false; break; }
+                        DEER_PROBE(g_attn_probe, blockIdx.x == PROBE_BLOCK, it - PROBE_TILE0, 5);
                         tcgen05_fence_after();
                         const uint32_t p_tmem = tmem_base + (uint32_t)(P_COL + (it & 1) * (ATT_TILE / 2));
                         const bool blk = (t == last_tile);
@@ -396,6 +410,7 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         // S of this tile was complete before its softmax, hence before this point: K and V are both consumed
                         umma_commit(bar(BAR_SLOT_EMPTY + sl));
                         umma_commit(bar(BAR_O_DONE));             // phase `it` of o_done: O includes this tile
+                        DEER_PROBE(g_attn_probe, blockIdx.x == PROBE_BLOCK, it - PROBE_TILE0, 6);
                     }
                 }
             }
@@ -448,6 +463,7 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     const int sb = it % NS, pb = it & 1, sl = it % NSLOT;
                     const bool got = mbar_wait(bar(BAR_S_FULL + sb), (uint32_t)(it / NS) & 1u, abort_flag);
                     if (!__all_sync(0xffffffffu, got)) { alive = false; break; }   // warp-uniform: the aligned TMEM ops stay converged
+                    DEER_PROBE(g_attn_probe, wtid == 0 && blockIdx.x == PROBE_BLOCK, it - PROBE_TILE0, 3);
                     tcgen05_fence_after();
                     uint32_t sr[ATT_TILE];
                     TMEM_LD_X32(t_lane + sb * ATT_TILE, (sr));
@@ -564,6 +580,7 @@ block_attn_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     tcgen05_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar(BAR_P_READY + pb));
+                    DEER_PROBE(g_attn_probe, wtid == 0 && blockIdx.x == PROBE_BLOCK, it - PROBE_TILE0, 4);
                 }
                 if (!alive) break;
 

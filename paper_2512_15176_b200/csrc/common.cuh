@@ -126,3 +126,20 @@ __device__ __forceinline__ void deer_report(int32_t* status, int32_t code) {
 }
 
 #endif  // __CUDACC__
+
+// ---- timing probes (measurement builds only) -----------------------------------------
+// `python -m paper_2512_15176_b200.build --probes` compiles the library a second time with DEER_TIMING_PROBES
+// defined (libdeer_probes.so): a few kernels then record SM clock values at the hand-overs of their pipelines, for
+// `profile_case.py --probes` to read.  Nothing is skipped or reordered; without the define the macros vanish.
+#ifdef DEER_TIMING_PROBES
+#define DEER_PROBE_ROWS 64
+#define DEER_PROBE_COLS 8
+#define DEER_PROBE(table, on, row, col)                                                     \
+    do {                                                                                    \
+        if ((on) && (row) >= 0 && (row) < DEER_PROBE_ROWS) (table)[(row)][(col)] = clock64(); \
+    } while (0)
+#else
+#define DEER_PROBE(table, on, row, col) \
+    do {                                \
+    } while (0)
+#endif

@@ -28,6 +28,23 @@
 #include "lmhead.cuh"
 #include "sm100.cuh"
 
+#ifdef DEER_TIMING_PROBES
+// Per leader block of the block-pair kernel (row = block index, the first DEER_PROBE_ROWS of them): SM clocks the
+// MMA-issuing thread spent in all (0), waiting for operands (1), waiting for an accumulator (2); MMAs issued (3).
+__device__ long long g_lmhead_probe[DEER_PROBE_ROWS][DEER_PROBE_COLS];
+extern "C" int deer_lmhead_probe_read(long long* host) {
+    return (int)cudaMemcpyFromSymbol(host, g_lmhead_probe, sizeof(g_lmhead_probe));
+}
+#define LM_PROBE_T0(v) const long long v = clock64()
+#define LM_PROBE_ADD(acc, v) acc += clock64() - v
+#else
+#define LM_PROBE_T0(v) \
+    do {               \
+    } while (0)
+#define LM_PROBE_ADD(acc, v) \
+    do {                     \
+    } while (0)
+#endif
 namespace lmhead {
 namespace umma {
 
@@ -522,29 +539,51 @@ lmhead_umma_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
         if (leader && lane == 0 && n_tiles > 0) {
             int it = 0;
             bool ok = true;
+#ifdef DEER_TIMING_PROBES
+            long long w_full = 0, w_acc = 0, n_mma = 0;
+#endif
+            LM_PROBE_T0(t_begin);
             for (int t = 0; t < n_tiles && ok; ++t) {
                 int row0, g;
                 tile_span(tl, t, row0, g);
                 const uint32_t idesc = make_idesc_bf16_pair(g * 16);
                 const int buf = t & 1;
                 const uint32_t aph = (uint32_t)(t >> 1) & 1u;
+                LM_PROBE_T0(t_acc);
                 if (!mbar_wait(tempty_bar(buf), aph ^ 1u, abort_flag)) break;
+                LM_PROBE_ADD(w_acc, t_acc);
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * MAXN);
                 for (int kb = 0; kb < KB; ++kb, ++it) {
                     const int s = it % a.stages;
                     const uint32_t ph = (uint32_t)(it / a.stages) & 1u;
+                    LM_PROBE_T0(t_full);
                     if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+                    LM_PROBE_ADD(w_full, t_full);
                     tcgen05_fence_after();
                     const uint32_t sa = smem_base + s * stage_bytes;
                     const uint64_t ad = smem_desc_sw128_kmajor(sa), bd = smem_desc_sw128_kmajor(sa + A_SPAN);
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k)
                         umma_bf16_ss_pair(d_tmem, ad + 2 * k, bd + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+#ifdef DEER_TIMING_PROBES
+                    n_mma += BK / 16;
+#endif
                     umma_commit_pair(empty_bar(s), 3);
                 }
                 if (ok) umma_commit_pair(tfull_bar(buf), 3);
             }
+#ifdef DEER_TIMING_PROBES
+            {
+                const int bi = (int)(blockIdx.y * gridDim.x + blockIdx.x) >> 1;       // leader blocks, in launch order
+                if (bi < DEER_PROBE_ROWS) {
+                    g_lmhead_probe[bi][0] = clock64() - t_begin;
+                    g_lmhead_probe[bi][1] = w_full;
+                    g_lmhead_probe[bi][2] = w_acc;
+                    g_lmhead_probe[bi][3] = n_mma;
+                }
+            }
+#endif
         }
     } else {
         // ---------------- epilogue: 4 warps in each block, one TMEM lane quarter each ----------------

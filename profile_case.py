@@ -10,6 +10,11 @@ program that profiler captures are taken from.
 
 Prints the average CUDA-event time per call and the achieved GB/s over the
 call's algorithmic bytes.
+
+With --probes (attn, lmhead) the calls run on the library built with timing probes
+(`python -m paper_2512_15176_b200.build --probes`): the attention kernel records SM clock values at the hand-overs of
+its pipeline for 64 tiles of one thread block, the block-pair LM head what its MMA-issuing thread's time goes to, and
+the tables are printed after the timing line (times with probes are a little longer than without).
 """
 from __future__ import annotations
 
@@ -52,7 +57,11 @@ def main():
     ap.add_argument("--bidir", action="store_true")
     ap.add_argument("--iters", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=1)
+    ap.add_argument("--probes", action="store_true", help="attn, lmhead: run on the library built with timing probes and print them")
     a = ap.parse_args()
+    if a.probes:
+        from paper_2512_15176_b200 import build as B_
+        L.LIB_PATH = B_.build(probes=True)
     dev = "cuda"
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     flush_rd = torch.zeros(64 << 20, dtype=torch.int32, device=dev)
@@ -187,6 +196,39 @@ def main():
     ms = float(np.mean([e0.elapsed_time(e1) for e0, e1 in ev]))
     print(f"{a.what}: {ms * 1e3:.1f} us/call, {nbytes / ms / 1e6:.1f} GB/s over {nbytes} algorithmic bytes, "
           f"{flops / ms / 1e9:.1f} TFLOP/s")
+    if a.probes:
+        print_probes(a.what)
+
+
+def print_probes(what: str) -> None:
+    """The probe tables of the last call (library built with DEER_TIMING_PROBES)."""
+    import ctypes
+    lib = L.lib()
+    buf = (ctypes.c_longlong * (64 * 8))()
+    if what == "attn":
+        lib.deer_attn_probe_read.argtypes = [ctypes.c_void_p]
+        lib.deer_attn_probe_read(buf)
+        d = np.array(buf[:], dtype=np.int64).reshape(64, 8)
+        d = d[(d[:, :7] > 0).all(axis=1)]
+        if len(d) < 8:
+            print("probes: the probed block had too few tiles")
+            return
+        names = ["slot free seen", "K landed seen", "S committed", "S complete seen", "P handed over", "P+V seen", "O committed"]
+        print(f"probes: {len(d)} tiles of one block; tile period {np.median(np.diff(d[:, 0])):.0f} cycles (median)")
+        for j in range(6):
+            print(f"  {names[j]:16s} -> {names[j + 1]:16s} {np.median(d[:, j + 1] - d[:, j]):7.0f} cycles")
+        print(f"  {names[6]:16s} -> {names[0]:16s} {np.median(d[4:, 0] - d[:-4, 6]):7.0f} cycles (four tiles on: the ring's depth)")
+    elif what == "lmhead":
+        lib.deer_lmhead_probe_read.argtypes = [ctypes.c_void_p]
+        lib.deer_lmhead_probe_read(buf)
+        d = np.array(buf[:], dtype=np.int64).reshape(64, 8)
+        d = d[d[:, 3] > 0]
+        if len(d) == 0:
+            print("probes: the block-pair kernel did not run (M <= 128)")
+            return
+        print(f"probes: {len(d)} leader blocks; {d[:, 3].mean():.0f} MMAs each, {(d[:, 0] / d[:, 3]).mean():.1f} cycles per MMA; "
+              f"waiting for operands {100 * (d[:, 1] / d[:, 0]).mean():.1f} %, for an accumulator {100 * (d[:, 2] / d[:, 0]).mean():.1f} %, "
+              f"issuing {100 * (1 - (d[:, 1] + d[:, 2]) / d[:, 0]).mean():.1f} %")
 
 
 if __name__ == "__main__":
