@@ -72,6 +72,22 @@ __global__ void __launch_bounds__(128) qk_norm_rope_kernel(deer_kv_desc kv, cons
         const long long bi = r / Hkv;
         const int hh = (int)(r % Hkv);
         const long long src = (bi * (Hq + 2 * Hkv) + Hq + Hkv + hh) * D;
+        if (part && D <= 128) {
+            // this lane's (up to four) columns of every partial product together, four partial products in flight:
+            // one column and one partial product at a time would put their load latencies end to end
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
+            for (int s = 0; s < ksplit; ++s) {
+                const float* ps = part + (long long)s * part_stride + src;
+#pragma unroll
+                for (int t = 0; t < 4; ++t)
+                    if (lane + 32 * t < D) acc[t] += ps[lane + 32 * t];
+            }
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+                if (lane + 32 * t < D) vb[r * D + lane + 32 * t] = __float2bfloat16(acc[t]);
+            return;
+        }
         for (int d = lane; d < D; d += 32) vb[r * D + d] = __float2bfloat16(packed_at(src + d));
         return;
     }
