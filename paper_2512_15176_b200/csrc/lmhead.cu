@@ -30,10 +30,20 @@ __global__ void __launch_bounds__(256) lmhead_finalize_kernel(FinalizeArgs a) {
     float rm = -INFINITY, rs = 0.f;
     int32_t ri = 0x7fffffff;
     bool aborted = false;
-    for (int pt = lane; pt < a.nparts; pt += 32) {
-        const Partial pr = a.part[(size_t)pt * a.M + m];
-        aborted |= (pr.idx == PARTIAL_ABORTED);
-        merge_sel(rm, ri, rs, pr.m, pr.idx, pr.s, a.inv_t_log2);
+    // a lane's partials are requested together (one after the other their latencies would add up), then merged
+    for (int pt0 = lane; pt0 < a.nparts; pt0 += 32 * 8) {
+        Partial pr[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int pt = pt0 + 32 * j;
+            if (pt < a.nparts) pr[j] = a.part[(size_t)pt * a.M + m];
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (pt0 + 32 * j >= a.nparts) break;
+            aborted |= (pr[j].idx == PARTIAL_ABORTED);
+            merge_sel(rm, ri, rs, pr[j].m, pr[j].idx, pr[j].s, a.inv_t_log2);
+        }
     }
     aborted = __any_sync(0xffffffffu, aborted);
 #pragma unroll
