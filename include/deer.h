@@ -463,7 +463,8 @@ int deer_moe_mlp(const void* x, const void* w_router, const void* w_gate_up, con
  * called on a stream that is being captured.
  * Buffers that follow one another in memory on both the host and the device
  * side -- q, k_blk, v_blk in that order; accept_len, out_ids, n_out in that
- * order -- are moved by one copy instead of three.
+ * order -- are moved by one copy instead of three; in the recorded form the
+ * last kernel writes the results into the page-locked host buffers itself.
  * ---------------------------------------------------------------------- */
 typedef struct deer_step_dev {
     void* q; void* k_blk; void* v_blk; void* attn_out;     /* bf16 staging, shapes as in deer_block_attn */

@@ -127,6 +127,11 @@ __device__ __forceinline__ void deer_report(int32_t* status, int32_t code) {
 
 #endif  // __CUDACC__
 
+// ---- calls between the library's own files (not part of the C ABI) ----------------------
+int deer_accept_commit_mirrored(deer_kv* kv, const int32_t* seq_ids, int mode, int B, int k, const int32_t* draft_ids,
+                                const int32_t* target_ids, int32_t eos_id, int32_t* accept_len, int32_t* out_ids, int32_t* n_out,
+                                int32_t* mirror_accept_len, int32_t* mirror_out_ids, int32_t* mirror_n_out, void* stream);
+
 // ---- timing probes (measurement builds only) -----------------------------------------
 // `python -m paper_2512_15176_b200.build --probes` compiles the library a second time with DEER_TIMING_PROBES
 // defined (libdeer_probes.so): a few kernels then record SM clock values at the hand-overs of their pipelines, for

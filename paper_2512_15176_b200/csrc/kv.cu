@@ -184,11 +184,13 @@ kv_commit_kernel(deer_kv_desc d, const int32_t* __restrict__ seq_ids, const int3
 }
 
 // Greedy acceptance and the commit of what it accepted, one thread per sequence: the end of a greedy verify step in
-// one launch.
+// one launch.  The mirror_* pointers, when given, receive a second copy of the three results (page-locked host
+// memory the device can write: the host-buffer step then needs no copy back).
 __global__ void __launch_bounds__(KV_THREADS)
 kv_accept_commit_kernel(deer_kv_desc d, const int32_t* __restrict__ seq_ids, int B, int k, int kd, const int32_t* __restrict__ draft,
                         const int32_t* __restrict__ target, int32_t eos_id, int32_t* __restrict__ accept_len,
-                        int32_t* __restrict__ out_ids, int32_t* __restrict__ n_out) {
+                        int32_t* __restrict__ out_ids, int32_t* __restrict__ n_out, int32_t* __restrict__ mirror_accept_len,
+                        int32_t* __restrict__ mirror_out_ids, int32_t* __restrict__ mirror_n_out) {
     __shared__ int warp_sums[32];
     __shared__ int total;
     const int b = threadIdx.x;
@@ -200,6 +202,12 @@ kv_accept_commit_kernel(deer_kv_desc d, const int32_t* __restrict__ seq_ids, int
         a = greedy_accept_row(draft + (size_t)b * k, target + (size_t)b * k, out_ids + (size_t)b * k, k, kd, eos_id, &n);
         accept_len[b] = a;
         n_out[b] = n;
+        if (mirror_accept_len) {
+            mirror_accept_len[b] = a;
+            mirror_n_out[b] = n;
+            for (int i = 0; i < k; ++i) mirror_out_ids[(size_t)b * k + i] = out_ids[(size_t)b * k + i];
+            __threadfence_system();
+        }
     }
     commit_rows(d, seq_ids, a, B, k, warp_sums, &total);
 }
@@ -223,9 +231,11 @@ extern "C" int deer_kv_commit(deer_kv* kv, const int32_t* seq_ids, const int32_t
     return DEER_OK;
 }
 
-extern "C" int deer_accept_commit(deer_kv* kv, const int32_t* seq_ids, int mode, int B, int k, const int32_t* draft_ids,
-                                  const int32_t* target_ids, int32_t eos_id, int32_t* accept_len, int32_t* out_ids, int32_t* n_out,
-                                  void* stream) {
+// deer_accept_commit with a second copy of the results written to mirror_* (all three or none; memory the device
+// can write, e.g. page-locked host memory).  Not part of the C ABI: the host-buffer step uses it.
+int deer_accept_commit_mirrored(deer_kv* kv, const int32_t* seq_ids, int mode, int B, int k, const int32_t* draft_ids,
+                                const int32_t* target_ids, int32_t eos_id, int32_t* accept_len, int32_t* out_ids, int32_t* n_out,
+                                int32_t* mirror_accept_len, int32_t* mirror_out_ids, int32_t* mirror_n_out, void* stream) {
     DEER_CHECK_ARG(kv && seq_ids && draft_ids && target_ids && accept_len && out_ids && n_out, DEER_ERR_INVALID_ARG,
                    "deer_accept_commit: null argument");
     DEER_CHECK_ARG((mode & ~DEER_ACC_BONUS) == DEER_ACC_GREEDY, DEER_ERR_UNSUPPORTED,
@@ -235,6 +245,14 @@ extern "C" int deer_accept_commit(deer_kv* kv, const int32_t* seq_ids, int mode,
     if (B == 0) return DEER_OK;
     const int kd = (mode & DEER_ACC_BONUS) ? k - 1 : k;
     DEER_CUDA(launch_pdl(kv_accept_commit_kernel, dim3(1), dim3(KV_THREADS), 0, static_cast<cudaStream_t>(stream), kv->d, seq_ids, B, k,
-                         kd, draft_ids, target_ids, eos_id, accept_len, out_ids, n_out));
+                         kd, draft_ids, target_ids, eos_id, accept_len, out_ids, n_out, mirror_accept_len, mirror_out_ids,
+                         mirror_n_out));
     return DEER_OK;
+}
+
+extern "C" int deer_accept_commit(deer_kv* kv, const int32_t* seq_ids, int mode, int B, int k, const int32_t* draft_ids,
+                                  const int32_t* target_ids, int32_t eos_id, int32_t* accept_len, int32_t* out_ids, int32_t* n_out,
+                                  void* stream) {
+    return deer_accept_commit_mirrored(kv, seq_ids, mode, B, k, draft_ids, target_ids, eos_id, accept_len, out_ids, n_out, nullptr,
+                                       nullptr, nullptr, stream);
 }

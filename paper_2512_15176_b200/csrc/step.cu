@@ -126,10 +126,22 @@ int enqueue(deer_kv* kv, const deer_step_dev* dev, const void* w, const void* q_
     rc = deer_lmhead_select(dev->h, w, (int)M, hid, V, DEER_SEL_ARGMAX, 1.f, nullptr, dev->target_ids, nullptr, nullptr, nullptr,
                             nullptr, dev->lm_ws, dev->lm_ws_bytes, stream);
     if (rc != DEER_OK) return rc;
+    // In the recorded form (page-locked result buffers, which the device can write) the last kernel leaves a second
+    // copy of the results in the host buffers itself; otherwise they are copied back, in one piece where they follow
+    // one another inside one allocation on both sides.
+    if (fork) {
+        void *ma = nullptr, *mo = nullptr, *mn = nullptr;        // the host buffers as the device addresses them
+        if (cudaHostGetDevicePointer(&ma, accept_len_host, 0) == cudaSuccess && cudaHostGetDevicePointer(&mo, out_ids_host, 0) == cudaSuccess &&
+            cudaHostGetDevicePointer(&mn, n_out_host, 0) == cudaSuccess) {
+            return deer_accept_commit_mirrored(kv, dev->seq_ids, DEER_ACC_GREEDY, B, k, dev->draft_ids, dev->target_ids, -1,
+                                               dev->accept_len, dev->out_ids, dev->n_out, static_cast<int32_t*>(ma),
+                                               static_cast<int32_t*>(mo), static_cast<int32_t*>(mn), stream);
+        }
+        cudaGetLastError();
+    }
     rc = deer_accept_commit(kv, dev->seq_ids, DEER_ACC_GREEDY, B, k, dev->draft_ids, dev->target_ids, -1, dev->accept_len,
                             dev->out_ids, dev->n_out, stream);
     if (rc != DEER_OK) return rc;
-    // and so do the three results on the way back
     if (accept_len_host + B == out_ids_host && out_ids_host + M == n_out_host && dev->accept_len + B == dev->out_ids &&
         dev->out_ids + M == dev->n_out && one_allocation(accept_len_host, (2 * (size_t)B + M) * sizeof(int32_t)) &&
         one_allocation(dev->accept_len, (2 * (size_t)B + M) * sizeof(int32_t))) {
