@@ -398,6 +398,15 @@ def measure(cfg, steps, warmup, dev, peaks, flush, world=1, rank=0, with_e2e=Fal
         marks.append([ev_ph[0].elapsed_time(ev_ph[i]) for i in (1, 2, 3)])
     status = L.deer_kv_status(kv)
     accepted = int(vs.accept_len.sum().item()) if not bidir else None
+    # The drafts were planted against the head's own argmax, so the accepted lengths of the timed steps must be the
+    # planted prefix lengths: what was timed did the work.
+    planted_ok = None
+    if greedy and not bidir:
+        last = steps - 1 if step_drafts is not None else 0
+        want = W.planted_prefix_lengths(cfg, last) if step_drafts is not None else W.planted_prefix_lengths(cfg)
+        planted_ok = bool((vs.accept_len.cpu().numpy() == want).all())
+        if not planted_ok:
+            raise RuntimeError(f"{cfg.name}: accepted lengths differ from the planted prefix lengths")
 
     # ---- end to end: host buffers in, results out, every step (the greedy verify step has such a call) ----
     e2e_s, h2d, d2h = 0.0, 0, 0
@@ -432,6 +441,8 @@ def measure(cfg, steps, warmup, dev, peaks, flush, world=1, rank=0, with_e2e=Fal
             dt = time.perf_counter() - t0
             if s >= 3:
                 e2e_s += dt
+        if not (ha.numpy() == W.planted_prefix_lengths(cfg)).all():
+            raise RuntimeError(f"{cfg.name}: the host-buffer step's accepted lengths differ from the planted prefix lengths")
     clocks = clock_sampler.stop() if clock_sampler is not None else None
     total_s, e2e_total = max_over_ranks([float(sum(step_ms)) / 1e3, e2e_s], dev, world)
 
@@ -466,7 +477,8 @@ def measure(cfg, steps, warmup, dev, peaks, flush, world=1, rank=0, with_e2e=Fal
                    "lmhead_ms": lm_s * 1e3, "lmhead_gbs": ab["lmhead"] / lm_s / 1e9, "lmhead_tflops": fl["lmhead"] / lm_s / 1e12,
                    "accept_commit_ms": acc_s * 1e3, "step_ms_with_phase_events": float(m[:, 2].mean())},
         "gpu_launches": steps * vs.launches_per_step(),
-        "kv_status": status, "accepted_tokens_last_step": accepted, "wall_s_timed_loop": wall,
+        "kv_status": status, "accepted_tokens_last_step": accepted, "accepted_equals_planted": planted_ok,
+        "wall_s_timed_loop": wall,
         "consecutive_steps": bool(step_drafts is not None),
         "flops_per_step": fl["total"], "clocks": clocks,
     }
@@ -591,7 +603,8 @@ def run_ours(args, cfg):
         "e2e": head.get("e2e", {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
                                 "note": "the host-buffer entry point covers the greedy verify step only"}),
         "gpu_launches": head["gpu_launches"], "clocks": head["clocks"], "kv_status": head["kv_status"],
-        "accepted_tokens_last_step": head["accepted_tokens_last_step"], "wall_s_timed_loop": head["wall_s_timed_loop"],
+        "accepted_tokens_last_step": head["accepted_tokens_last_step"], "accepted_equals_planted": head["accepted_equals_planted"],
+        "wall_s_timed_loop": head["wall_s_timed_loop"],
         "flops_per_step": head["flops_per_step"],
     }
     if others:
